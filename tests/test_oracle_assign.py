@@ -1,0 +1,317 @@
+"""Pins for the oracle's layout tables and Algorithm 1 (CPU only).
+
+None of these re-types the oracle's formula: they use the paper's Fig. 1 layout with values
+derived by hand, an exhaustive enumeration of Eq. 1, invariants, and special cases.
+"""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle as O
+import workloads as W
+from conftest import golden_lines
+
+
+# ---------------------------------------------------------------- hash -------------------
+def test_hash_vectors():
+    n_checked = 0
+    for f in golden_lines("hash_vectors.txt"):
+        seed, t, e, stream = int(f[0]), int(f[1]), int(f[2]), int(f[3])
+        x = int(f[5], 16)
+        assert O.hash32(seed, t, e, stream) == x
+        assert [O.hash_index(x, n) for n in (2, 3, 8)] == [int(v) for v in f[6:9]]
+        n_checked += 1
+    assert n_checked == 5
+
+
+@pytest.mark.parametrize("n", [2, 3, 5, 8])
+@pytest.mark.parametrize("stream", [0, 1])
+def test_hash_index_uniform(n, stream):
+    """'Uniformly sample' (Section 3.3, Step 2): chi-square of the index over many (t, e)."""
+    counts = np.zeros(n)
+    draws = 0
+    for seed in (1, 36959):
+        for t in range(4000):
+            for e in (0, 3, 200):
+                counts[O.hash_index(O.hash32(seed, t, e, stream), n)] += 1
+                draws += 1
+    chi2 = ((counts - draws / n) ** 2 / (draws / n)).sum()
+    # 99.99% quantile of chi2 with <= 7 dof is < 30
+    assert chi2 < 30.0, (counts, chi2)
+
+
+def test_hash_index_range_edges():
+    assert O.hash_index(0, 8) == 0
+    assert O.hash_index(0xFFFFFFFF, 8) == 7
+    assert O.hash_index(0xFFFFFFFF, 1) == 0
+    assert O.hash_index(0x80000000, 2) == 1
+    assert O.hash_index(0x7FFFFFFF, 2) == 0
+
+
+# ---------------------------------------------------------------- layout tables ----------
+def test_fig1_layout_tables(fig1):
+    g = fig1
+    N, Q, S, E = g["nodes"], g["ranks_per_node"], g["slots_per_rank"], g["experts"]
+    tab = O.layout_tables(N, Q, S, E, g["slot_expert"], g["primary_slot"])
+    assert tab["nodes_mask"].tolist() == g["nodes_mask"]
+    assert tab["primary"].tolist() == g["primary_slot"]
+    assert tab["r_count"].sum(axis=1).tolist() == g["replica_count"]
+    for (e, n), slots in g["r_list"].items():
+        assert tab["r_count"][e, n] == len(slots)
+        assert tab["r_list"][e, n, :len(slots)].tolist() == slots
+
+
+def test_layout_default_primary_is_lowest_slot(fig1):
+    g = fig1
+    tab = O.layout_tables(2, 2, 2, 4, g["slot_expert"], None)
+    assert tab["primary"].tolist() == [0, 1, 2, 6]
+
+
+@pytest.mark.parametrize("slots,why", [
+    ([0, 1, 2, 0, 1, 2, 0, 0], "expert 3 has no replica (Eq. 2, first constraint)"),
+    ([0, 0, 2, 1, 1, 2, 3, 0], "expert 0 twice on rank 0"),
+    ([0, 1, 2, 0, 1, 2, 3, 4], "id out of range"),
+    ([0, 1, 2, 0, 1, 2, 3, -2], "negative id other than -1"),
+])
+def test_layout_rejects(slots, why):
+    with pytest.raises(O.OracleError):
+        O.layout_tables(2, 2, 2, 4, slots, None)
+
+
+def test_layout_rejects_primary_not_holding_expert(fig1):
+    with pytest.raises(O.OracleError):
+        O.layout_tables(2, 2, 2, 4, fig1["slot_expert"], [1, 4, 2, 6])
+
+
+def test_layout_accepts_empty_slots():
+    tab = O.layout_tables(2, 2, 2, 4, [0, -1, 1, -1, 2, -1, 3, 0], None)
+    assert tab["r_count"].sum(axis=1).tolist() == [2, 1, 1, 1]
+
+
+# ---------------------------------------------------------------- Fig. 1 worked example --
+def _fig1_inputs(g):
+    ids = np.array([tk["ids"] for tk in g["tokens"]], np.int32)
+    src = np.array([tk["src"] for tk in g["tokens"]], np.int32)
+    return ids, src
+
+
+@pytest.mark.parametrize("seed", [0, 1, 36959, 2**63 + 5])
+def test_fig1_assignment(fig1, seed):
+    g = fig1
+    ids, src = _fig1_inputs(g)
+    r = O.assign(2, 2, 2, 4, g["slot_expert"], g["primary_slot"], ids, src, seed)
+    assert r["remote_nodes"].tolist() == [tk["cobalt"] for tk in g["tokens"]]
+    assert r["V"] == g["V_cobalt"] and r["V_naive"] == g["V_naive"]
+    for t, k, slot in g["forced"]:
+        assert r["assigned_slot"][t, k] == slot
+    for t, k, allowed in g["free"]:
+        assert r["assigned_slot"][t, k] in allowed
+    assert r["slot_load"].sum() == ids.size
+    assert r["slot_load"][6] == 6          # d has one replica: all six tasks land on slot 6
+
+
+def test_fig1_seeded_picks(fig1):
+    g = fig1
+    ids, src = _fig1_inputs(g)
+    for seed, t, k, slot in g["seeded"]:
+        r = O.assign(2, 2, 2, 4, g["slot_expert"], g["primary_slot"], ids, src, seed)
+        assert r["assigned_slot"][t, k] == slot
+
+
+def test_fig1_naive_rule(fig1):
+    g = fig1
+    ids, src = _fig1_inputs(g)
+    r = O.assign(2, 2, 2, 4, g["slot_expert"], g["primary_slot"], ids, src, 7, naive=True)
+    assert r["remote_nodes"].tolist() == [tk["naive"] for tk in g["tokens"]]
+    assert r["V"] == g["V_naive"]
+    assert (r["assigned_slot"] == np.array(g["primary_slot"])[ids]).all()
+
+
+# ---------------------------------------------------------------- tie-break of lines 5-8 --
+def _layout_from_nodes(expert_nodes, N):
+    """One rank per node (Q = 1), S = number of experts: expert e sits on the listed nodes."""
+    E = len(expert_nodes)
+    slot = np.full(N * E, -1, np.int32)
+    for e, nodes in enumerate(expert_nodes):
+        for n in nodes:
+            slot[n * E + e] = e
+    return slot
+
+
+def test_tiebreak_smallest_mask_wins():
+    # N = 4, source node 0, bits 0,1,2 <-> nodes 1,2,3.  Experts on {1,2},{2,3},{1,3}: masks
+    # 011,110,101; every single node misses one expert; the 2-node covers are 011,101,110 and
+    # the ascending scan with strict '<' keeps 011 = nodes {1,2}.
+    N, S = 4, 4
+    slot = _layout_from_nodes([[1, 2], [2, 3], [1, 3], [0]], N)
+    ids = np.array([[0, 1, 2]], np.int32)
+    for seed in range(20):
+        r = O.assign(N, 1, S, 4, slot, None, ids, np.array([0], np.int32), seed)
+        nodes = r["assigned_slot"][0] // S
+        assert r["remote_nodes"][0] == 2
+        assert nodes[1] == 2 and nodes[2] == 1 and nodes[0] in (1, 2)
+    # experts on {1},{2,3}: covers 011 and 101 both have two nodes -> 011 -> second expert on node 2
+    slot = _layout_from_nodes([[1], [2, 3], [0], [0]], N)
+    ids = np.array([[0, 1]], np.int32)
+    for seed in range(20):
+        r = O.assign(N, 1, S, 4, slot, None, ids, np.array([0], np.int32), seed)
+        assert (r["assigned_slot"][0] // S).tolist() == [1, 2]
+
+
+def test_node_pick_is_spread_over_the_cover():
+    # both experts on nodes {1,2,3}, source node 0: b* = 001 (node 1) -> always node 1.
+    N, S = 4, 2
+    slot = _layout_from_nodes([[1, 2, 3], [1, 2, 3]], N)
+    ids = np.tile(np.array([[0, 1]], np.int32), (200, 1))
+    r = O.assign(N, 1, S, 2, slot, None, ids, np.zeros(200, np.int32), 5)
+    assert ((r["assigned_slot"] // S) == 1).all() and (r["remote_nodes"] == 1).all()
+    # experts on {1,2} and {3}, plus one on {1,2}: b* = 101 (nodes 1,3) -- expert 0 -> node 1
+    slot = _layout_from_nodes([[1, 2], [3], [0]], N)
+    ids = np.tile(np.array([[0, 1]], np.int32), (50, 1))
+    r = O.assign(N, 1, 3, 3, slot, None, ids, np.zeros(50, np.int32), 5)
+    assert ((r["assigned_slot"] // 3) == np.array([1, 3])).all()
+
+
+def test_random_node_uses_every_node_of_the_mask():
+    # source node 0; experts 0 and 1 both only on nodes {1,2} ... b* = 001 always (one node covers).
+    # To see RandomNode spread, need b* with 2 bits and an expert whose mask has both:
+    # experts: A on {1}, B on {2}, C on {1,2}: b* = 011, C may go to node 1 or 2.
+    N, S = 3, 3
+    slot = _layout_from_nodes([[1], [2], [1, 2]], N)
+    T = 4000
+    ids = np.tile(np.array([[0, 1, 2]], np.int32), (T, 1))
+    r = O.assign(N, 1, S, 3, slot, None, ids, np.zeros(T, np.int32), 11)
+    nodes_c = r["assigned_slot"][:, 2] // S
+    n1 = int((nodes_c == 1).sum())
+    assert set(np.unique(nodes_c)) == {1, 2}
+    assert abs(n1 - T / 2) < 4 * np.sqrt(T / 4)       # 4 sigma of a fair coin
+
+
+# ---------------------------------------------------------------- invariants --------------
+def _invariants(w, r, naive):
+    N, Q, S, E = w.N, w.Q, w.S, w.E
+    slots = r["assigned_slot"]
+    # Eq. 2 third constraint: the assigned replica holds the task's expert
+    assert (w.slot_expert[slots] == w.topk_ids).all()
+    # sum_r sum_e w_er = K T (Section 3.1)
+    assert int(r["slot_load"].sum()) == w.T * w.K
+    assert (np.bincount(slots.ravel(), minlength=w.D) == r["slot_load"]).all()
+    # Eq. 1 evaluated from the assignment itself equals the reported terms
+    V, per = O.traffic(N, Q, S, E, w.slot_expert, w.topk_ids, w.src_rank, slots)
+    assert V == r["V"] and (per == r["remote_nodes"]).all()
+    # never more remote nodes than the naive primary-replica rule, token by token
+    assert (r["remote_nodes"] <= naive["remote_nodes"]).all()
+    assert r["V"] <= naive["V"] == r["V_naive"]
+    # experts present on the source node stay there
+    src_node = w.src_rank // Q
+    holds_local = np.zeros((w.G // Q, E), bool)
+    for d, e in enumerate(w.slot_expert):
+        if e >= 0:
+            holds_local[d // (S * Q), e] = True
+    local = holds_local[src_node[:, None], w.topk_ids]
+    assert ((slots // (S * Q))[local] == np.broadcast_to(src_node[:, None], slots.shape)[local]).all()
+    all_local = local.all(axis=1)
+    assert (r["remote_nodes"][all_local] == 0).all()
+
+
+@pytest.mark.parametrize("name", ["1", "1a", "2", "3"])
+def test_invariants_on_configs(name):
+    w = W.make_config(name, T=3000)
+    r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, w.seed)
+    naive = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank,
+                     w.seed, naive=True)
+    _invariants(w, r, naive)
+    if name == "1a":
+        # one replica per expert: nothing to choose, the method degenerates to the naive rule
+        assert (r["assigned_slot"] == naive["assigned_slot"]).all()
+        assert r["V"] == naive["V"]
+    else:
+        assert r["V"] < naive["V"]
+
+
+@pytest.mark.parametrize("N,Q,S,E,K", [(1, 4, 3, 9, 3), (3, 2, 4, 13, 4), (8, 1, 5, 20, 5), (2, 3, 3, 7, 1)])
+def test_invariants_on_odd_shapes(N, Q, S, E, K):
+    w = W.make_custom(501, E, K, 8, N, Q, S, seed=99 + N, C=3, p_in=0.6, n_empty=2)
+    r = O.assign(N, Q, S, E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 1234)
+    naive = O.assign(N, Q, S, E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 1234, naive=True)
+    _invariants(w, r, naive)
+    if N == 1:
+        assert r["V"] == 0 and naive["V"] == 0
+
+
+# ---------------------------------------------------------------- exactness (Eq. 1) -------
+@pytest.mark.parametrize("N,Q,S,E,K,seed", [(2, 2, 2, 4, 2, 1), (3, 2, 3, 8, 3, 2), (4, 2, 3, 10, 4, 3),
+                                           (4, 1, 4, 6, 3, 4), (4, 2, 2, 12, 4, 5)])
+def test_alg1_matches_bruteforce_minimum(N, Q, S, E, K, seed):
+    """Algorithm 1's BitCount(b*) is the exact per-token minimum of Eq. 1 over all replica choices."""
+    w = W.make_custom(120, E, K, 8, N, Q, S, seed=seed, C=2, p_in=0.5)
+    r = O.assign(N, Q, S, E, w.slot_expert, None, w.topk_ids, w.src_rank, 77)
+    for t in range(w.T):
+        best = O.min_remote_nodes_bruteforce(w.slot_expert.tolist(), S, Q, w.topk_ids[t].tolist(),
+                                             int(w.src_rank[t]))
+        assert r["remote_nodes"][t] == best, t
+
+
+def test_bruteforce_on_fig1(fig1):
+    g = fig1
+    for tk in g["tokens"]:
+        assert O.min_remote_nodes_bruteforce(g["slot_expert"], 2, 2, tk["ids"], tk["src"]) == tk["cobalt"]
+
+
+# ---------------------------------------------------------------- randomness --------------
+def test_replica_pick_is_uniform_within_node():
+    """'Replicas of the same expert within a node receive equal workloads in expectation'."""
+    # one node, 4 ranks, expert 0 on all four ranks, expert 1 on ranks 0 and 2
+    slot = np.array([0, 1, 0, -1, 0, 1, 0, -1], np.int32)
+    T = 8000
+    ids = np.tile(np.array([[0, 1]], np.int32), (T, 1))
+    r = O.assign(1, 4, 2, 2, slot, None, ids, np.zeros(T, np.int32), 2024)
+    c0 = np.bincount(r["assigned_slot"][:, 0], minlength=8)[[0, 2, 4, 6]]
+    c1 = np.bincount(r["assigned_slot"][:, 1], minlength=8)[[1, 5]]
+    assert c0.sum() == T and c1.sum() == T
+    assert (((c0 - T / 4) ** 2) / (T / 4)).sum() < 25.0      # chi2, 3 dof
+    assert (((c1 - T / 2) ** 2) / (T / 2)).sum() < 20.0      # chi2, 1 dof
+
+
+def test_id_order_permutation_permutes_outputs():
+    """D_t is a set: listing a token's ids in another order only reorders its outputs."""
+    w = W.make_config("3", T=500)
+    r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 5)
+    perm = np.array([3, 0, 5, 1, 4, 2])
+    r2 = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids[:, perm].copy(),
+                  w.src_rank, 5)
+    assert (r2["assigned_slot"] == r["assigned_slot"][:, perm]).all()
+    assert (r2["remote_nodes"] == r["remote_nodes"]).all()
+
+
+def test_seed_changes_slots_not_cost():
+    w = W.make_config("3", T=2000)
+    a = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 1)
+    b = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 2)
+    assert (a["remote_nodes"] == b["remote_nodes"]).all()
+    assert (a["assigned_slot"] != b["assigned_slot"]).any()
+    c = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, 1)
+    assert (a["assigned_slot"] == c["assigned_slot"]).all()
+
+
+def test_remote_nodes_used_equal_the_cover():
+    """Per token the set of remote nodes used has exactly BitCount(b*) members, even over all seeds."""
+    w = W.make_custom(300, 12, 4, 8, 4, 2, 3, seed=8, C=3, p_in=0.7)
+    for seed in range(5):
+        r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, None, w.topk_ids, w.src_rank, seed)
+        nodes = r["assigned_slot"] // (w.S * w.Q)
+        src = w.src_rank // w.Q
+        for t in range(w.T):
+            used = set(nodes[t].tolist()) - {int(src[t])}
+            assert len(used) == r["remote_nodes"][t]
+
+
+def test_input_validation():
+    slot = [0, 1, 2, 0, 1, 2, 3, 0]
+    with pytest.raises(O.OracleError):
+        O.assign(2, 2, 2, 4, slot, None, np.array([[0, 0]], np.int32), np.array([0], np.int32), 1)
+    with pytest.raises(O.OracleError):
+        O.assign(2, 2, 2, 4, slot, None, np.array([[0, 4]], np.int32), np.array([0], np.int32), 1)
+    with pytest.raises(O.OracleError):
+        O.assign(2, 2, 2, 4, slot, None, np.array([[0, 1]], np.int32), np.array([4], np.int32), 1)
