@@ -1,0 +1,171 @@
+/*
+ * cobalt.h -- C ABI of the B200 (sm_100a) token-routing library for Cobalt, the
+ * co-activation-aware MoE training method.
+ *
+ * One training step's gating output (top-K expert ids and gate weights per token) and a given
+ * expert layout (every expert's replicas placed on (node, rank) slots; the layout is a plain
+ * data structure, not hardware) go through four stages:
+ *
+ *   cobalt_coact_stats   expert co-activation counts and per-expert loads   (Section 3.2, Stage 1)
+ *   cobalt_assign        communication-aware task assignment                (Section 3.3, Algorithm 1)
+ *   cobalt_permute       destination-grouped send buffer                    (Fig. 1, "Dispatch")
+ *   cobalt_combine       inverse permutation + gate-weighted sum            (Fig. 1, "Weighted sum")
+ *
+ * Symbols (Table 1): E experts, K experts per token, G = N*Q ranks on N nodes with Q ranks
+ * each, T tokens, D_t the selected experts of token t, s_t its source rank, P_r the experts
+ * on rank r, r_te the rank that runs task (t, e).  Each rank has S expert slots; the global
+ * slot id is d = r*S + j (rank = d / S, node = d / (S*Q)); D = G*S destinations; a (token,
+ * expert) pair has index p = t*K + k; P = T*K pairs.  r_te is reported as a global slot id.
+ *
+ * Conventions for every call unless stated otherwise
+ *  - Pointers named *_host are host memory; all others are DEVICE pointers borrowed from the
+ *    caller for the duration of the enqueued work.  The library allocates nothing per call;
+ *    scratch comes from the caller-provided workspace (size from the *_workspace_bytes
+ *    query, 256-byte aligned).  Only the layout handle owns device memory.
+ *  - Device pointers must be 16-byte aligned.
+ *  - Calls enqueue kernels on `stream` (a cudaStream_t, NULL = default stream) and return
+ *    without synchronising; outputs are valid once the stream reaches that point.
+ *  - Return value: COBALT_OK or a negative COBALT_ERR_* code.  Nothing is enqueued when an
+ *    argument check fails.  The library never throws, exits, traps or waits unboundedly.
+ *  - Data preconditions: ids in [0, E) and distinct within a token (D_t is a set); source
+ *    ranks in [0, G); assigned slots in [0, D).  A violation never causes an out-of-bounds
+ *    access: the kernel sets a bit in the device error word, skips the offending token or
+ *    pair (its outputs are unspecified; slots are written as -1), and carries on.
+ */
+#ifndef COBALT_H_
+#define COBALT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define COBALT_VERSION 100
+
+#define COBALT_OK 0
+#define COBALT_ERR_INVALID_ARG (-1)          /* null / negative / misaligned argument, bad layout */
+#define COBALT_ERR_WORKSPACE_TOO_SMALL (-2)
+#define COBALT_ERR_UNSUPPORTED (-3)          /* outside the supported size envelope (see below) */
+#define COBALT_ERR_CUDA (-4)                 /* a CUDA runtime call failed; see cobalt_last_cuda_error */
+
+/* Supported envelope: N <= 8 nodes, K <= 16, E <= 1024, D <= 4096, P = T*K < 2^31,
+ * H a multiple of 8 (rows are whole 16-byte vectors). */
+#define COBALT_MAX_NODES 8
+#define COBALT_MAX_TOPK 16
+#define COBALT_MAX_EXPERTS 1024
+#define COBALT_MAX_DESTS 4096
+
+/* bits of the device error word (cobalt_read_and_clear_device_error) */
+#define COBALT_DEVERR_BAD_EXPERT_ID 0x1u     /* id outside [0, E) */
+#define COBALT_DEVERR_DUPLICATE_ID 0x2u      /* an expert listed twice in one token */
+#define COBALT_DEVERR_BAD_SRC_RANK 0x4u      /* source rank outside [0, G) */
+#define COBALT_DEVERR_BAD_SLOT 0x8u          /* assigned slot / row index outside its range */
+#define COBALT_DEVERR_WAIT_TIMEOUT 0x10u     /* a bounded on-chip wait ran out (copy pipeline) */
+
+/* flag bits */
+#define COBALT_STATS_ACCUMULATE 0x1u         /* add to coact/load instead of overwriting them */
+#define COBALT_ASSIGN_NAIVE 0x1u             /* primary-replica rule instead of Algorithm 1 */
+#define COBALT_IMPL_MASK 0xF00u              /* kernel variant override, 0 = library default */
+#define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
+#define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies through shared memory */
+
+typedef struct cobalt_layout cobalt_layout_t;   /* opaque, owned by the library */
+typedef void* cobalt_stream_t;                  /* a cudaStream_t */
+
+const char* cobalt_status_string(int status);
+int cobalt_version(void);
+/* The cudaError_t of the most recent failed runtime call on this thread (0 if none). */
+int cobalt_last_cuda_error(void);
+
+/* ---- expert layout (Section 3.1: P = {P_r}; Section 3.3: R_{e,n}, N_e) -------------------
+ * slot_expert_host[r*S + j] is the expert in slot j of rank r, or -1 for an empty slot.
+ * primary_slot_host[e] is the slot of e's primary replica (used by the naive rule and for
+ * V_naive); NULL means "the lowest slot holding e".
+ * A layout is rejected with COBALT_ERR_INVALID_ARG when an expert has no replica (Eq. 2,
+ * first constraint), an expert sits twice on one rank (Section 3.2, Stage 2), an id is outside
+ * [-1, E), or a given primary slot does not hold its expert; with COBALT_ERR_UNSUPPORTED
+ * outside the size envelope.  cobalt_layout_check runs only these host-side checks (no device
+ * needed).  cobalt_layout_create also builds the device tables (one allocation, one copy, on
+ * the current device; synchronous) and returns a handle to be released with
+ * cobalt_layout_destroy (NULL is accepted). */
+int cobalt_layout_check(int32_t num_nodes, int32_t ranks_per_node, int32_t slots_per_rank,
+                        int32_t num_experts, const int32_t* slot_expert_host,
+                        const int32_t* primary_slot_host);
+int cobalt_layout_create(cobalt_layout_t** out, int32_t num_nodes, int32_t ranks_per_node,
+                         int32_t slots_per_rank, int32_t num_experts,
+                         const int32_t* slot_expert_host, const int32_t* primary_slot_host);
+int cobalt_layout_destroy(cobalt_layout_t* layout);
+/* D = G*S of a layout (0 for NULL). */
+int32_t cobalt_layout_num_dests(const cobalt_layout_t* layout);
+
+/* ---- stage 1: per-step statistics (Section 3.2, Stage 1) ---------------------------------
+ * load[e]      = number of tokens selecting e (the task count whose EMA is w^_e)
+ * coact[i*E+j] = number of tokens selecting both i and j (whose EMA is c^_ij); symmetric,
+ *                diagonal = load.
+ * topk_ids: int32 [T, K] row-major.  coact: uint32 [E*E].  load: uint32 [E].
+ * Outputs are overwritten unless COBALT_STATS_ACCUMULATE is set.  T = 0 is allowed. */
+size_t cobalt_coact_stats_workspace_bytes(int64_t T, int32_t K, int32_t E);
+int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
+                       uint32_t* coact, uint32_t* load, uint32_t flags,
+                       void* workspace, size_t workspace_bytes, cobalt_stream_t stream);
+
+/* ---- stage 2: communication-aware task assignment (Section 3.3, Algorithm 1) --------------
+ * Per token: experts present on the source node N(s_t) run there; for the others the
+ * smallest set of remote nodes covering them is found by enumerating (N-1)-bit masks in
+ * ascending order (first minimum wins), each such expert picks a node of that set and every
+ * expert picks a replica inside its node, both uniformly through a counter hash of
+ * (seed, t, e) so that results do not depend on launch shape.
+ * src_rank: int32 [T], or NULL to use src_rank_uniform for every token.
+ * Outputs: assigned_slot int32 [T*K] (r_te as global slot id); optional (NULL to skip)
+ * slot_load uint32 [D] = w_er (Section 3.1), remote_nodes uint8 [T] = the token's term of
+ * Eq. 1, totals uint64 [2] = { V of this assignment, V of the naive primary-replica rule }.
+ * The optional outputs are overwritten.  COBALT_ASSIGN_NAIVE assigns every task to its
+ * expert's primary replica instead (the one-replica-per-expert baseline). */
+size_t cobalt_assign_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);
+int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids,
+                  const int32_t* src_rank, int32_t src_rank_uniform, int64_t T, int32_t K,
+                  uint64_t seed, int32_t* assigned_slot, uint32_t* slot_load,
+                  uint8_t* remote_nodes, uint64_t* totals, uint32_t flags,
+                  void* workspace, size_t workspace_bytes, cobalt_stream_t stream);
+
+/* ---- stage 3: dispatch-side permutation (Fig. 1, "Dispatch"; Section 1) --------------------
+ * Groups the P pairs by destination slot, keeping ascending pair index inside a destination:
+ *   dest_counts[d]  = #{p : assigned_slot[p] = d}                     uint32 [D]
+ *   dest_offsets    = exclusive scan of dest_counts, last entry = P   uint32 [D+1]
+ *   row_of_pair[p]  = dest_offsets[d_p] + #{q < p : d_q = d_p}        int32 [P]
+ *   pair_of_row     = inverse of row_of_pair (NULL to skip)           int32 [P]
+ *   send[row_of_pair[p]] = x[p / K]    bit copy of H 16-bit elements  bf16 [P, H]
+ * x is bf16 [T, H].  cobalt_permute = cobalt_permute_index followed by cobalt_permute_rows;
+ * the two halves are exported so that the maps can be reused (e.g. for another tensor). */
+size_t cobalt_permute_workspace_bytes(int64_t T, int32_t K, int32_t D);
+int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
+                         uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                         int32_t* pair_of_row, void* workspace, size_t workspace_bytes,
+                         cobalt_stream_t stream);
+int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K,
+                        int32_t H, void* send, uint32_t flags, cobalt_stream_t stream);
+int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
+                   const void* x, int32_t H, void* send, uint32_t* dest_counts,
+                   uint32_t* dest_offsets, int32_t* row_of_pair, int32_t* pair_of_row,
+                   uint32_t flags, void* workspace, size_t workspace_bytes,
+                   cobalt_stream_t stream);
+
+/* ---- stage 4: combine (Fig. 1, "Weighted sum"; Section 1) ----------------------------------
+ * y[t][h] = bf16( sum_{k<K} gate_w[t*K+k] * float(expert_out[row_of_pair[t*K+k]][h]) ),
+ * fp32 accumulation in ascending k, one round-to-nearest-even at the end.
+ * expert_out: bf16 [P, H] in the row order of `send`.  gate_w: fp32 [P].  y: bf16 [T, H]. */
+int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w,
+                   int64_t T, int32_t K, int32_t H, void* y, uint32_t flags,
+                   cobalt_stream_t stream);
+
+/* ---- device error word -------------------------------------------------------------------
+ * Waits for `stream`, copies the COBALT_DEVERR_* bits set by kernels on the current device
+ * since the last call into *out_bits_host and clears them. */
+int cobalt_read_and_clear_device_error(uint32_t* out_bits_host, cobalt_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COBALT_H_ */

@@ -1,0 +1,224 @@
+// Stage 1: per-step co-activation counts and expert loads (Section 3.2, Stage 1).
+//
+// coact[i][j] = #tokens selecting both i and j is symmetric with the load on its diagonal,
+// so each CTA histograms only the lower triangle (hi >= lo) of its tokens into a private
+// shared-memory tile: K(K+1)/2 shared-memory integer adds per token.  CTAs are grouped in
+// thread-block clusters; after a cluster barrier each CTA sums its share of the tile rows over
+// all CTAs of the cluster through distributed shared memory and merges the result into global
+// memory with integer reductions, mirroring (hi, lo) to (lo, hi) and writing the diagonal to
+// `load` as well.  Only integer adds are used, so the result is independent of scheduling.
+// Experts counts whose triangle does not fit in shared memory take a direct global-atomic path.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace cobalt {
+
+constexpr int kStatsThreads = 512;
+constexpr size_t kStatsMaxTileBytes = 200 * 1024;
+
+__host__ __device__ inline size_t tri_entries(int E) { return static_cast<size_t>(E) * (E + 1) / 2; }
+
+template <int KT>
+__device__ __forceinline__ bool load_token_ids(const int32_t* __restrict__ ids, int64_t t, int K, int E,
+                                               int32_t (&id)[(KT > 0) ? KT : COBALT_MAX_TOPK],
+                                               uint32_t* err_word)
+{
+    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    const int32_t* row = ids + t * K;
+    if (KT > 0 && KT % 4 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 4; ++a) {
+            const int4 v = __ldg(reinterpret_cast<const int4*>(row) + a);
+            id[4 * a] = v.x; id[4 * a + 1] = v.y; id[4 * a + 2] = v.z; id[4 * a + 3] = v.w;
+        }
+    } else if (KT > 0 && KT % 2 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 2; ++a) {
+            const int2 v = __ldg(reinterpret_cast<const int2*>(row) + a);
+            id[2 * a] = v.x; id[2 * a + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a)
+            if (a < K) id[a] = __ldg(row + a);
+    }
+    uint32_t bad = 0;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            if (id[a] < 0 || id[a] >= E) bad |= COBALT_DEVERR_BAD_EXPERT_ID;
+#pragma unroll
+            for (int b = 0; b < a; ++b)
+                if (id[b] == id[a]) bad |= COBALT_DEVERR_DUPLICATE_ID;
+        }
+    }
+    if (bad) flag_error(err_word, bad);
+    return bad == 0;
+}
+
+template <int KT>
+__global__ void __launch_bounds__(kStatsThreads)
+coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E,
+                  uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(16) uint32_t tri[];
+    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    const int K = (KT > 0) ? KT : K_rt;
+    cg::cluster_group cluster = cg::this_cluster();
+
+    const int n_tri = static_cast<int>(tri_entries(E));
+    for (int i = threadIdx.x; i < n_tri; i += blockDim.x) tri[i] = 0;
+    __syncthreads();
+
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
+        int32_t id[KMAX];
+        if (!load_token_ids<KT>(topk_ids, t, K, E, id, err_word)) continue;
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a) {
+#pragma unroll
+            for (int b = a; b < KMAX; ++b) {
+                if (b < K) {
+                    const int hi = max(id[a], id[b]), lo = min(id[a], id[b]);
+                    atomicAdd(&tri[hi * (hi + 1) / 2 + lo], 1u);
+                }
+            }
+        }
+    }
+
+    cluster.sync();  // every tile of the cluster is complete
+    const unsigned csize = cluster.num_blocks();
+    const unsigned crank = cluster.block_rank();
+    const uint32_t* peer[8];
+#pragma unroll
+    for (unsigned r = 0; r < 8; ++r) peer[r] = cluster.map_shared_rank(tri, r < csize ? r : 0);
+
+    for (int hi = static_cast<int>(crank); hi < E; hi += static_cast<int>(csize)) {
+        const int base = hi * (hi + 1) / 2;
+        for (int lo = threadIdx.x; lo <= hi; lo += blockDim.x) {
+            uint32_t sum = 0;
+#pragma unroll
+            for (unsigned r = 0; r < 8; ++r)
+                if (r < csize) sum += peer[r][base + lo];
+            if (sum) {
+                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], sum);
+                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], sum);
+                else atomicAdd(&load[hi], sum);
+            }
+        }
+    }
+    cluster.sync();  // no CTA may exit while a peer still reads its tile
+}
+
+// Fallback for expert counts whose triangle does not fit in shared memory.
+__global__ void __launch_bounds__(256)
+coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int E,
+                    uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
+{
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
+        int32_t id[COBALT_MAX_TOPK];
+        if (!load_token_ids<0>(topk_ids, t, K, E, id, err_word)) continue;
+        for (int a = 0; a < K; ++a) {
+            atomicAdd(&load[id[a]], 1u);
+            for (int b = 0; b < K; ++b) atomicAdd(&coact[static_cast<size_t>(id[a]) * E + id[b]], 1u);
+        }
+    }
+}
+
+template <int KT>
+static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
+                       uint32_t* err_word, int n_sm, cudaStream_t stream)
+{
+    auto kernel = coact_tile_kernel<KT>;
+    const size_t smem = tri_entries(E) * sizeof(uint32_t);
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+
+    // one CTA per ~2 tokens per thread, at most one per SM, in clusters of up to 8
+    int64_t want = (T + 2 * kStatsThreads - 1) / (2 * kStatsThreads);
+    int n_cta = static_cast<int>(want < 1 ? 1 : (want > n_sm ? n_sm : want));
+    int csize = 8;
+    while (csize > n_cta) csize >>= 1;
+
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(kStatsThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    for (; csize >= 1; csize >>= 1) {
+        attr[0].val.clusterDim.x = csize;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3(static_cast<unsigned>(n_cta / csize * csize));
+        int max_clusters = 0;
+        cudaError_t q = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
+        if (q == cudaSuccess && max_clusters >= 1) break;
+        (void)cudaGetLastError();
+    }
+    if (csize < 1) return COBALT_ERR_UNSUPPORTED;
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, coact, load, err_word));
+    return COBALT_OK;
+}
+
+}  // namespace cobalt
+
+using namespace cobalt;
+
+extern "C" {
+
+size_t cobalt_coact_stats_workspace_bytes(int64_t T, int32_t K, int32_t E)
+{
+    (void)T; (void)K; (void)E;
+    return 0;  // privatised tiles live in shared memory
+}
+
+int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E, uint32_t* coact,
+                       uint32_t* load, uint32_t flags, void* workspace, size_t workspace_bytes,
+                       cobalt_stream_t stream)
+{
+    (void)workspace; (void)workspace_bytes;
+    if (T < 0 || K < 1 || E < 1 || !coact || !load) return COBALT_ERR_INVALID_ARG;
+    if (K > E) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || E > COBALT_MAX_EXPERTS || T * static_cast<int64_t>(K) >= (1ll << 31))
+        return COBALT_ERR_UNSUPPORTED;
+    if (T > 0 && !topk_ids) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(topk_ids) || !aligned16(coact) || !aligned16(load)) return COBALT_ERR_INVALID_ARG;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!(flags & COBALT_STATS_ACCUMULATE)) {
+        COBALT_CUDA_TRY(cudaMemsetAsync(coact, 0, sizeof(uint32_t) * static_cast<size_t>(E) * E, s));
+        COBALT_CUDA_TRY(cudaMemsetAsync(load, 0, sizeof(uint32_t) * static_cast<size_t>(E), s));
+    }
+    if (T == 0) return COBALT_OK;
+
+    uint32_t* err_word = nullptr;
+    int rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+    int n_sm = 0;
+    rc = sm_count(&n_sm);
+    if (rc != COBALT_OK) return rc;
+
+    if (tri_entries(E) * sizeof(uint32_t) > kStatsMaxTileBytes) {
+        int64_t want = (T + 255) / 256;
+        const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
+        coact_global_kernel<<<grid, 256, 0, s>>>(topk_ids, T, K, E, coact, load, err_word);
+        COBALT_CUDA_TRY(cudaGetLastError());
+        return COBALT_OK;
+    }
+    switch (K) {
+        case 1: return launch_tile<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        case 2: return launch_tile<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        case 4: return launch_tile<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        case 6: return launch_tile<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        case 8: return launch_tile<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        default: return launch_tile<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+    }
+}
+
+}  // extern "C"

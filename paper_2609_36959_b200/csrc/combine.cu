@@ -1,0 +1,125 @@
+// Stage 4: inverse permutation + gate-weighted sum (Fig. 1, "Weighted sum").
+//
+//   y[t][h] = bf16( sum_{k<K} g[t][k] * float(out[row_of_pair[t*K+k]][h]) )
+//
+// Read-dominated streaming kernel: a thread owns one 16-byte vector (8 bf16 columns) of a
+// token, issues its K gathered row loads back to back (K * 16 bytes in flight per thread),
+// accumulates in fp32 in ascending k and stores one 16-byte vector.  Rows are read once and
+// written once, so both directions bypass L1 allocation.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace cobalt {
+
+constexpr int kCombineThreads = 256;
+
+__device__ __forceinline__ void fma_bf16x2(float& a0, float& a1, uint32_t packed, float w)
+{
+    a0 = fmaf(w, __uint_as_float(packed << 16), a0);
+    a1 = fmaf(w, __uint_as_float(packed & 0xFFFF0000u), a1);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <int KT>
+__global__ void __launch_bounds__(kCombineThreads)
+combine_kernel(const uint4* __restrict__ out, const int32_t* __restrict__ row_of_pair,
+               const float* __restrict__ gate_w, int64_t T, int K_rt, int n_vec, int64_t P,
+               uint4* __restrict__ y, uint32_t* __restrict__ err_word)
+{
+    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    const int K = (KT > 0) ? KT : K_rt;
+    for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
+        int64_t row[KMAX];
+        float w[KMAX];
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            if (k < K) {
+                const int32_t r = __ldg(row_of_pair + t * K + k);
+                const bool valid = (r >= 0 && r < P);
+                row[k] = valid ? static_cast<int64_t>(r) * n_vec : -1;
+                w[k] = valid ? __ldg(gate_w + t * K + k) : 0.0f;
+                if (!valid && threadIdx.x == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+            }
+        }
+        for (int v = threadIdx.x; v < n_vec; v += blockDim.x) {
+            uint4 val[KMAX];
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k)
+                if (k < K) val[k] = (row[k] >= 0) ? ld_stream16(out + row[k] + v) : make_uint4(0, 0, 0, 0);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) {
+                if (k < K) {
+                    fma_bf16x2(acc[0], acc[1], val[k].x, w[k]);
+                    fma_bf16x2(acc[2], acc[3], val[k].y, w[k]);
+                    fma_bf16x2(acc[4], acc[5], val[k].z, w[k]);
+                    fma_bf16x2(acc[6], acc[7], val[k].w, w[k]);
+                }
+            }
+            uint4 o;
+            o.x = pack_bf16x2(acc[0], acc[1]);
+            o.y = pack_bf16x2(acc[2], acc[3]);
+            o.z = pack_bf16x2(acc[4], acc[5]);
+            o.w = pack_bf16x2(acc[6], acc[7]);
+            st_stream16(y + t * n_vec + v, o);
+        }
+    }
+}
+
+}  // namespace cobalt
+
+using namespace cobalt;
+
+extern "C" {
+
+int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
+                   int32_t K, int32_t H, void* y, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1 || H < 1) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31))
+        return COBALT_ERR_UNSUPPORTED;
+    if (T == 0) return COBALT_OK;
+    if (!expert_out || !row_of_pair || !gate_w || !y) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(expert_out) || !aligned16(y) || !aligned16(row_of_pair) || !aligned16(gate_w))
+        return COBALT_ERR_INVALID_ARG;
+    const uint32_t impl = flags & COBALT_IMPL_MASK;
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR) return COBALT_ERR_INVALID_ARG;
+
+    uint32_t* err_word = nullptr;
+    int rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+    int n_sm = 0;
+    rc = sm_count(&n_sm);
+    if (rc != COBALT_OK) return rc;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n_vec = H / 8;
+    const int64_t P = T * K;
+    const unsigned grid = static_cast<unsigned>(T < 16ll * n_sm ? T : 16ll * n_sm);
+    const uint4* src = static_cast<const uint4*>(expert_out);
+    uint4* dst = static_cast<uint4*>(y);
+#define COBALT_COMBINE_CASE(KT)                                                                         \
+    case KT:                                                                                            \
+        combine_kernel<KT><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, err_word); \
+        break
+    switch (K) {
+        COBALT_COMBINE_CASE(1);
+        COBALT_COMBINE_CASE(2);
+        COBALT_COMBINE_CASE(4);
+        COBALT_COMBINE_CASE(6);
+        COBALT_COMBINE_CASE(8);
+        default:
+            combine_kernel<0><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, err_word);
+    }
+#undef COBALT_COMBINE_CASE
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,108 @@
+// Shared host/device helpers of the sm_100a token-routing library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cobalt.h"
+
+namespace cobalt {
+
+// ---- host side ---------------------------------------------------------------------------
+// Records a failed runtime call for cobalt_last_cuda_error() and maps it to COBALT_ERR_CUDA.
+int record_cuda_error(cudaError_t err);
+
+#define COBALT_CUDA_TRY(expr)                                        \
+    do {                                                             \
+        cudaError_t cobalt_err__ = (expr);                           \
+        if (cobalt_err__ != cudaSuccess)                             \
+            return ::cobalt::record_cuda_error(cobalt_err__);        \
+    } while (0)
+
+// Address of the current device's error word (kernels receive it as an argument).
+int device_error_word(uint32_t** out);
+
+// Number of SMs of the current device (cached per device).
+int sm_count(int* out);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Device tables built from a layout (Section 3.3: R_{e,n} and N_e), one contiguous blob of
+// 32-bit words that kernels copy into shared memory:
+//   ent[e*N + n]   = (offset into rlist << 8) | |R_{e,n}|
+//   primary[e]     = slot of e's primary replica
+//   rlist[...]     = slots of R_{e,n}, ascending, all (e, n) groups back to back
+//   nodes[e]       = bitmask over nodes holding e (one word each)
+struct LayoutView {
+    int32_t N, Q, S, E, G, D;
+    int32_t n_replicas;       // entries of rlist
+    int32_t words;            // total 32-bit words of the blob
+    const uint32_t* blob;     // device
+    __host__ __device__ int ent_off() const { return 0; }
+    __host__ __device__ int primary_off() const { return E * N; }
+    __host__ __device__ int rlist_off() const { return E * N + E; }
+    __host__ __device__ int nodes_off() const { return E * N + E + n_replicas; }
+};
+
+}  // namespace cobalt
+
+struct cobalt_layout {
+    cobalt::LayoutView view;
+    int device;
+};
+
+namespace cobalt {
+
+// ---- device side -------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// Counter hash behind Algorithm 1's RandomNode (stream 0) and UniformChoice (stream 1): a pure
+// function of (seed, token, expert, stream), all arithmetic modulo 2^32, so that the draw does
+// not depend on thread or launch shape.
+__device__ __forceinline__ uint32_t route_hash(uint32_t seed_lo, uint32_t seed_hi, uint32_t t,
+                                               uint32_t e, uint32_t stream)
+{
+    uint32_t x = seed_lo ^ 0x6A09E667u;
+    x = (x ^ t) * 0x9E3779B9u;
+    x ^= x >> 16;
+    x = (x ^ seed_hi) * 0xBB67AE85u;
+    x ^= x >> 15;
+    x = (x ^ (2u * e + stream)) * 0x9E3779B9u;
+    x ^= x >> 16;
+    x *= 0xBB67AE85u;
+    x ^= x >> 15;
+    x *= 0x6A09E667u;
+    x ^= x >> 16;
+    return x;
+}
+
+// floor(x * n / 2^32): an index in [0, n)
+__device__ __forceinline__ uint32_t hash_index(uint32_t x, uint32_t n) { return __umulhi(x, n); }
+
+__device__ __forceinline__ void flag_error(uint32_t* err_word, uint32_t bits)
+{
+    atomicOr(err_word, bits);
+}
+
+// streaming (read-once / write-once) 16-byte accesses that stay out of L1
+__device__ __forceinline__ uint4 ld_stream16(const void* p)
+{
+    uint4 v;
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream16(void* p, uint4 v)
+{
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x),
+                 "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+#endif  // __CUDACC__
+
+}  // namespace cobalt

@@ -1,0 +1,525 @@
+// Stage 3: dispatch-side permutation (Fig. 1, "Dispatch").
+//
+// Index part (deterministic, no position atomics): the pair range is cut into chunks of
+// contiguous pairs;
+//   K1  per-chunk histogram over the D destinations              -> ws[d][chunk]
+//   K2  per-destination exclusive scan across chunks (in place)  -> ws[d][chunk], dest_counts
+//   K3  per chunk: exclusive scan of dest_counts over d (dest_offsets), then the stable rank
+//       of every pair inside its chunk: each warp owns a contiguous sub-range, counts it,
+//       the CTA scans the per-warp counts in warp order, and each warp walks its sub-range
+//       again, ranking equal destinations inside a 32-pair step by lane order
+//       (__match_any_sync + popcount of lower lanes).
+// Row part: K4 moves each token's row to its K rows of the send buffer.  Two variants: plain
+// 16-byte streaming loads/stores, and a bulk-async-copy pipeline (global -> shared ring ->
+// K global rows) driven by one warp per CTA.
+#include "common.cuh"
+
+namespace cobalt {
+
+constexpr int kPermThreads = 256;
+constexpr int kPermWarps = kPermThreads / 32;
+constexpr int kMinChunk = 2048;      // pairs per chunk (multiple of kPermThreads)
+constexpr int kMaxChunks = 2048;
+
+struct ChunkPlan {
+    int64_t P;
+    int chunk;        // pairs per chunk
+    int n_chunks;
+};
+
+static ChunkPlan plan_chunks(int64_t P)
+{
+    ChunkPlan c;
+    c.P = P;
+    int64_t chunk = kMinChunk;
+    while ((P + chunk - 1) / chunk > kMaxChunks) chunk *= 2;
+    c.chunk = static_cast<int>(chunk);
+    c.n_chunks = static_cast<int>((P + chunk - 1) / chunk);
+    if (c.n_chunks < 1) c.n_chunks = 1;
+    return c;
+}
+
+// ---- K1 -----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kPermThreads)
+perm_hist_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
+                 uint32_t* __restrict__ ws, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ uint32_t hist[];
+    for (int d = threadIdx.x; d < D; d += blockDim.x) hist[d] = 0;
+    __syncthreads();
+    const int64_t p0 = static_cast<int64_t>(blockIdx.x) * chunk;
+    const int64_t p1 = min(P, p0 + chunk);
+    bool bad = false;
+    for (int64_t p = p0 + threadIdx.x; p < p1; p += blockDim.x) {
+        const int32_t d = __ldg(slot + p);
+        if (d >= 0 && d < D) atomicAdd(&hist[d], 1u);
+        else bad = true;
+    }
+    if (bad) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+    __syncthreads();
+    for (int d = threadIdx.x; d < D; d += blockDim.x)
+        ws[static_cast<size_t>(d) * n_chunks + blockIdx.x] = hist[d];
+}
+
+// ---- K2: one warp per destination ---------------------------------------------------------
+__global__ void __launch_bounds__(kPermThreads)
+perm_scan_kernel(uint32_t* __restrict__ ws, int D, int n_chunks, uint32_t* __restrict__ dest_counts)
+{
+    const int d = blockIdx.x * kPermWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (d >= D) return;
+    uint32_t* row = ws + static_cast<size_t>(d) * n_chunks;
+    uint32_t running = 0;
+    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+        const int c = c0 + lane;
+        const uint32_t v = (c < n_chunks) ? row[c] : 0u;
+        uint32_t incl = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += up;
+        }
+        if (c < n_chunks) row[c] = running + incl - v;
+        running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (lane == 0) dest_counts[d] = running;
+}
+
+// ---- K3 -----------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kPermThreads)
+perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
+                 const uint32_t* __restrict__ ws, const uint32_t* __restrict__ dest_counts,
+                 uint32_t* __restrict__ dest_offsets, int32_t* __restrict__ row_of_pair,
+                 int32_t* __restrict__ pair_of_row)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t* base = sm;                 // [D]   first row of this chunk inside destination d
+    uint32_t* wcnt = sm + D;             // [kPermWarps][D]
+    __shared__ uint32_t warp_sums[kPermWarps];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // exclusive scan of dest_counts over d: thread-contiguous segments, then a block scan
+    const int per = (D + kPermThreads - 1) / kPermThreads;
+    const int d_lo = min(D, tid * per), d_hi = min(D, d_lo + per);
+    uint32_t local = 0;
+    for (int d = d_lo; d < d_hi; ++d) local += __ldg(dest_counts + d);
+    uint32_t incl = local;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    for (int i = tid; i < kPermWarps * D; i += kPermThreads) wcnt[i] = 0;
+    __syncthreads();
+    uint32_t before = incl - local;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    for (int d = d_lo; d < d_hi; ++d) {
+        if (blockIdx.x == 0) dest_offsets[d] = before;
+        base[d] = before + __ldg(ws + static_cast<size_t>(d) * n_chunks + blockIdx.x);
+        before += __ldg(dest_counts + d);
+    }
+    if (blockIdx.x == 0 && tid == kPermThreads - 1) dest_offsets[D] = before;  // last thread ends at D
+
+    // warp sub-ranges of the chunk, in pair order
+    const int64_t c0 = static_cast<int64_t>(blockIdx.x) * chunk;
+    const int sub = chunk / kPermWarps;
+    const int64_t w0 = c0 + static_cast<int64_t>(warp) * sub;
+    const int64_t w1 = min(P, w0 + sub);
+    uint32_t* mine = wcnt + warp * D;
+
+    // pass A: count this warp's sub-range per destination (warp-private, no atomics)
+    for (int64_t q = w0; q < w1; q += 32) {
+        const int64_t p = q + lane;
+        int32_t d = (p < w1) ? __ldg(slot + p) : -1;
+        if (d >= D) d = -1;
+        const uint32_t key = static_cast<uint32_t>(d);
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, key);
+        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
+        __syncwarp();
+    }
+    __syncthreads();
+    // pass B: per destination, turn the per-warp counts into starting rows (warp order)
+    for (int d = tid; d < D; d += kPermThreads) {
+        uint32_t run = base[d];
+#pragma unroll
+        for (int w = 0; w < kPermWarps; ++w) {
+            const uint32_t c = wcnt[w * D + d];
+            wcnt[w * D + d] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    // pass C: stable rank inside the warp's sub-range
+    for (int64_t q = w0; q < w1; q += 32) {
+        const int64_t p = q + lane;
+        int32_t d = (p < w1) ? __ldg(slot + p) : -1;
+        const bool in_range = (p < w1);
+        if (d >= D) d = -1;
+        const uint32_t key = static_cast<uint32_t>(d);
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, key);
+        if (d >= 0) {
+            const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
+            row_of_pair[p] = static_cast<int32_t>(row);
+            if (pair_of_row) pair_of_row[row] = static_cast<int32_t>(p);
+        } else if (in_range) {
+            row_of_pair[p] = -1;
+        }
+        __syncwarp();
+        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);
+        __syncwarp();
+    }
+}
+
+// ---- K4, vector variant -------------------------------------------------------------------
+template <int KT>
+__global__ void __launch_bounds__(256)
+perm_rows_vector_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row_of_pair, int64_t T,
+                        int K_rt, int n_vec, int64_t P, uint4* __restrict__ send,
+                        uint32_t* __restrict__ err_word)
+{
+    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    const int K = (KT > 0) ? KT : K_rt;
+    for (int64_t t = blockIdx.x; t < T; t += gridDim.x) {
+        int64_t row[KMAX];
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            if (k < K) {
+                const int32_t r = __ldg(row_of_pair + t * K + k);
+                row[k] = (r >= 0 && r < P) ? static_cast<int64_t>(r) * n_vec : -1;
+                if (r >= P && threadIdx.x == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+            }
+        }
+        const uint4* src = x + t * n_vec;
+#pragma unroll 2
+        for (int v = threadIdx.x; v < n_vec; v += blockDim.x) {
+            const uint4 val = ld_stream16(src + v);
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k)
+                if (k < K && row[k] >= 0) st_stream16(send + row[k] + v, val);
+        }
+    }
+}
+
+// ---- K4, bulk-async-copy variant ----------------------------------------------------------
+constexpr int kBulkStages = 6;
+constexpr int kBulkLag = 3;                      // stages of loads in flight ahead of the stores
+constexpr int kBulkMaxStageBytes = 18432;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+// Bounded wait for a phase of an mbarrier; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    const uint32_t addr = smem_addr(bar);
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_addr(smem_src)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// One warp per CTA.  Work item i: `rows_per_item` whole rows of consecutive tokens (n_seg == 1),
+// or one column segment of one token's row (n_seg > 1, rows_per_item == 1).
+__global__ void __launch_bounds__(32)
+perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_pair, int64_t T,
+                      int K, int64_t P, uint32_t row_bytes, int rows_per_item, int n_seg,
+                      uint32_t seg_bytes, uint32_t stage_bytes, int64_t n_items,
+                      uint8_t* __restrict__ send, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ __align__(8) uint64_t full[kBulkStages];
+    __shared__ int32_t rows_sm[kBulkStages][32];
+
+    const int lane = threadIdx.x;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kBulkStages; ++s) mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    const int64_t first = blockIdx.x;
+    const int64_t step = gridDim.x;
+    const int64_t n_mine = (n_items > first) ? (n_items - first + step - 1) / step : 0;
+
+    auto item_tokens = [&](int64_t item, int64_t& t0, int& n_rows, uint32_t& col, uint32_t& bytes) {
+        if (n_seg == 1) {
+            t0 = item * rows_per_item;
+            n_rows = (T - t0 < rows_per_item) ? static_cast<int>(T - t0) : rows_per_item;
+            col = 0;
+            bytes = row_bytes;
+        } else {
+            t0 = item / n_seg;
+            n_rows = 1;
+            col = static_cast<uint32_t>(item % n_seg) * seg_bytes;
+            bytes = min(seg_bytes, row_bytes - col);
+        }
+    };
+    auto lane_row = [&](int64_t item) -> int32_t {
+        int64_t t0; int n_rows; uint32_t col, bytes;
+        item_tokens(item, t0, n_rows, col, bytes);
+        if (lane < n_rows * K) return __ldg(row_of_pair + t0 * K + lane);
+        return -1;
+    };
+
+    bool ok = true;
+    int32_t pref = (n_mine > 0) ? lane_row(first) : -1;
+    for (int64_t j = 0; j < n_mine + kBulkLag && ok; ++j) {
+        if (j < n_mine) {
+            // produce item j: its stage was last used by item j - kBulkStages
+            const int s = static_cast<int>(j % kBulkStages);
+            bulk_wait_read<kBulkStages - kBulkLag - 1>();
+            rows_sm[s][lane] = pref;
+            if (j + 1 < n_mine) pref = lane_row(first + (j + 1) * step);
+            __syncwarp();
+            if (lane == 0) {
+                int64_t t0; int n_rows; uint32_t col, bytes;
+                item_tokens(first + j * step, t0, n_rows, col, bytes);
+                const uint32_t total = (n_seg == 1) ? static_cast<uint32_t>(n_rows) * row_bytes : bytes;
+                mbar_expect_tx(&full[s], total);
+                bulk_load(ring + static_cast<size_t>(s) * stage_bytes,
+                          x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s]);
+            }
+        }
+        if (j >= kBulkLag) {
+            // consume item c: wait for its rows, then fan each row out to its K destinations
+            const int64_t c = j - kBulkLag;
+            const int s = static_cast<int>(c % kBulkStages);
+            ok = mbar_wait(&full[s], static_cast<uint32_t>((c / kBulkStages) & 1));
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok) {
+                int64_t t0; int n_rows; uint32_t col, bytes;
+                item_tokens(first + c * step, t0, n_rows, col, bytes);
+                const int32_t row = rows_sm[s][lane];
+                if (row >= 0 && row < P) {
+                    const int r = lane / K;
+                    bulk_store(send + static_cast<size_t>(row) * row_bytes + col,
+                               ring + static_cast<size_t>(s) * stage_bytes + static_cast<size_t>(r) * row_bytes,
+                               bytes);
+                } else if (row >= P) {
+                    flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+                }
+            }
+            bulk_commit();
+        }
+    }
+    bulk_wait_all();
+    if (!ok) {
+        if (lane == 0) flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
+        // give loads still in flight a bounded chance to land before the ring is released
+        for (int s = 0; s < kBulkStages; ++s) {
+            (void)mbar_wait(&full[s], 0);
+            (void)mbar_wait(&full[s], 1);
+        }
+    }
+}
+
+static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int K, int H, void* send,
+                       uint32_t flags, cudaStream_t stream)
+{
+    uint32_t* err_word = nullptr;
+    int rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+    int n_sm = 0;
+    rc = sm_count(&n_sm);
+    if (rc != COBALT_OK) return rc;
+    const int64_t P = T * K;
+    const uint32_t row_bytes = static_cast<uint32_t>(H) * 2u;
+    uint32_t impl = flags & COBALT_IMPL_MASK;
+    if (impl == 0) impl = COBALT_IMPL_BULK;
+
+    if (impl == COBALT_IMPL_VECTOR) {
+        const int n_vec = H / 8;
+        const unsigned grid = static_cast<unsigned>(T < 16ll * n_sm ? T : 16ll * n_sm);
+        const uint4* xs = static_cast<const uint4*>(x);
+        uint4* out = static_cast<uint4*>(send);
+#define COBALT_ROWS_CASE(KT)                                                                              \
+    case KT:                                                                                              \
+        perm_rows_vector_kernel<KT><<<grid, 256, 0, stream>>>(xs, row_of_pair, T, K, n_vec, P, out, err_word); \
+        break
+        switch (K) {
+            COBALT_ROWS_CASE(1);
+            COBALT_ROWS_CASE(2);
+            COBALT_ROWS_CASE(4);
+            COBALT_ROWS_CASE(6);
+            COBALT_ROWS_CASE(8);
+            default:
+                perm_rows_vector_kernel<0><<<grid, 256, 0, stream>>>(xs, row_of_pair, T, K, n_vec, P, out, err_word);
+        }
+#undef COBALT_ROWS_CASE
+        COBALT_CUDA_TRY(cudaGetLastError());
+        return COBALT_OK;
+    }
+
+    // bulk variant: pick the work-item shape
+    int rows_per_item = 1, n_seg = 1;
+    uint32_t seg_bytes = row_bytes;
+    if (row_bytes <= static_cast<uint32_t>(kBulkMaxStageBytes)) {
+        rows_per_item = kBulkMaxStageBytes / row_bytes;
+        if (rows_per_item > 32 / K) rows_per_item = 32 / K;
+        if (rows_per_item < 1) rows_per_item = 1;
+    } else {
+        n_seg = (row_bytes + kBulkMaxStageBytes - 1) / kBulkMaxStageBytes;
+        seg_bytes = static_cast<uint32_t>(round_up((row_bytes + n_seg - 1) / n_seg, 16));
+        n_seg = (row_bytes + seg_bytes - 1) / seg_bytes;
+    }
+    const uint32_t stage_bytes =
+        static_cast<uint32_t>(round_up(n_seg == 1 ? static_cast<size_t>(rows_per_item) * row_bytes : seg_bytes, 128));
+    const int64_t n_items = (n_seg == 1) ? (T + rows_per_item - 1) / rows_per_item : T * n_seg;
+    const size_t smem = static_cast<size_t>(kBulkStages) * stage_bytes;
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem)));
+    int per_sm = static_cast<int>((220 * 1024) / (smem + 1024));
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 8) per_sm = 8;
+    int64_t grid = static_cast<int64_t>(n_sm) * per_sm;
+    if (grid > n_items) grid = n_items;
+    perm_rows_bulk_kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
+        static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
+        stage_bytes, n_items, static_cast<uint8_t*>(send), err_word);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
+static int check_index_args(int64_t T, int32_t K, int32_t D)
+{
+    if (T < 0 || K < 1 || D < 1) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || D > COBALT_MAX_DESTS || T * static_cast<int64_t>(K) >= (1ll << 31))
+        return COBALT_ERR_UNSUPPORTED;
+    return COBALT_OK;
+}
+
+}  // namespace cobalt
+
+using namespace cobalt;
+
+extern "C" {
+
+size_t cobalt_permute_workspace_bytes(int64_t T, int32_t K, int32_t D)
+{
+    if (check_index_args(T, K, D) != COBALT_OK) return 0;
+    const ChunkPlan c = plan_chunks(T * K);
+    return round_up(static_cast<size_t>(D) * c.n_chunks * sizeof(uint32_t), 256);
+}
+
+int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
+                         uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                         int32_t* pair_of_row, void* workspace, size_t workspace_bytes,
+                         cobalt_stream_t stream)
+{
+    int rc = check_index_args(T, K, D);
+    if (rc != COBALT_OK) return rc;
+    if (!dest_counts || !dest_offsets) return COBALT_ERR_INVALID_ARG;
+    if (T > 0 && (!assigned_slot || !row_of_pair)) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(assigned_slot) || !aligned16(row_of_pair) || !aligned16(pair_of_row) ||
+        !aligned16(dest_counts) || !aligned16(dest_offsets) || !aligned16(workspace))
+        return COBALT_ERR_INVALID_ARG;
+    const size_t need = cobalt_permute_workspace_bytes(T, K, D);
+    if (!workspace || workspace_bytes < need) return COBALT_ERR_WORKSPACE_TOO_SMALL;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t P = T * K;
+    const ChunkPlan c = plan_chunks(P);
+    uint32_t* ws = static_cast<uint32_t*>(workspace);
+    uint32_t* err_word = nullptr;
+    rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+
+    perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
+                                                                            c.n_chunks, ws, err_word);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    perm_scan_kernel<<<(D + kPermWarps - 1) / kPermWarps, kPermThreads, 0, s>>>(ws, D, c.n_chunks, dest_counts);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
+    if (smem > 48 * 1024)
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem)));
+    perm_rank_kernel<<<c.n_chunks, kPermThreads, smem, s>>>(assigned_slot, P, D, c.chunk, c.n_chunks, ws,
+                                                            dest_counts, dest_offsets, row_of_pair, pair_of_row);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
+int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
+                        void* send, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1 || H < 1) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31))
+        return COBALT_ERR_UNSUPPORTED;
+    if (T == 0) return COBALT_OK;
+    if (!x || !row_of_pair || !send) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(send) || !aligned16(row_of_pair)) return COBALT_ERR_INVALID_ARG;
+    const uint32_t impl = flags & COBALT_IMPL_MASK;
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK) return COBALT_ERR_INVALID_ARG;
+    return launch_rows(x, row_of_pair, T, K, H, send, flags, static_cast<cudaStream_t>(stream));
+}
+
+int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D, const void* x, int32_t H,
+                   void* send, uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                   int32_t* pair_of_row, uint32_t flags, void* workspace, size_t workspace_bytes,
+                   cobalt_stream_t stream)
+{
+    // validate the row half first so that nothing is enqueued on a bad argument
+    if (H < 1) return COBALT_ERR_INVALID_ARG;
+    if (H % 8 != 0) return COBALT_ERR_UNSUPPORTED;
+    if (T > 0 && (!x || !send)) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(send)) return COBALT_ERR_INVALID_ARG;
+    const uint32_t impl = flags & COBALT_IMPL_MASK;
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK) return COBALT_ERR_INVALID_ARG;
+    int rc = cobalt_permute_index(assigned_slot, T, K, D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
+                                  workspace, workspace_bytes, stream);
+    if (rc != COBALT_OK) return rc;
+    return cobalt_permute_rows(x, row_of_pair, T, K, H, send, flags, stream);
+}
+
+}  // extern "C"

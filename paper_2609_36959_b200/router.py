@@ -1,0 +1,95 @@
+"""Device buffers for one routing step and the four-stage call sequence.
+
+Plumbing only: torch allocates the buffers once (the C library allocates nothing per call)
+and every stage below is one C-ABI call into the CUDA kernels, enqueued on the current torch
+stream.  `route()` works on data already resident on the device; `route_host()` is the same
+step driven from pinned host buffers (inputs copied in, results copied out).
+"""
+from __future__ import annotations
+
+from typing import Callable, Optional
+
+import torch
+
+from . import binding as cb
+
+
+class RouteStep:
+    def __init__(self, layout: "cb.Layout", T: int, K: int, H: int, device: Optional[torch.device] = None,
+                 alias_expert_out: bool = True):
+        self.layout, self.T, self.K, self.H = layout, T, K, H
+        self.E, self.D, self.P = layout.E, layout.D, T * K
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+        self.device = dev
+
+        def z(shape, dtype):
+            return torch.zeros(shape, dtype=dtype, device=dev)
+
+        # inputs
+        self.topk_ids = z((T, K), torch.int32)
+        self.gate_w = z((T, K), torch.float32)
+        self.src_rank = z((T,), torch.int32)
+        self.x = z((T, H), torch.bfloat16)
+        # stage outputs
+        self.coact = z((self.E, self.E), torch.int32)
+        self.load = z((self.E,), torch.int32)
+        self.assigned_slot = z((T, K), torch.int32)
+        self.slot_load = z((self.D,), torch.int32)
+        self.remote_nodes = z((T,), torch.uint8)
+        self.totals = z((2,), torch.int64)
+        self.dest_counts = z((self.D,), torch.int32)
+        self.dest_offsets = z((self.D + 1,), torch.int32)
+        self.row_of_pair = z((self.P,), torch.int32)
+        self.pair_of_row = z((self.P,), torch.int32)
+        self.send = z((self.P, H), torch.bfloat16)
+        # without real experts between dispatch and combine, combine may read the send buffer
+        self.expert_out = self.send if alias_expert_out else z((self.P, H), torch.bfloat16)
+        self.y = z((T, H), torch.bfloat16)
+        ws = max(cb.coact_stats_workspace_bytes(T, K, self.E), cb.assign_workspace_bytes(layout, T, K),
+                 cb.permute_workspace_bytes(T, K, self.D), 256)
+        self.workspace = torch.empty((ws,), dtype=torch.uint8, device=dev)
+
+    # -- the four stages, device-resident --------------------------------------------------
+    def stats(self, flags: int = 0) -> None:
+        cb.coact_stats(self.topk_ids, self.E, self.coact, self.load, flags=flags, workspace=self.workspace)
+
+    def assign(self, seed: int, flags: int = 0) -> None:
+        cb.assign(self.layout, self.topk_ids, self.src_rank, seed, self.assigned_slot, slot_load=self.slot_load,
+                  remote_nodes=self.remote_nodes, totals=self.totals, flags=flags, workspace=self.workspace)
+
+    def permute(self, flags: int = 0) -> None:
+        cb.permute(self.assigned_slot, self.D, self.x, self.send, self.dest_counts, self.dest_offsets,
+                   self.row_of_pair, self.pair_of_row, self.workspace, flags=flags)
+
+    def combine(self, flags: int = 0) -> None:
+        cb.combine(self.expert_out, self.row_of_pair, self.gate_w, self.y, flags=flags)
+
+    def route(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None) -> None:
+        """stats -> assign -> permute -> [experts(send, expert_out)] -> combine on the current stream."""
+        self.stats()
+        self.assign(seed)
+        self.permute()
+        if experts is not None:
+            experts(self.send, self.expert_out)
+        self.combine()
+
+    # -- the same step from pinned host memory ----------------------------------------------
+    def route_host(self, seed: int, ids_h: torch.Tensor, w_h: torch.Tensor, src_h: torch.Tensor,
+                   x_h: torch.Tensor, y_h: torch.Tensor, coact_h: torch.Tensor, load_h: torch.Tensor,
+                   slot_load_h: torch.Tensor, totals_h: torch.Tensor) -> None:
+        self.topk_ids.copy_(ids_h, non_blocking=True)
+        self.gate_w.copy_(w_h, non_blocking=True)
+        self.src_rank.copy_(src_h, non_blocking=True)
+        self.x.copy_(x_h, non_blocking=True)
+        self.route(seed)
+        y_h.copy_(self.y, non_blocking=True)
+        coact_h.copy_(self.coact, non_blocking=True)
+        load_h.copy_(self.load, non_blocking=True)
+        slot_load_h.copy_(self.slot_load, non_blocking=True)
+        totals_h.copy_(self.totals, non_blocking=True)
+
+    def h2d_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.topk_ids, self.gate_w, self.src_rank, self.x))
+
+    def d2h_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.y, self.coact, self.load, self.slot_load, self.totals))

@@ -1,0 +1,315 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Integer outputs must be bit-identical; the combine must satisfy
+|gpu - oracle| <= 1e-2 + 1e-2 |oracle| against the oracle's fp32 accumulation."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import workloads as W
+from gpu_util import (assert_combine_close, bf16_tensor_from_bits, bits_from_bf16_tensor, make_step,
+                      oracle_assign, u32)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def cb():
+    import paper_2609_36959_b200 as cb
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return cb
+
+
+def check_index_stages(cb, w, step, seed):
+    """stats, assign and the index half of permute, compared in full. Returns the oracle results."""
+    step.stats()
+    step.assign(seed)
+    cb.permute_index(step.assigned_slot, w.D, step.dest_counts, step.dest_offsets, step.row_of_pair,
+                     step.pair_of_row, step.workspace)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+
+    coact, load = O.coact_stats(w.topk_ids, w.E)
+    assert (u32(step.coact) == coact).all()
+    assert (u32(step.load) == load).all()
+
+    r = oracle_assign(w, seed)
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    assert (u32(step.slot_load) == r["slot_load"]).all()
+    assert (step.remote_nodes.cpu().numpy() == r["remote_nodes"]).all()
+    assert step.totals.cpu().tolist() == [r["V"], r["V_naive"]]
+
+    p = O.permute(r["assigned_slot"], w.D)
+    assert (u32(step.dest_counts) == p["dest_counts"]).all()
+    assert (u32(step.dest_offsets) == p["dest_offsets"]).all()
+    assert (step.row_of_pair.cpu().numpy() == p["row_of_pair"]).all()
+    assert (step.pair_of_row.cpu().numpy() == p["pair_of_row"]).all()
+    return r, p
+
+
+# ---------------------------------------------------------------------------------------------
+# the benchmark configs at sizes the oracle handles in full
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["1", "1a", "2", "3"])
+def test_config_full_elementwise(cb, name):
+    w = W.make_config(name)
+    layout, step = make_step(w, alias_expert_out=False)
+    r, p = check_index_stages(cb, w, step, w.seed)
+
+    x = w.hidden_rows()
+    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR, 0):
+        step.send.zero_()
+        step.permute(flags=impl)
+        torch.cuda.synchronize()
+        send = bits_from_bf16_tensor(step.send)
+        assert (send == x[p["pair_of_row"] // w.K]).all(), f"impl {impl:#x}"
+        assert (step.row_of_pair.cpu().numpy() == p["row_of_pair"]).all()
+
+    out = w.expert_out_rows()
+    step.expert_out.copy_(bf16_tensor_from_bits(out, "cpu"))
+    step.combine()
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    assert_combine_close(bits_from_bf16_tensor(step.y), O.combine(out, p["row_of_pair"], w.gate_w))
+
+
+@pytest.mark.parametrize("name", ["4", "5"])
+def test_config_full_size_sampled(cb, name):
+    """Largest configs in the launch configuration the bench times: index outputs in full,
+    payload on sampled rows/tokens, plus properties that hold at any size."""
+    w = W.make_config(name)
+    layout, step = make_step(w, alias_expert_out=True)
+    r, p = check_index_stages(cb, w, step, w.seed)
+
+    step.permute()
+    step.combine()                    # identity experts: expert_out aliases send
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+
+    rng = np.random.default_rng(5)
+    offs = p["dest_offsets"].astype(np.int64)
+    edges = np.concatenate([offs[:-1], offs[1:] - 1])
+    edges = edges[(edges >= 0) & (edges < w.P)]
+    rows = np.unique(np.concatenate([rng.integers(0, w.P, 3000), edges, [0, w.P - 1]]))
+    got = bits_from_bf16_tensor(step.send[torch.from_numpy(rows).cuda()])
+    tok = p["pair_of_row"][rows] // w.K
+    x_bits = bits_from_bf16_tensor(step.x[torch.from_numpy(tok).cuda()])
+    # x on the device is the uploaded generator output; compare against freshly generated rows too
+    some = tok[:64]
+    for t, xb in zip(some, x_bits[:64]):
+        assert (w.hidden_rows(int(t), int(t) + 1)[0] == xb).all()
+    assert (got == x_bits).all()
+
+    tokens = np.unique(np.concatenate([rng.integers(0, w.T, 1500), [0, w.T - 1]]))
+    rop = p["row_of_pair"].reshape(w.T, w.K)[tokens]                     # [n, K]
+    rows_needed = bits_from_bf16_tensor(step.expert_out[torch.from_numpy(rop.ravel()).cuda()])
+    y_ref = O.combine(rows_needed, np.arange(rop.size, dtype=np.int32), w.gate_w[tokens])
+    y_gpu = bits_from_bf16_tensor(step.y[torch.from_numpy(tokens).cuda()])
+    assert_combine_close(y_gpu, y_ref)
+
+    # any-size properties: identity experts and weights summing to one give back x (bf16 rounding)
+    diff = (step.y.float() - step.x.float()).abs()
+    bound = 2.0 ** -7 * step.x.float().abs() + 1e-6
+    assert bool((diff <= bound).all())
+    # every send row equals the row of the token its pair belongs to (checked on the device)
+    tok_of_row = (step.pair_of_row // w.K).long()
+    n_chunk = 1 << 16
+    for r0 in range(0, w.P, n_chunk * 16):
+        r1 = min(w.P, r0 + n_chunk)
+        same = step.send[r0:r1].view(torch.int16) == step.x[tok_of_row[r0:r1]].view(torch.int16)
+        assert bool(same.all())
+
+
+# ---------------------------------------------------------------------------------------------
+# edge shapes
+# ---------------------------------------------------------------------------------------------
+EDGE = [
+    # T, E, K, H, N, Q, S, empty
+    (1, 4, 1, 8, 1, 2, 2, 0),
+    (1, 8, 3, 24, 2, 2, 2, 0),
+    (7, 9, 2, 40, 3, 2, 2, 1),
+    (33, 13, 3, 72, 4, 2, 3, 2),
+    (1000, 20, 5, 136, 8, 1, 5, 0),
+    (1000, 24, 6, 264, 4, 3, 3, 3),
+    (2049, 40, 8, 520, 2, 4, 6, 0),
+    (4099, 100, 16, 64, 4, 8, 5, 7),
+    (5000, 257, 7, 32, 4, 4, 20, 0),
+    (3000, 17, 4, 16392, 2, 2, 5, 0),     # a row larger than one pipeline stage
+    (70000, 6, 2, 8, 4, 2, 1, 0),
+]
+
+
+@pytest.mark.parametrize("T,E,K,H,N,Q,S,empty", EDGE)
+def test_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
+    w = W.make_custom(T, E, K, H, N, Q, S, seed=1000 + T + E, C=3, p_in=0.6, n_empty=empty)
+    layout, step = make_step(w, alias_expert_out=False)
+    r, p = check_index_stages(cb, w, step, 4242)
+    x = w.hidden_rows()
+    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR):
+        step.send.zero_()
+        step.permute(flags=impl)
+        torch.cuda.synchronize()
+        assert (bits_from_bf16_tensor(step.send) == x[p["pair_of_row"] // K]).all()
+    out = w.expert_out_rows()
+    step.expert_out.copy_(bf16_tensor_from_bits(out, "cpu"))
+    step.combine()
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    assert_combine_close(bits_from_bf16_tensor(step.y), O.combine(out, p["row_of_pair"], w.gate_w))
+
+
+def test_large_expert_count_takes_global_path(cb):
+    """E = 700: the co-activation triangle exceeds shared memory."""
+    w = W.make_custom(6000, 700, 8, 8, 4, 8, 24, seed=3, C=7, p_in=0.7)
+    layout, step = make_step(w, with_x=False)
+    check_index_stages(cb, w, step, 9)
+
+
+def test_empty_batch(cb):
+    w = W.make_custom(0, 8, 2, 16, 2, 2, 3, seed=1)
+    layout, step = make_step(w)
+    step.route(5)
+    torch.cuda.synchronize()
+    assert int(step.coact.sum()) == 0 and int(step.slot_load.sum()) == 0
+    assert step.dest_offsets.cpu().tolist() == [0] * (w.D + 1)
+    assert step.totals.cpu().tolist() == [0, 0]
+
+
+# ---------------------------------------------------------------------------------------------
+# modes and flags
+# ---------------------------------------------------------------------------------------------
+def test_naive_rule_and_uniform_source(cb):
+    w = W.make_config("3", T=5000)
+    layout, step = make_step(w, with_x=False)
+    step.assign(w.seed, flags=cb.ASSIGN_NAIVE)
+    torch.cuda.synchronize()
+    r = oracle_assign(w, w.seed, naive=True)
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    assert (step.remote_nodes.cpu().numpy() == r["remote_nodes"]).all()
+    assert step.totals.cpu().tolist() == [r["V"], r["V_naive"]]
+
+    w.src_rank[:] = 13
+    cb.assign(layout, step.topk_ids, 13, 77, step.assigned_slot, slot_load=step.slot_load,
+              remote_nodes=step.remote_nodes, totals=step.totals)
+    torch.cuda.synchronize()
+    r = oracle_assign(w, 77)
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    assert (u32(step.slot_load) == r["slot_load"]).all()
+    # optional outputs may be skipped
+    out = torch.zeros_like(step.assigned_slot)
+    cb.assign(layout, step.topk_ids, 13, 77, out)
+    torch.cuda.synchronize()
+    assert (out.cpu().numpy() == r["assigned_slot"]).all()
+
+
+def test_fig1_layout_on_gpu(cb, fig1):
+    g = fig1
+    ids = np.array([tk["ids"] for tk in g["tokens"]], np.int32)
+    src = np.array([tk["src"] for tk in g["tokens"]], np.int32)
+    layout = cb.Layout(2, 2, 2, 4, g["slot_expert"], g["primary_slot"])
+    out = torch.zeros((12, 2), dtype=torch.int32, device="cuda")
+    remote = torch.zeros(12, dtype=torch.uint8, device="cuda")
+    totals = torch.zeros(2, dtype=torch.int64, device="cuda")
+    cb.assign(layout, torch.from_numpy(ids).cuda(), torch.from_numpy(src).cuda(), 36959, out,
+              remote_nodes=remote, totals=totals)
+    torch.cuda.synchronize()
+    assert remote.cpu().tolist() == [tk["cobalt"] for tk in g["tokens"]]
+    assert totals.cpu().tolist() == [g["V_cobalt"], g["V_naive"]]
+    for seed, t, k, slot in g["seeded"]:
+        assert int(out[t, k]) == slot
+
+
+def test_stats_accumulate_flag(cb):
+    w = W.make_config("3", T=3000)
+    layout, step = make_step(w, with_x=False)
+    step.stats()
+    step.stats(flags=cb.STATS_ACCUMULATE)
+    torch.cuda.synchronize()
+    coact, load = O.coact_stats(w.topk_ids, w.E)
+    assert (u32(step.coact) == 2 * coact).all() and (u32(step.load) == 2 * load).all()
+    step.stats()
+    torch.cuda.synchronize()
+    assert (u32(step.coact) == coact).all()
+
+
+def test_results_do_not_depend_on_the_run(cb):
+    w = W.make_config("4", T=30000)
+    layout, step = make_step(w)
+    step.route(w.seed)
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (step.coact, step.assigned_slot, step.row_of_pair, step.pair_of_row, step.send, step.y)]
+    for _ in range(5):
+        step.route(w.seed)
+        torch.cuda.synchronize()
+        for a, b in zip(ref, (step.coact, step.assigned_slot, step.row_of_pair, step.pair_of_row, step.send, step.y)):
+            assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                               b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+
+
+def test_round_trip_identity_and_one_hot(cb):
+    w = W.make_config("2", T=4000)
+    layout, step = make_step(w)
+    step.gate_w.zero_()
+    pick = torch.arange(w.T, device="cuda") % w.K
+    step.gate_w[torch.arange(w.T, device="cuda"), pick] = 1.0
+    step.route(w.seed)
+    torch.cuda.synchronize()
+    # one-hot weights select exactly one expert row = the token's own row
+    assert torch.equal(step.y.view(torch.int16), step.x.view(torch.int16))
+
+
+# ---------------------------------------------------------------------------------------------
+# bad data and bad arguments: flagged, never faulting
+# ---------------------------------------------------------------------------------------------
+def test_bad_data_sets_the_error_word(cb):
+    w = W.make_config("1", T=2000)
+    layout, step = make_step(w)
+    good = oracle_assign(w, 3)
+    ids = w.topk_ids.copy()
+    ids[10, 0] = w.E + 5           # out of range
+    ids[20, 1] = ids[20, 0]        # duplicate
+    step.topk_ids.copy_(torch.from_numpy(ids))
+    step.src_rank[30] = w.G        # bad source rank
+    step.stats()
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == cb.DEVERR_BAD_EXPERT_ID | cb.DEVERR_DUPLICATE_ID
+    step.assign(3)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == (cb.DEVERR_BAD_EXPERT_ID | cb.DEVERR_DUPLICATE_ID |
+                                                cb.DEVERR_BAD_SRC_RANK)
+    got = step.assigned_slot.cpu().numpy()
+    keep = np.ones(w.T, bool)
+    keep[[10, 20, 30]] = False
+    assert (got[keep] == good["assigned_slot"][keep]).all()      # other tokens unaffected
+    assert (got[~keep] == -1).all()
+    assert int(step.slot_load.sum()) == (w.T - 3) * w.K
+    # the permutation skips the pairs without a slot and says so
+    step.permute()
+    step.combine()
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() & cb.DEVERR_BAD_SLOT
+    assert int(step.dest_offsets[-1]) == (w.T - 3) * w.K
+    assert cb.read_and_clear_device_error() == 0
+
+
+def test_argument_checks(cb):
+    w = W.make_config("1", T=256)
+    layout, step = make_step(w)
+    small = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(cb.CobaltError) as e:
+        cb.permute_index(step.assigned_slot, w.D, step.dest_counts, step.dest_offsets, step.row_of_pair,
+                         step.pair_of_row, small)
+    assert e.value.status == cb.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(cb.CobaltError) as e:
+        cb.assign(layout, step.topk_ids, w.G, 1, step.assigned_slot)       # uniform source rank out of range
+    assert e.value.status == cb.ERR_INVALID_ARG
+    x7 = torch.zeros((w.T, 12), dtype=torch.bfloat16, device="cuda")
+    send7 = torch.zeros((w.P, 12), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(cb.CobaltError) as e:
+        cb.permute_rows(x7, step.row_of_pair, w.K, send7)                   # H not a multiple of 8
+    assert e.value.status == cb.ERR_UNSUPPORTED
+    with pytest.raises(cb.CobaltError) as e:
+        cb.Layout(2, 2, 2, 4, [0, 0, 2, 0, 1, 2, 3, 0])
+    assert e.value.status == cb.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0

@@ -14,6 +14,8 @@ per-expert popularity pi.  Ids are kept in draw order.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 from typing import Optional
 
@@ -197,11 +199,19 @@ class Workload:
     def _rows(self, stream: int, r0: int, r1: int) -> np.ndarray:
         out = np.empty((r1 - r0, self.H), dtype=np.uint16)
         b0, b1 = r0 // _ROW_BLOCK, (r1 + _ROW_BLOCK - 1) // _ROW_BLOCK
-        for blk in range(b0, b1):
+
+        def fill(blk: int) -> None:
             lo, hi = blk * _ROW_BLOCK, (blk + 1) * _ROW_BLOCK
             vals = _rng(self.seed, stream, blk).standard_normal((_ROW_BLOCK, self.H), dtype=np.float32)
             a, b = max(lo, r0), min(hi, r1)
             out[a - r0:b - r0] = bf16_bits_from_f32(vals[a - lo:b - lo])
+
+        if b1 - b0 > 8:   # blocks are independent streams: draw them on several host threads
+            with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+                list(pool.map(fill, range(b0, b1)))
+        else:
+            for blk in range(b0, b1):
+                fill(blk)
         return out
 
     def hidden_rows(self, t0: int = 0, t1: Optional[int] = None) -> np.ndarray:
