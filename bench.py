@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the token-routing hot path (stats -> assign -> permute -> combine) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--impl reference]
+
+One "step" is one pass of all four stages over one batch of synthetic gating output.  The
+default workload is the largest benchmark config (T=131072, E=256, K=8, H=7168, 4x8 ranks).
+Rank 0 prints ONE JSON line: whole-job routed (token, expert) pairs per second with inputs
+resident in HBM (`value`), the same step driven from pinned host buffers (`e2e`), the HBM
+roofline of the dominant kernel (`roofline`) and of every stage (`stages`), the CPU oracle
+timed on a bounded sample (`cpu_baseline`), and the SM clocks seen during the timed region.
+With --gpus N > 1 (launched by torchrun) every rank routes its own replica of the workload:
+the path has no cross-GPU step, so scaling is weak and no collective is on the data path.
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import datetime
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "routed token-expert pairs/sec"
+UNIT = "pairs/s"
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
+KERNELS_PER_STEP = 7               # stats 1, assign 1, permute 4 (hist, scan, rank, rows), combine 1
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (bytes per pair, measured on a reduced token count and scaled by the pairs of a launch)
+NCU_TRAFFIC_BYTES_PER_PAIR = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="5")
+    ap.add_argument("--tokens", type=int, default=None, help="override T (reduced-size runs for profiling)")
+    ap.add_argument("--impl", default="cobalt", choices=["cobalt", "reference"])
+    ap.add_argument("--cpu-sample-tokens", type=int, default=None,
+                    help="tokens of the workload the CPU oracle is timed on (default 32768; 8192 for --impl reference)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(w, T=None):
+    T = w.T if T is None else T
+    return (f"config {w.name}: T={T} E={w.E} K={w.K} H={w.H} bf16, layout {w.N} nodes x {w.Q} ranks x "
+            f"{w.S} slots (D={w.D}), P={T * w.K} pairs")
+
+
+def stage_bytes(w):
+    """Algorithmic bytes each stage must move (ids/maps int32, rows bf16)."""
+    T, K, E, H, D, P = w.T, w.K, w.E, w.H, w.D, w.P
+    return {
+        "coact_stats": 4 * P + 4 * E * E + 4 * E,
+        "assign": 4 * P + 4 * T + 4 * P + 4 * D + T,
+        "permute_index": 4 * P + 4 * P + 4 * P + 4 * (2 * D + 1),
+        "permute_rows": 2 * T * H + 2 * P * H + 4 * P,
+        "combine": 2 * P * H + 2 * T * H + 4 * P + 4 * P,
+    }
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# ---------------------------------------------------------------------------------------------
+def oracle_step(w, x_bits):
+    """All four stages of the oracle, as it stands, on the host. Returns seconds."""
+    import oracle as O
+    t0 = time.perf_counter()
+    O.coact_stats(w.topk_ids, w.E)
+    r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, w.seed)
+    p = O.permute(r["assigned_slot"], w.D, x_bits)
+    O.combine(p["send"], p["row_of_pair"], w.gate_w)
+    return time.perf_counter() - t0
+
+
+def cpu_sample(config, tokens):
+    import workloads as W
+    w = W.make_config(config, T=tokens)
+    return w, w.hidden_rows()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w, x_bits = cpu_sample(args.config, args.cpu_sample_tokens or 8192)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_step(w, x_bits)
+    budget_s = 120.0
+    times = []
+    for _ in range(max(1, args.steps)):
+        times.append(oracle_step(w, x_bits))
+        if sum(times) > budget_s:
+            break
+    sec = sum(times) / len(times)
+    value = w.P / sec
+    name = workload_name(w, T=args.tokens or _default_T(args.config))
+    sample = f"first {w.T} tokens of the workload ({w.P} pairs), all four stages, single thread"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def _default_T(config):
+    return {"1": 4096, "1a": 4096, "2": 16384, "3": 32768, "4": 65536, "5": 131072}[str(config)]
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, device_id):
+        self.proc = None
+        self.device_index = device_id      # an index or a "GPU-<uuid>" string
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.device_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and throttle reasons over the samples taken inside [t_begin, t_end]
+        (wall-clock seconds since the epoch); all samples if no window is given or none fall in it."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.1)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        rows = []
+        for line in out.splitlines():
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[4:8]))
+            except ValueError:
+                continue
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        window = "timed region" if inside else "whole run (no sample fell inside the timed region)"
+        use = inside or rows
+        reasons = set()
+        for r in use:
+            for name, v in zip(self.NAMES, r[4]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
+                "sm_max_mhz": max(r[2] for r in use) if use else None,
+                "power_w_max": max(r[3] for r in use) if use else None,
+                "reasons": sorted(reasons), "samples": len(use), "window": window}
+
+
+# ---------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------
+def run_cobalt(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_36959_b200 as cb
+    import workloads as W
+    from paper_2609_36959_b200.router import RouteStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the routing path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    distributed = world > 1
+    if distributed:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = W.make_config(args.config, T=args.tokens)
+    layout = cb.Layout(w.N, w.Q, w.S, w.E, w.slot_expert.tolist(), w.primary_slot.tolist())
+    step = RouteStep(layout, w.T, w.K, w.H)
+
+    # pinned host copies of the inputs (the e2e leg reads them every step)
+    ids_h = torch.from_numpy(w.topk_ids).pin_memory()
+    w_h = torch.from_numpy(w.gate_w).pin_memory()
+    src_h = torch.from_numpy(w.src_rank).pin_memory()
+    x_h = torch.empty((w.T, w.H), dtype=torch.bfloat16).pin_memory()
+    blk = 16384
+    for t0 in range(0, w.T, blk):
+        t1 = min(w.T, t0 + blk)
+        x_h[t0:t1].copy_(torch.from_numpy(w.hidden_rows(t0, t1).view(np.int16)).view(torch.bfloat16))
+    step.topk_ids.copy_(ids_h); step.gate_w.copy_(w_h); step.src_rank.copy_(src_h); step.x.copy_(x_h)
+    torch.cuda.synchronize()
+
+    names = ["coact_stats", "assign", "permute_index", "permute_rows", "combine"]
+
+    def one_step(events=None):
+        def mark(i):
+            if events is not None:
+                events[i].record()
+        mark(0)
+        step.stats()
+        mark(1)
+        step.assign(w.seed)
+        mark(2)
+        # cobalt_permute is exactly these two calls; split so the row mover is timed on its own
+        cb.permute_index(step.assigned_slot, w.D, step.dest_counts, step.dest_offsets, step.row_of_pair,
+                         step.pair_of_row, step.workspace)
+        mark(3)
+        cb.permute_rows(step.x, step.row_of_pair, w.K, step.send)
+        mark(4)
+        step.combine()
+        mark(5)
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_id = local_rank
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(3, args.warmup)):
+        one_step()
+    barrier()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    barrier()
+    t_epoch0 = time.time()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        one_step(ev[i])
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop(t_epoch0, t_epoch0 + t_wall) if rank == 0 else None
+
+    total_ms = ev[0][0].elapsed_time(ev[-1][5])
+    stage_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in ev) / args.steps for i, n in enumerate(names)}
+    err_bits = cb.read_and_clear_device_error()
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if distributed:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * w.P / (ms_per_step * 1e-3)
+
+    # end to end from pinned host buffers: H2D of the inputs, four stages, D2H of the results
+    e2e = None
+    if not args.no_e2e:
+        y_h = torch.empty((w.T, w.H), dtype=torch.bfloat16).pin_memory()
+        coact_h = torch.empty((w.E, w.E), dtype=torch.int32).pin_memory()
+        load_h = torch.empty((w.E,), dtype=torch.int32).pin_memory()
+        sl_h = torch.empty((w.D,), dtype=torch.int32).pin_memory()
+        tot_h = torch.empty((2,), dtype=torch.int64).pin_memory()
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
+        e1.record()
+        barrier()
+        t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if distributed:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t2.item()) / n_e2e
+        e2e = {"value": world * w.P / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": step.h2d_bytes(), "d2h_bytes_per_step": step.d2h_bytes(), "steps": n_e2e}
+
+    if rank == 0:
+        peak, peak_src = hbm_peak()
+        sb = stage_bytes(w)
+        stages = {}
+        for n in names:
+            gbs = sb[n] / (stage_ms[n] * 1e-3) / 1e9
+            stages[n] = {"ms": stage_ms[n], "bytes": sb[n], "gbs": gbs, "frac": gbs / peak,
+                         "pairs_per_s": w.P / (stage_ms[n] * 1e-3)}
+        dom = max(("permute_rows", "combine"), key=lambda n: stage_ms[n])
+        traffic = NCU_TRAFFIC_BYTES_PER_PAIR.get(dom)
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": stages[dom]["gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": stages[dom]["frac"], "peak_source": peak_src,
+                    "traffic": None if traffic is None else traffic * w.P,
+                    "algorithmic_bytes": sb[dom], "ms_per_launch": stage_ms[dom]}
+        totals = step.totals.cpu().tolist()
+        load = step.slot_load.cpu().numpy().astype(np.int64).reshape(w.G, w.S).sum(axis=1)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 rows, u32 counts, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": workload_name(w), "seed": int(w.seed),
+                       "l2": "no explicit flush: each step streams the 15 GB send buffer through L2 twice, "
+                             "so every stage starts cold" if w.P * w.H * 2 > (1 << 28) else
+                             "inputs smaller than L2: stages run warm",
+                       "parallelism": "replicas only (no cross-GPU step on this path)"},
+            "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "roofline": roofline, "stages": stages, "clocks": clocks,
+            "traffic_model": {"V_cobalt": totals[0], "V_naive": totals[1],
+                              "cross_node_reduction": (1 - totals[0] / totals[1]) if totals[1] else None,
+                              "rank_load_imbalance": float(load.max() / load.mean()) if load.sum() else None},
+            "device_error_bits": err_bits, "wall_s_timed_region": t_wall,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            ws, xs = cpu_sample(args.config, min(args.cpu_sample_tokens or 32768, w.T))
+            sec = min(oracle_step(ws, xs), oracle_step(ws, xs))
+            line["cpu_baseline"] = {"value": ws.P / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": f"first {ws.T} tokens of the workload ({ws.P} pairs), all four "
+                                              f"stages, single thread, best of 2 runs, {sec:.2f} s each"}
+        print(json.dumps(line))
+    if distributed:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cobalt(args)
+
+
+if __name__ == "__main__":
+    main()
