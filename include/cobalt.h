@@ -49,6 +49,7 @@ extern "C" {
 #define COBALT_ERR_WORKSPACE_TOO_SMALL (-2)
 #define COBALT_ERR_UNSUPPORTED (-3)          /* outside the supported size envelope (see below) */
 #define COBALT_ERR_CUDA (-4)                 /* a CUDA runtime call failed; see cobalt_last_cuda_error */
+#define COBALT_ERR_SCRATCH_LIMIT (-5)        /* problem needs more than the library's built-in scratch */
 
 /* Supported envelope: N <= 8 nodes, K <= 16, E <= 1024, D <= 4096, P = T*K < 2^31,
  * H a multiple of 8 (rows are whole 16-byte vectors). */
@@ -151,6 +152,30 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
                    uint32_t* dest_offsets, int32_t* row_of_pair, int32_t* pair_of_row,
                    uint32_t flags, void* workspace, size_t workspace_bytes,
                    cobalt_stream_t stream);
+
+/* ---- index half of stage 3 for callers that cannot provide device scratch -------------------
+ * (No counterpart in the paper: this is a packaging variant of cobalt_permute_index, same
+ * inputs, same outputs, bit-identical results.)
+ * Some callers cannot allocate device memory where they call the library: code running inside
+ * a framework that forbids allocator calls on its hot path, plugins that receive nothing but
+ * their input and output buffers, and jobs whose memory pool was sized up front and is fully
+ * committed.  For them the per-chunk histogram scratch is a fixed array inside the library
+ * image, COBALT_STATIC_SCRATCH_WORDS uint32 (4 MiB), which every GPU that loads the library
+ * holds until the process exits.  The call needs D * ceil(P / chunk) words, where chunk is
+ * 2048 pairs (doubled until there are at most 2048 chunks); larger problems are refused with
+ * COBALT_ERR_SCRATCH_LIMIT and nothing is enqueued.  D = 288 fits for every P; D = 4096 fits up
+ * to P = 524288.  The call itself performs no device or host allocation.
+ * The first call on each device looks up the array's device address (with that device
+ * current) and caches it; make that first call outside any stream capture.
+ * All calls share the one array and it keeps whatever the previous call left there.  Nothing
+ * has to be cleared between calls, because the first kernel overwrites every word the later
+ * ones read, but two calls that overlap on the GPU (different streams, or different host
+ * threads without ordering) race on it: serialise them on one stream or with events. */
+#define COBALT_STATIC_SCRATCH_WORDS (1u << 20)
+int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
+                                uint32_t* dest_counts, uint32_t* dest_offsets,
+                                int32_t* row_of_pair, int32_t* pair_of_row,
+                                cobalt_stream_t stream);
 
 /* ---- stage 4: combine (Fig. 1, "Weighted sum"; Section 1) ----------------------------------
  * y[t][h] = bf16( sum_{k<K} gate_w[t*K+k] * float(expert_out[row_of_pair[t*K+k]][h]) ),

@@ -21,6 +21,8 @@ ERR_INVALID_ARG = -1
 ERR_WORKSPACE_TOO_SMALL = -2
 ERR_UNSUPPORTED = -3
 ERR_CUDA = -4
+ERR_SCRATCH_LIMIT = -5
+STATIC_SCRATCH_WORDS = 1 << 20
 
 DEVERR_BAD_EXPERT_ID = 0x1
 DEVERR_DUPLICATE_ID = 0x2
@@ -40,6 +42,7 @@ EXPORTS = (
     "cobalt_coact_stats_workspace_bytes", "cobalt_coact_stats",
     "cobalt_assign_workspace_bytes", "cobalt_assign",
     "cobalt_permute_workspace_bytes", "cobalt_permute_index", "cobalt_permute_rows", "cobalt_permute",
+    "cobalt_permute_index_static",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -71,6 +74,7 @@ def _load() -> C.CDLL:
         "cobalt_assign": (C.c_int, [vp, vp, vp, i32, i64, i32, u64, vp, vp, vp, vp, u32, vp, sz, vp]),
         "cobalt_permute_workspace_bytes": (sz, [i64, i32, i32]),
         "cobalt_permute_index": (C.c_int, [vp, i64, i32, i32, vp, vp, vp, vp, vp, sz, vp]),
+        "cobalt_permute_index_static": (C.c_int, [vp, i64, i32, i32, vp, vp, vp, vp, vp]),
         "cobalt_permute_rows": (C.c_int, [vp, vp, i64, i32, i32, vp, u32, vp]),
         "cobalt_permute": (C.c_int, [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, vp, u32, vp, sz, vp]),
         "cobalt_combine": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, u32, vp]),
@@ -242,6 +246,25 @@ def permute_index(assigned_slot: torch.Tensor, D: int, dest_counts: torch.Tensor
                                      _ptr(row_of_pair, torch.int32, "row_of_pair"),
                                      _ptr(pair_of_row, torch.int32, "pair_of_row"),
                                      _ptr(workspace), _ws_bytes(workspace), _stream()), "cobalt_permute_index")
+
+
+def permute_index_static(assigned_slot: torch.Tensor, D: int, dest_counts: torch.Tensor,
+                         dest_offsets: torch.Tensor, row_of_pair: torch.Tensor,
+                         pair_of_row: Optional[torch.Tensor]) -> None:
+    """permute_index for callers that cannot hand over device scratch (a framework hot path that
+    bans allocator calls, a plugin given only its inputs and outputs, a fully committed memory
+    pool): the scratch is a fixed 4 MiB array inside the library.  Same outputs as
+    permute_index; raises with ERR_SCRATCH_LIMIT when D * chunks exceeds STATIC_SCRATCH_WORDS.
+    Calls share that array, so do not let two of them overlap on the GPU; make the first call
+    on a device outside stream capture (it looks up the array's address)."""
+    T, K = assigned_slot.shape
+    _check_index_outputs(T, K, D, dest_counts, dest_offsets, row_of_pair, pair_of_row, "permute_index_static")
+    _check(_lib.cobalt_permute_index_static(_ptr(assigned_slot, torch.int32, "assigned_slot"), T, K, D,
+                                            _ptr(dest_counts, torch.int32, "dest_counts"),
+                                            _ptr(dest_offsets, torch.int32, "dest_offsets"),
+                                            _ptr(row_of_pair, torch.int32, "row_of_pair"),
+                                            _ptr(pair_of_row, torch.int32, "pair_of_row"), _stream()),
+           "cobalt_permute_index_static")
 
 
 def permute_rows(x: torch.Tensor, row_of_pair: torch.Tensor, K: int, send: torch.Tensor, *, flags: int = 0) -> None:

@@ -490,6 +490,78 @@ int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int
     return COBALT_OK;
 }
 
+// ---- no-allocation variant of the index half ------------------------------------------------
+// Same three kernels as cobalt_permute_index, but the per-chunk histogram scratch lives in a
+// fixed device array that is part of the library image instead of a caller-provided buffer.
+// It is meant for callers that have no way to obtain device scratch at the point of the call:
+// code running under a framework that forbids allocator calls on its hot path, plugins that are
+// handed only their input and output buffers, and processes whose memory pool was sized up
+// front and is already fully committed.  Every GPU that loads the library carries the array
+// (COBALT_STATIC_SCRATCH_WORDS * 4 bytes) until the process exits.
+static __device__ __align__(256) uint32_t g_static_perm_scratch[COBALT_STATIC_SCRATCH_WORDS];
+
+// The array's name is only a host-side handle; the kernels need its device address, looked up
+// once per device (with that device current) and cached here.
+static uint32_t* g_static_perm_scratch_ptr[64] = {nullptr};
+
+static int static_scratch_address(uint32_t** out)
+{
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && g_static_perm_scratch_ptr[dev]) {
+        *out = g_static_perm_scratch_ptr[dev];
+        return COBALT_OK;
+    }
+    uint32_t* ptr = nullptr;
+    COBALT_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_perm_scratch));
+    if (!ptr) return COBALT_ERR_CUDA;
+    if (dev >= 0 && dev < 64) g_static_perm_scratch_ptr[dev] = ptr;
+    *out = ptr;
+    return COBALT_OK;
+}
+
+int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
+                                uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                                int32_t* pair_of_row, cobalt_stream_t stream)
+{
+    int rc = check_index_args(T, K, D);
+    if (rc != COBALT_OK) return rc;
+    if (!dest_counts || !dest_offsets) return COBALT_ERR_INVALID_ARG;
+    if (T > 0 && (!assigned_slot || !row_of_pair)) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(assigned_slot) || !aligned16(row_of_pair) || !aligned16(pair_of_row) ||
+        !aligned16(dest_counts) || !aligned16(dest_offsets))
+        return COBALT_ERR_INVALID_ARG;
+    const int64_t P = T * K;
+    const ChunkPlan c = plan_chunks(P);
+    if (static_cast<int64_t>(D) * c.n_chunks > static_cast<int64_t>(COBALT_STATIC_SCRATCH_WORDS))
+        return COBALT_ERR_SCRATCH_LIMIT;
+
+    uint32_t* ws = nullptr;
+    rc = static_scratch_address(&ws);
+    if (rc != COBALT_OK) return rc;
+    uint32_t* err_word = nullptr;
+    rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+
+    // The histogram kernel stores every scratch word the later kernels read (all D x n_chunks
+    // entries, zeros included), so nothing left over from an earlier call is ever consumed and
+    // no clearing pass is needed.
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
+                                                                            c.n_chunks, ws, err_word);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    perm_scan_kernel<<<(D + kPermWarps - 1) / kPermWarps, kPermThreads, 0, s>>>(ws, D, c.n_chunks, dest_counts);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
+    if (smem > 48 * 1024)
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem)));
+    perm_rank_kernel<<<c.n_chunks, kPermThreads, smem, s>>>(assigned_slot, P, D, c.chunk, c.n_chunks, ws,
+                                                            dest_counts, dest_offsets, row_of_pair, pair_of_row);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
 int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
                         void* send, uint32_t flags, cobalt_stream_t stream)
 {

@@ -131,6 +131,7 @@ const char* cobalt_status_string(int status)
         case COBALT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case COBALT_ERR_UNSUPPORTED: return "outside the supported size envelope";
         case COBALT_ERR_CUDA: return "CUDA runtime error";
+        case COBALT_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
