@@ -191,6 +191,24 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------------------------
+# aggregation over ranks (every rank routes its own replica; nothing crosses GPUs on the data path)
+# ---------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, device) -> float:
+    """Slowest rank's time: all-reduce(MAX) when a process group is up, else the value itself."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, pairs_per_rank: int, ms_per_step: float) -> float:
+    """Pairs routed by all ranks per second of the slowest rank's step time (weak scaling)."""
+    return world * pairs_per_rank / (ms_per_step * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------
 def run_cobalt(args):
@@ -277,12 +295,8 @@ def run_cobalt(args):
     stage_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in ev) / args.steps for i, n in enumerate(names)}
     err_bits = cb.read_and_clear_device_error()
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if distributed:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
-    ms_per_step = total_ms_max / args.steps
-    value = world * w.P / (ms_per_step * 1e-3)
+    ms_per_step = max_over_ranks(total_ms, "cuda") / args.steps
+    value = whole_job_value(world, w.P, ms_per_step)
 
     # end to end from pinned host buffers: H2D of the inputs, four stages, D2H of the results
     e2e = None
@@ -302,11 +316,8 @@ def run_cobalt(args):
             step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
         e1.record()
         barrier()
-        t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if distributed:
-            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t2.item()) / n_e2e
-        e2e = {"value": world * w.P / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), "cuda") / n_e2e
+        e2e = {"value": whole_job_value(world, w.P, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": step.h2d_bytes(), "d2h_bytes_per_step": step.d2h_bytes(), "steps": n_e2e}
 
     if rank == 0:
