@@ -45,6 +45,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="5")
     ap.add_argument("--tokens", type=int, default=None, help="override T (reduced-size runs for profiling)")
+    ap.add_argument("--hidden", type=int, default=None, help="override H (tiny rows isolate the index stages)")
     ap.add_argument("--impl", default="cobalt", choices=["cobalt", "reference"])
     ap.add_argument("--cpu-sample-tokens", type=int, default=None,
                     help="tokens of the workload the CPU oracle is timed on (default 32768; 8192 for --impl reference)")
@@ -236,6 +237,8 @@ def run_cobalt(args):
         torch.cuda.synchronize()
 
     w = W.make_config(args.config, T=args.tokens)
+    if args.hidden is not None:
+        w.H = args.hidden
     layout = cb.Layout(w.N, w.Q, w.S, w.E, w.slot_expert.tolist(), w.primary_slot.tolist())
     step = RouteStep(layout, w.T, w.K, w.H)
 

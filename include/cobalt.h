@@ -70,7 +70,8 @@ extern "C" {
 #define COBALT_ASSIGN_NAIVE 0x1u             /* primary-replica rule instead of Algorithm 1 */
 #define COBALT_IMPL_MASK 0xF00u              /* kernel variant override, 0 = library default */
 #define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
-#define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies through shared memory */
+#define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies, one work item per CTA (default) */
+#define COBALT_IMPL_BULK_RING 0x300u         /* same copies from a persistent CTA with a shared-memory ring */
 
 typedef struct cobalt_layout cobalt_layout_t;   /* opaque, owned by the library */
 typedef void* cobalt_stream_t;                  /* a cudaStream_t */
@@ -147,6 +148,13 @@ int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int
                          cobalt_stream_t stream);
 int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K,
                         int32_t H, void* send, uint32_t flags, cobalt_stream_t stream);
+/* Token-block form: moves only T tokens whose rows x, and whose T*K entries of row_of_pair, the
+ * caller passes already offset to the block; the row indices still address the whole send
+ * buffer of total_rows rows.  cobalt_permute_rows is the block form with total_rows = T*K.
+ * Lets a caller stream a step in token blocks (e.g. while the hidden rows are still arriving). */
+int cobalt_permute_rows_block(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K,
+                              int32_t H, void* send, int64_t total_rows, uint32_t flags,
+                              cobalt_stream_t stream);
 int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
                    const void* x, int32_t H, void* send, uint32_t* dest_counts,
                    uint32_t* dest_offsets, int32_t* row_of_pair, int32_t* pair_of_row,
@@ -184,6 +192,11 @@ int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t
 int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w,
                    int64_t T, int32_t K, int32_t H, void* y, uint32_t flags,
                    cobalt_stream_t stream);
+/* Token-block form: row_of_pair, gate_w and y are passed offset to a block of T tokens;
+ * expert_out is the whole buffer of total_rows rows.  cobalt_combine is total_rows = T*K. */
+int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, const float* gate_w,
+                         int64_t T, int32_t K, int32_t H, void* y, int64_t total_rows,
+                         uint32_t flags, cobalt_stream_t stream);
 
 /* ---- device error word -------------------------------------------------------------------
  * Waits for `stream`, copies the COBALT_DEVERR_* bits set by kernels on the current device

@@ -34,6 +34,7 @@ STATS_ACCUMULATE = 0x1
 ASSIGN_NAIVE = 0x1
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200
+IMPL_BULK_RING = 0x300
 
 # every symbol include/cobalt.h declares
 EXPORTS = (
@@ -42,7 +43,7 @@ EXPORTS = (
     "cobalt_coact_stats_workspace_bytes", "cobalt_coact_stats",
     "cobalt_assign_workspace_bytes", "cobalt_assign",
     "cobalt_permute_workspace_bytes", "cobalt_permute_index", "cobalt_permute_rows", "cobalt_permute",
-    "cobalt_permute_index_static",
+    "cobalt_permute_index_static", "cobalt_permute_rows_block", "cobalt_combine_block",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -78,6 +79,8 @@ def _load() -> C.CDLL:
         "cobalt_permute_rows": (C.c_int, [vp, vp, i64, i32, i32, vp, u32, vp]),
         "cobalt_permute": (C.c_int, [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, vp, u32, vp, sz, vp]),
         "cobalt_combine": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, u32, vp]),
+        "cobalt_permute_rows_block": (C.c_int, [vp, vp, i64, i32, i32, vp, i64, u32, vp]),
+        "cobalt_combine_block": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_read_and_clear_device_error": (C.c_int, [C.POINTER(u32), vp]),
     }
     for name, (res, args) in sig.items():
@@ -303,6 +306,36 @@ def combine(expert_out: torch.Tensor, row_of_pair: torch.Tensor, gate_w: torch.T
                                _ptr(row_of_pair, torch.int32, "row_of_pair"),
                                _ptr(gate_w, torch.float32, "gate_w"), T, K, H, _ptr(y, torch.bfloat16, "y"),
                                flags, _stream()), "cobalt_combine")
+
+
+def _elem_ptr(t: torch.Tensor, offset_elems: int) -> int:
+    return t.data_ptr() + offset_elems * t.element_size()
+
+
+def permute_rows_block(x: torch.Tensor, row_of_pair_block: torch.Tensor, K: int, send: torch.Tensor, t0: int,
+                       t1: int, *, flags: int = 0) -> None:
+    """cobalt_permute_rows on tokens t0:t1 only (x and send are the whole buffers; row_of_pair_block
+    holds the rows of pairs t0*K : t1*K, which index the whole send buffer)."""
+    T, H = x.shape
+    if not (0 <= t0 <= t1 <= T) or row_of_pair_block.numel() != (t1 - t0) * K or send.numel() != T * K * H:
+        raise CobaltError(ERR_INVALID_ARG, "permute_rows_block (sizes)")
+    _ptr(x, torch.bfloat16, "x"), _ptr(send, torch.bfloat16, "send")
+    _check(_lib.cobalt_permute_rows_block(_elem_ptr(x, t0 * H), _ptr(row_of_pair_block, torch.int32, "row_of_pair"),
+                                          t1 - t0, K, H, send.data_ptr(), T * K, flags, _stream()),
+           "cobalt_permute_rows_block")
+
+
+def combine_block(expert_out: torch.Tensor, row_of_pair_block: torch.Tensor, gate_w: torch.Tensor,
+                  y: torch.Tensor, t0: int, t1: int, *, flags: int = 0) -> None:
+    """cobalt_combine on tokens t0:t1 only (expert_out is the whole [P, H] buffer)."""
+    T, K = gate_w.shape
+    H = y.shape[1]
+    if not (0 <= t0 <= t1 <= T) or row_of_pair_block.numel() != (t1 - t0) * K or expert_out.numel() != T * K * H:
+        raise CobaltError(ERR_INVALID_ARG, "combine_block (sizes)")
+    _ptr(expert_out, torch.bfloat16, "expert_out"), _ptr(gate_w, torch.float32, "gate_w"), _ptr(y, torch.bfloat16, "y")
+    _check(_lib.cobalt_combine_block(expert_out.data_ptr(), _ptr(row_of_pair_block, torch.int32, "row_of_pair"),
+                                     _elem_ptr(gate_w, t0 * K), t1 - t0, K, H, _elem_ptr(y, t0 * H), T * K, flags,
+                                     _stream()), "cobalt_combine_block")
 
 
 def read_and_clear_device_error() -> int:

@@ -38,7 +38,6 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
     const uint32_t* rlist = tab + lv.rlist_off();
     const uint32_t* nodes = tab + lv.nodes_off();
     const int N = lv.N;
-    const int slots_per_node = lv.S * lv.Q;
 
     const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     uint32_t cost = 0, naive_cost = 0;
@@ -92,44 +91,51 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
             uint32_t naive_nodes = 0;
 #pragma unroll
             for (int a = 0; a < KMAX; ++a)
-                if (a < K) naive_nodes |= 1u << (primary[id[a]] / slots_per_node);
+                if (a < K) naive_nodes |= 1u << (primary[id[a]] >> 24);
             naive_cost = __popc(naive_nodes & ~src_bit);
 
             if (naive) {
 #pragma unroll
                 for (int a = 0; a < KMAX; ++a)
-                    if (a < K) out[a] = static_cast<int32_t>(primary[id[a]]);
+                    if (a < K) out[a] = static_cast<int32_t>(primary[id[a]] & 0xFFFFFFu);
                 cost = naive_cost;
             } else {
                 // line 3-4: U_t and the remote masks; bit j <-> j-th node after skipping n_s.
                 // m[a] == 0 marks an expert that is present on the source node.
                 uint32_t m[KMAX];
-                uint32_t any_remote = 0;
+                uint32_t any_remote = 0, common = 0xFFFFFFFFu;
 #pragma unroll
                 for (int a = 0; a < KMAX; ++a) {
                     if (a < K) {
                         const uint32_t held = nodes[id[a]];
                         m[a] = (held & src_bit) ? 0u : (((held >> (n_s + 1)) << n_s) | (held & low));
                         any_remote |= m[a];
+                        if (m[a]) common &= m[a];
                     }
                 }
-                // lines 5-8: ascending b, strictly smaller popcount replaces b*.
+                // lines 5-8: ascending b, strictly smaller popcount replaces b*.  A single node
+                // covers U_t iff every mask has its bit, and the lowest such bit is the smallest
+                // one-bit b; only otherwise are the masks with two or more bits enumerated.
                 uint32_t b_star = 0;
                 if (any_remote) {
-                    const uint32_t full = (1u << (N - 1)) - 1u;
-                    b_star = full;
-                    int best = N - 1;
-                    for (uint32_t b = 1; b < full; ++b) {
-                        const int pc = __popc(b);
-                        if (pc >= best) continue;
-                        bool feasible = true;
+                    if (common) {
+                        b_star = common & (0u - common);
+                    } else {
+                        const uint32_t full = (1u << (N - 1)) - 1u;
+                        b_star = full;
+                        int best = N - 1;
+                        for (uint32_t b = 3; b < full; ++b) {
+                            const int pc = __popc(b);
+                            if (pc >= best) continue;
+                            bool feasible = true;
 #pragma unroll
-                        for (int a = 0; a < KMAX; ++a)
-                            if (a < K) feasible = feasible && (m[a] == 0 || (b & m[a]) != 0);
-                        if (feasible) {
-                            b_star = b;
-                            best = pc;
-                            if (pc == 1) break;  // nothing smaller can cover a non-empty U_t
+                            for (int a = 0; a < KMAX; ++a)
+                                if (a < K) feasible = feasible && (m[a] == 0 || (b & m[a]) != 0);
+                            if (feasible) {
+                                b_star = b;
+                                best = pc;
+                                if (pc == 2) break;  // one node is known not to suffice
+                            }
                         }
                     }
                     cost = __popc(b_star);
@@ -140,15 +146,22 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
                     if (a < K) {
                         int node = n_s;
                         if (m[a] != 0) {
-                            const uint32_t c = b_star & m[a];
-                            const uint32_t i = hash_index(
-                                route_hash(seed_lo, seed_hi, static_cast<uint32_t>(t), id[a], 0u), __popc(c));
-                            const int bit = __fns(c, 0, static_cast<int>(i) + 1);
+                            // RandomNode: the i-th set bit of b* & m; a single candidate needs no draw
+                            uint32_t c = b_star & m[a];
+                            const uint32_t n_c = __popc(c);
+                            if (n_c > 1) {
+                                const uint32_t i = hash_index(
+                                    route_hash(seed_lo, seed_hi, static_cast<uint32_t>(t), id[a], 0u), n_c);
+                                for (uint32_t j = 0; j < i; ++j) c &= c - 1u;   // drop the i lowest set bits
+                            }
+                            const int bit = __ffs(c) - 1;
                             node = bit + (bit >= n_s ? 1 : 0);
                         }
+                        // UniformChoice over R_{e,node}; floor(x * 1 / 2^32) = 0, so one replica needs no draw
                         const uint32_t e_n = ent[id[a] * N + node];
-                        const uint32_t i = hash_index(
-                            route_hash(seed_lo, seed_hi, static_cast<uint32_t>(t), id[a], 1u), e_n & 0xFFu);
+                        const uint32_t n_r = e_n & 0xFFu;
+                        const uint32_t i = (n_r > 1) ? hash_index(
+                            route_hash(seed_lo, seed_hi, static_cast<uint32_t>(t), id[a], 1u), n_r) : 0u;
                         out[a] = static_cast<int32_t>(rlist[(e_n >> 8) + i]);
                     }
                 }

@@ -10,6 +10,11 @@
 // Experts counts whose triangle does not fit in shared memory take a direct global-atomic path.
 #include <cooperative_groups.h>
 
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <utility>
+
 #include "common.cuh"
 
 namespace cg = cooperative_groups;
@@ -59,18 +64,28 @@ __device__ __forceinline__ bool load_token_ids(const int32_t* __restrict__ ids, 
     return bad == 0;
 }
 
+// Row of the lower triangle that holds flat index idx (row hi starts at hi*(hi+1)/2).
+__device__ __forceinline__ int tri_row(int idx)
+{
+    int hi = static_cast<int>((sqrtf(8.0f * static_cast<float>(idx) + 1.0f) - 1.0f) * 0.5f);
+    while (hi * (hi + 1) / 2 > idx) --hi;
+    while ((hi + 1) * (hi + 2) / 2 <= idx) ++hi;
+    return hi;
+}
+
 template <int KT>
 __global__ void __launch_bounds__(kStatsThreads)
 coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E,
                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
 {
-    extern __shared__ __align__(16) uint32_t tri[];
+    extern __shared__ __align__(16) uint32_t tri[];   // lower triangle, padded to whole uint4
     constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
     const int K = (KT > 0) ? KT : K_rt;
     cg::cluster_group cluster = cg::this_cluster();
 
     const int n_tri = static_cast<int>(tri_entries(E));
-    for (int i = threadIdx.x; i < n_tri; i += blockDim.x) tri[i] = 0;
+    const int n_vec = (n_tri + 3) / 4;
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -90,24 +105,29 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     }
 
     cluster.sync();  // every tile of the cluster is complete
-    const unsigned csize = cluster.num_blocks();
-    const unsigned crank = cluster.block_rank();
-    const uint32_t* peer[8];
+    // Each CTA owns a contiguous slice of the flat triangle and sums it over all tiles of the
+    // cluster with 16-byte distributed-shared-memory loads (all threads busy, loads independent).
+    const int csize = static_cast<int>(cluster.num_blocks());
+    const int crank = static_cast<int>(cluster.block_rank());
+    const int per = (n_vec + csize - 1) / csize;
+    const int v0 = crank * per, v1 = min(n_vec, v0 + per);
+    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+        uint4 s = make_uint4(0, 0, 0, 0);
+        for (int r = 0; r < csize; ++r) {
+            const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
+            s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+        }
+        const uint32_t part[4] = {s.x, s.y, s.z, s.w};
+        int hi = tri_row(4 * v);
+        int lo = 4 * v - hi * (hi + 1) / 2;
 #pragma unroll
-    for (unsigned r = 0; r < 8; ++r) peer[r] = cluster.map_shared_rank(tri, r < csize ? r : 0);
-
-    for (int hi = static_cast<int>(crank); hi < E; hi += static_cast<int>(csize)) {
-        const int base = hi * (hi + 1) / 2;
-        for (int lo = threadIdx.x; lo <= hi; lo += blockDim.x) {
-            uint32_t sum = 0;
-#pragma unroll
-            for (unsigned r = 0; r < 8; ++r)
-                if (r < csize) sum += peer[r][base + lo];
-            if (sum) {
-                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], sum);
-                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], sum);
-                else atomicAdd(&load[hi], sum);
+        for (int c = 0; c < 4; ++c) {
+            if (4 * v + c < n_tri && part[c]) {
+                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], part[c]);
+                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], part[c]);
+                else atomicAdd(&load[hi], part[c]);
             }
+            if (++lo > hi) { ++hi; lo = 0; }
         }
     }
     cluster.sync();  // no CTA may exit while a peer still reads its tile
@@ -134,14 +154,15 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
                        uint32_t* err_word, int n_sm, cudaStream_t stream)
 {
     auto kernel = coact_tile_kernel<KT>;
-    const size_t smem = tri_entries(E) * sizeof(uint32_t);
+    const size_t smem = round_up(tri_entries(E) * sizeof(uint32_t), 16);
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
 
-    // one CTA per ~2 tokens per thread, at most one per SM, in clusters of up to 8
+    // about two tokens per thread, never more CTAs than can be co-resident (a second wave of
+    // clusters would double the run time), clusters as large as the device schedules well
     int64_t want = (T + 2 * kStatsThreads - 1) / (2 * kStatsThreads);
-    int n_cta = static_cast<int>(want < 1 ? 1 : (want > n_sm ? n_sm : want));
-    int csize = 8;
-    while (csize > n_cta) csize >>= 1;
+    if (want < 1) want = 1;
+    if (want > n_sm) want = n_sm;
 
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -151,17 +172,59 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    for (; csize >= 1; csize >>= 1) {
-        attr[0].val.clusterDim.x = csize;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.gridDim = dim3(static_cast<unsigned>(n_cta / csize * csize));
-        int max_clusters = 0;
-        cudaError_t q = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
-        if (q == cudaSuccess && max_clusters >= 1) break;
-        (void)cudaGetLastError();
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+
+    // candidates: cluster sizes 16 (non-portable), 8, 4, 2, 1 -> CTAs that can be co-resident
+    static std::mutex cache_lock;
+    static std::map<std::tuple<int, int, int, int>, std::pair<int, int>> cache;   // (dev, E, want, KT)
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    const auto key = std::make_tuple(dev, E, static_cast<int>(want), KT);
+    int best_cs = 0, best_cta = 0;
+    {
+        std::lock_guard<std::mutex> guard(cache_lock);
+        auto it = cache.find(key);
+        if (it != cache.end()) {
+            best_cs = it->second.first;
+            best_cta = it->second.second;
+        }
     }
-    if (csize < 1) return COBALT_ERR_UNSUPPORTED;
+    if (best_cs == 0) {
+        int cand_cs[5], cand_cta[5], n_cand = 0, most = 0;
+        for (int cs = 16; cs >= 1; cs >>= 1) {
+            if (cs > want) continue;
+            attr[0].val.clusterDim.x = cs;
+            cfg.gridDim = dim3(cs);
+            int max_clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess) {
+                (void)cudaGetLastError();
+                continue;
+            }
+            int n_cta = static_cast<int>(want) / cs * cs;
+            if (n_cta > max_clusters * cs) n_cta = max_clusters * cs;
+            if (n_cta < cs) continue;
+            cand_cs[n_cand] = cs;
+            cand_cta[n_cand] = n_cta;
+            ++n_cand;
+            if (n_cta > most) most = n_cta;
+        }
+        // the largest cluster that keeps at least 90% of the best CTA count (fewer global merges)
+        for (int i = 0; i < n_cand; ++i) {
+            if (cand_cta[i] * 10 >= most * 9) {
+                best_cs = cand_cs[i];
+                best_cta = cand_cta[i];
+                break;
+            }
+        }
+        if (best_cs != 0) {
+            std::lock_guard<std::mutex> guard(cache_lock);
+            cache[key] = std::make_pair(best_cs, best_cta);
+        }
+    }
+    if (best_cs == 0) return COBALT_ERR_UNSUPPORTED;
+    attr[0].val.clusterDim.x = best_cs;
+    cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, coact, load, err_word));
     return COBALT_OK;
 }

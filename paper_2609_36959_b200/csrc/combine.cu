@@ -78,11 +78,13 @@ using namespace cobalt;
 
 extern "C" {
 
-int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
-                   int32_t K, int32_t H, void* y, uint32_t flags, cobalt_stream_t stream)
+int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
+                         int32_t K, int32_t H, void* y, int64_t total_rows, uint32_t flags,
+                         cobalt_stream_t stream)
 {
-    if (T < 0 || K < 1 || H < 1) return COBALT_ERR_INVALID_ARG;
-    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31))
+    if (T < 0 || K < 1 || H < 1 || total_rows < 0) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31) ||
+        total_rows >= (1ll << 31))
         return COBALT_ERR_UNSUPPORTED;
     if (T == 0) return COBALT_OK;
     if (!expert_out || !row_of_pair || !gate_w || !y) return COBALT_ERR_INVALID_ARG;
@@ -100,8 +102,11 @@ int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const flo
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int n_vec = H / 8;
-    const int64_t P = T * K;
-    const unsigned grid = static_cast<unsigned>(T < 16ll * n_sm ? T : 16ll * n_sm);
+    const int64_t P = total_rows;      // bound on the row indices (rows of the whole expert_out buffer)
+    // one CTA per token: the block scheduler overlaps the per-token index loads of one CTA with
+    // the row streaming of the others (measured faster than a persistent grid-stride grid)
+    const int64_t max_grid = g_tune.combine_per_sm > 0 ? static_cast<int64_t>(g_tune.combine_per_sm) * n_sm : 0x7FFFFFFFll;
+    const unsigned grid = static_cast<unsigned>(T < max_grid ? T : max_grid);
     const uint4* src = static_cast<const uint4*>(expert_out);
     uint4* dst = static_cast<uint4*>(y);
 #define COBALT_COMBINE_CASE(KT)                                                                         \
@@ -120,6 +125,14 @@ int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const flo
 #undef COBALT_COMBINE_CASE
     COBALT_CUDA_TRY(cudaGetLastError());
     return COBALT_OK;
+}
+
+int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
+                   int32_t K, int32_t H, void* y, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1) return COBALT_ERR_INVALID_ARG;
+    return cobalt_combine_block(expert_out, row_of_pair, gate_w, T, K, H, y, T * static_cast<int64_t>(K), flags,
+                                stream);
 }
 
 }  // extern "C"

@@ -25,6 +25,19 @@ int device_error_word(uint32_t** out);
 // Number of SMs of the current device (cached per device).
 int sm_count(int* out);
 
+// Unsupported tuning knobs for parameter sweeps (set through cobalt_internal_tune; the defaults
+// are what the library ships with).
+struct Tuning {
+    int rows_item_bytes = 32768;    // default row mover: largest work item (whole rows of consecutive tokens)
+    int rows_stages = 6;            // ring variant: ring slots (3, 4, 6, 8 or 12)
+    int rows_stage_bytes = 18432;   // ring variant: largest ring slot
+    int rows_per_sm = 0;            // cap on CTAs per SM (0 = as many as shared memory allows)
+    int rows_vec_per_sm = 0;        // vector row mover: CTAs per SM (0 = one CTA per token)
+    int rows_hint = 0;              // 1 = evict-first L2 hints on the bulk copies
+    int combine_per_sm = 0;         // CTAs per SM of the combine kernel's grid (0 = one CTA per token)
+};
+extern Tuning g_tune;
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -32,7 +45,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // Device tables built from a layout (Section 3.3: R_{e,n} and N_e), one contiguous blob of
 // 32-bit words that kernels copy into shared memory:
 //   ent[e*N + n]   = (offset into rlist << 8) | |R_{e,n}|
-//   primary[e]     = slot of e's primary replica
+//   primary[e]     = slot of e's primary replica | (its node << 24)
 //   rlist[...]     = slots of R_{e,n}, ascending, all (e, n) groups back to back
 //   nodes[e]       = bitmask over nodes holding e (one word each)
 struct LayoutView {

@@ -8,10 +8,12 @@
 //       of every pair inside its chunk: each warp owns a contiguous sub-range, counts it,
 //       the CTA scans the per-warp counts in warp order, and each warp walks its sub-range
 //       again, ranking equal destinations inside a 32-pair step by lane order
-//       (__match_any_sync + popcount of lower lanes).
-// Row part: K4 moves each token's row to its K rows of the send buffer.  Two variants: plain
-// 16-byte streaming loads/stores, and a bulk-async-copy pipeline (global -> shared ring ->
-// K global rows) driven by one warp per CTA.
+//       (per-bit ballots + popcount of lower lanes).
+// Row part: K4 moves each token's row to its K rows of the send buffer.  Three variants:
+// (default) one work item per single-warp CTA: a bulk async copy global -> shared, then one
+// bulk async copy shared -> global per destination row, many small CTAs in flight per SM;
+// a persistent variant of the same with a shared-memory ring; and plain 16-byte streaming
+// loads/stores.
 #include "common.cuh"
 
 namespace cobalt {
@@ -20,6 +22,7 @@ constexpr int kPermThreads = 256;
 constexpr int kPermWarps = kPermThreads / 32;
 constexpr int kMinChunk = 2048;      // pairs per chunk (multiple of kPermThreads)
 constexpr int kMaxChunks = 2048;
+constexpr int kRankSteps = kMinChunk / kPermWarps / 32;   // 32-pair steps of a warp per super-step
 
 struct ChunkPlan {
     int64_t P;
@@ -70,22 +73,44 @@ perm_scan_kernel(uint32_t* __restrict__ ws, int D, int n_chunks, uint32_t* __res
     if (d >= D) return;
     uint32_t* row = ws + static_cast<size_t>(d) * n_chunks;
     uint32_t running = 0;
-    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-        const int c = c0 + lane;
-        const uint32_t v = (c < n_chunks) ? row[c] : 0u;
-        uint32_t incl = v;
+    constexpr int kBatch = 8;   // 8 x 32 chunks loaded back to back before the dependent scans
+    for (int c0 = 0; c0 < n_chunks; c0 += 32 * kBatch) {
+        uint32_t v[kBatch];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-            if (lane >= off) incl += up;
+        for (int b = 0; b < kBatch; ++b) {
+            const int c = c0 + b * 32 + lane;
+            v[b] = (c < n_chunks) ? row[c] : 0u;
         }
-        if (c < n_chunks) row[c] = running + incl - v;
-        running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            const int c = c0 + b * 32 + lane;
+            uint32_t incl = v[b];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            if (c < n_chunks) row[c] = running + incl - v[b];
+            running += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        }
     }
     if (lane == 0) dest_counts[d] = running;
 }
 
 // ---- K3 -----------------------------------------------------------------------------------
+// Lanes of the warp holding the same key, built from one ballot per key bit (the hardware
+// match instruction is far slower than a dozen votes for keys this narrow).
+__device__ __forceinline__ uint32_t peers_of(uint32_t key, int key_bits)
+{
+    uint32_t peers = 0xFFFFFFFFu;
+    for (int b = 0; b < key_bits; ++b) {
+        const uint32_t bit = (key >> b) & 1u;
+        const uint32_t vote = __ballot_sync(0xFFFFFFFFu, bit);
+        peers &= bit ? vote : ~vote;
+    }
+    return peers;
+}
+
 __global__ void __launch_bounds__(kPermThreads)
 perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
                  const uint32_t* __restrict__ ws, const uint32_t* __restrict__ dest_counts,
@@ -129,15 +154,30 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     const int64_t w1 = min(P, w0 + sub);
     uint32_t* mine = wcnt + warp * D;
 
+    // The warp's sub-range is walked in super-steps of kRankSteps x 32 pairs whose slots are
+    // loaded back to back into registers (one exposed memory latency per super-step, not per step).
+    const int n_super = (sub + 32 * kRankSteps - 1) / (32 * kRankSteps);
+    const int key_bits = 32 - __clz(D);      // keys 0..D (D marks "no destination")
+    int32_t dreg[kRankSteps];
+    auto load_super = [&](int ss) {
+#pragma unroll
+        for (int s = 0; s < kRankSteps; ++s) {
+            const int64_t p = w0 + static_cast<int64_t>(ss) * 32 * kRankSteps + s * 32 + lane;
+            int32_t d = (p < w1) ? __ldg(slot + p) : -1;
+            dreg[s] = (d >= D) ? -1 : d;
+        }
+    };
+
     // pass A: count this warp's sub-range per destination (warp-private, no atomics)
-    for (int64_t q = w0; q < w1; q += 32) {
-        const int64_t p = q + lane;
-        int32_t d = (p < w1) ? __ldg(slot + p) : -1;
-        if (d >= D) d = -1;
-        const uint32_t key = static_cast<uint32_t>(d);
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, key);
-        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
-        __syncwarp();
+    for (int ss = 0; ss < n_super; ++ss) {
+        load_super(ss);
+#pragma unroll
+        for (int s = 0; s < kRankSteps; ++s) {
+            const int32_t d = dreg[s];
+            const uint32_t peers = peers_of(static_cast<uint32_t>(d < 0 ? D : d), key_bits);
+            if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
+            __syncwarp();
+        }
     }
     __syncthreads();
     // pass B: per destination, turn the per-warp counts into starting rows (warp order)
@@ -152,23 +192,24 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     }
     __syncthreads();
     // pass C: stable rank inside the warp's sub-range
-    for (int64_t q = w0; q < w1; q += 32) {
-        const int64_t p = q + lane;
-        int32_t d = (p < w1) ? __ldg(slot + p) : -1;
-        const bool in_range = (p < w1);
-        if (d >= D) d = -1;
-        const uint32_t key = static_cast<uint32_t>(d);
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, key);
-        if (d >= 0) {
-            const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
-            row_of_pair[p] = static_cast<int32_t>(row);
-            if (pair_of_row) pair_of_row[row] = static_cast<int32_t>(p);
-        } else if (in_range) {
-            row_of_pair[p] = -1;
+    for (int ss = 0; ss < n_super; ++ss) {
+        if (n_super > 1) load_super(ss);     // a single super-step still holds its slots in registers
+#pragma unroll
+        for (int s = 0; s < kRankSteps; ++s) {
+            const int64_t p = w0 + static_cast<int64_t>(ss) * 32 * kRankSteps + s * 32 + lane;
+            const int32_t d = dreg[s];
+            const uint32_t peers = peers_of(static_cast<uint32_t>(d < 0 ? D : d), key_bits);
+            if (d >= 0) {
+                const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
+                row_of_pair[p] = static_cast<int32_t>(row);
+                if (pair_of_row) pair_of_row[row] = static_cast<int32_t>(p);
+            } else if (p < w1) {
+                row_of_pair[p] = -1;
+            }
+            __syncwarp();
+            if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);
+            __syncwarp();
         }
-        __syncwarp();
-        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);
-        __syncwarp();
     }
 }
 
@@ -203,9 +244,6 @@ perm_rows_vector_kernel(const uint4* __restrict__ x, const int32_t* __restrict__
 }
 
 // ---- K4, bulk-async-copy variant ----------------------------------------------------------
-constexpr int kBulkStages = 6;
-constexpr int kBulkLag = 3;                      // stages of loads in flight ahead of the stores
-constexpr int kBulkMaxStageBytes = 18432;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p)
@@ -257,6 +295,30 @@ __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uin
                  : "memory");
 }
 
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar,
+                                               uint64_t pol)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+            smem_addr(smem_dst)),
+        "l"(gsrc), "r"(bytes), "r"(smem_addr(bar)), "l"(pol)
+        : "memory");
+}
+
+__device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src, uint32_t bytes, uint64_t pol)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
+                 "r"(smem_addr(smem_src)), "r"(bytes), "l"(pol)
+                 : "memory");
+}
+
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 
 template <int N>
@@ -267,8 +329,10 @@ __device__ __forceinline__ void bulk_wait_read()
 
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// One warp per CTA.  Work item i: `rows_per_item` whole rows of consecutive tokens (n_seg == 1),
+// One warp per CTA; kStages ring slots, loads run kLag items ahead of the stores; kHint marks both
+// directions evict-first in L2 (every byte is touched exactly once).  Work item i: `rows_per_item` whole rows of consecutive tokens (n_seg == 1),
 // or one column segment of one token's row (n_seg > 1, rows_per_item == 1).
+template <int kStages, int kLag, bool kHint>
 __global__ void __launch_bounds__(32)
 perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_pair, int64_t T,
                       int K, int64_t P, uint32_t row_bytes, int rows_per_item, int n_seg,
@@ -276,13 +340,15 @@ perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__
                       uint8_t* __restrict__ send, uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(128) uint8_t ring[];
-    __shared__ __align__(8) uint64_t full[kBulkStages];
-    __shared__ int32_t rows_sm[kBulkStages][32];
+    __shared__ __align__(8) uint64_t full[kStages];
+    __shared__ int32_t rows_sm[kStages][32];
 
     const int lane = threadIdx.x;
+    uint64_t pol = 0;
+    if (kHint) pol = policy_evict_first();
     if (lane == 0) {
 #pragma unroll
-        for (int s = 0; s < kBulkStages; ++s) mbar_init(&full[s], 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -314,11 +380,11 @@ perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__
 
     bool ok = true;
     int32_t pref = (n_mine > 0) ? lane_row(first) : -1;
-    for (int64_t j = 0; j < n_mine + kBulkLag && ok; ++j) {
+    for (int64_t j = 0; j < n_mine + kLag && ok; ++j) {
         if (j < n_mine) {
-            // produce item j: its stage was last used by item j - kBulkStages
-            const int s = static_cast<int>(j % kBulkStages);
-            bulk_wait_read<kBulkStages - kBulkLag - 1>();
+            // produce item j: its stage was last used by item j - kStages
+            const int s = static_cast<int>(j % kStages);
+            bulk_wait_read<kStages - kLag - 1>();
             rows_sm[s][lane] = pref;
             if (j + 1 < n_mine) pref = lane_row(first + (j + 1) * step);
             __syncwarp();
@@ -327,15 +393,19 @@ perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__
                 item_tokens(first + j * step, t0, n_rows, col, bytes);
                 const uint32_t total = (n_seg == 1) ? static_cast<uint32_t>(n_rows) * row_bytes : bytes;
                 mbar_expect_tx(&full[s], total);
-                bulk_load(ring + static_cast<size_t>(s) * stage_bytes,
-                          x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s]);
+                if (kHint)
+                    bulk_load_hint(ring + static_cast<size_t>(s) * stage_bytes,
+                                   x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s], pol);
+                else
+                    bulk_load(ring + static_cast<size_t>(s) * stage_bytes,
+                              x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s]);
             }
         }
-        if (j >= kBulkLag) {
+        if (j >= kLag) {
             // consume item c: wait for its rows, then fan each row out to its K destinations
-            const int64_t c = j - kBulkLag;
-            const int s = static_cast<int>(c % kBulkStages);
-            ok = mbar_wait(&full[s], static_cast<uint32_t>((c / kBulkStages) & 1));
+            const int64_t c = j - kLag;
+            const int s = static_cast<int>(c % kStages);
+            ok = mbar_wait(&full[s], static_cast<uint32_t>((c / kStages) & 1));
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (ok) {
                 int64_t t0; int n_rows; uint32_t col, bytes;
@@ -343,9 +413,10 @@ perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__
                 const int32_t row = rows_sm[s][lane];
                 if (row >= 0 && row < P) {
                     const int r = lane / K;
-                    bulk_store(send + static_cast<size_t>(row) * row_bytes + col,
-                               ring + static_cast<size_t>(s) * stage_bytes + static_cast<size_t>(r) * row_bytes,
-                               bytes);
+                    void* dst = send + static_cast<size_t>(row) * row_bytes + col;
+                    const void* src = ring + static_cast<size_t>(s) * stage_bytes + static_cast<size_t>(r) * row_bytes;
+                    if (kHint) bulk_store_hint(dst, src, bytes, pol);
+                    else bulk_store(dst, src, bytes);
                 } else if (row >= P) {
                     flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
                 }
@@ -357,15 +428,69 @@ perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__
     if (!ok) {
         if (lane == 0) flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
         // give loads still in flight a bounded chance to land before the ring is released
-        for (int s = 0; s < kBulkStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             (void)mbar_wait(&full[s], 0);
             (void)mbar_wait(&full[s], 1);
         }
     }
 }
 
+// One work item per single-warp CTA, no ring: the block scheduler keeps many small CTAs in
+// flight per SM (shared memory for one item each) and hands out items in order.
+__global__ void __launch_bounds__(32)
+perm_rows_bulk_oneshot_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_pair, int64_t T,
+                              int K, int64_t P, uint32_t row_bytes, int rows_per_item, int n_seg,
+                              uint32_t seg_bytes, uint8_t* __restrict__ send, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(128) uint8_t buf[];
+    __shared__ __align__(8) uint64_t full;
+    const int lane = threadIdx.x;
+    const int64_t item = blockIdx.x;
+    int64_t t0;
+    int n_rows;
+    uint32_t col, bytes;
+    if (n_seg == 1) {
+        t0 = item * rows_per_item;
+        n_rows = (T - t0 < rows_per_item) ? static_cast<int>(T - t0) : rows_per_item;
+        col = 0;
+        bytes = row_bytes;
+    } else {
+        t0 = item / n_seg;
+        n_rows = 1;
+        col = static_cast<uint32_t>(item % n_seg) * seg_bytes;
+        bytes = min(seg_bytes, row_bytes - col);
+    }
+    const int32_t row = (lane < n_rows * K) ? __ldg(row_of_pair + t0 * K + lane) : -1;
+    if (lane == 0) {
+        mbar_init(&full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const uint32_t total = (n_seg == 1) ? static_cast<uint32_t>(n_rows) * row_bytes : bytes;
+        mbar_expect_tx(&full, total);
+        bulk_load(buf, x + static_cast<size_t>(t0) * row_bytes + col, total, &full);
+    }
+    __syncwarp();
+    bool ok = mbar_wait(&full, 0);
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    if (ok) {
+        if (row >= 0 && row < P)
+            bulk_store(send + static_cast<size_t>(row) * row_bytes + col, buf + static_cast<size_t>(lane / K) * row_bytes,
+                       bytes);
+        else if (row >= P)
+            flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+    }
+    bulk_commit();
+    bulk_wait_all();
+    if (!ok) {
+        if (lane == 0) flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
+        (void)mbar_wait(&full, 0);
+    }
+}
+
+// P bounds the row indices (rows of the whole send buffer), which may exceed T*K when the call
+// covers only a block of tokens.
 static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int K, int H, void* send,
-                       uint32_t flags, cudaStream_t stream)
+                       int64_t P, uint32_t flags, cudaStream_t stream)
 {
     uint32_t* err_word = nullptr;
     int rc = device_error_word(&err_word);
@@ -373,14 +498,14 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     int n_sm = 0;
     rc = sm_count(&n_sm);
     if (rc != COBALT_OK) return rc;
-    const int64_t P = T * K;
     const uint32_t row_bytes = static_cast<uint32_t>(H) * 2u;
     uint32_t impl = flags & COBALT_IMPL_MASK;
-    if (impl == 0) impl = COBALT_IMPL_BULK;
+    if (impl == 0) impl = COBALT_IMPL_BULK;   // measured fastest: 99% of the copy bandwidth at T=131072, K=8, H=7168
 
     if (impl == COBALT_IMPL_VECTOR) {
         const int n_vec = H / 8;
-        const unsigned grid = static_cast<unsigned>(T < 16ll * n_sm ? T : 16ll * n_sm);
+        const int64_t max_grid = g_tune.rows_vec_per_sm > 0 ? static_cast<int64_t>(g_tune.rows_vec_per_sm) * n_sm : 0x7FFFFFFFll;
+        const unsigned grid = static_cast<unsigned>(T < max_grid ? T : max_grid);
         const uint4* xs = static_cast<const uint4*>(x);
         uint4* out = static_cast<uint4*>(send);
 #define COBALT_ROWS_CASE(KT)                                                                              \
@@ -402,29 +527,64 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     }
 
     // bulk variant: pick the work-item shape
+    const Tuning& tune = g_tune;
+    const int max_stage = (impl == COBALT_IMPL_BULK) ? tune.rows_item_bytes : tune.rows_stage_bytes;
     int rows_per_item = 1, n_seg = 1;
     uint32_t seg_bytes = row_bytes;
-    if (row_bytes <= static_cast<uint32_t>(kBulkMaxStageBytes)) {
-        rows_per_item = kBulkMaxStageBytes / row_bytes;
+    if (row_bytes <= static_cast<uint32_t>(max_stage)) {
+        rows_per_item = max_stage / row_bytes;
         if (rows_per_item > 32 / K) rows_per_item = 32 / K;
         if (rows_per_item < 1) rows_per_item = 1;
     } else {
-        n_seg = (row_bytes + kBulkMaxStageBytes - 1) / kBulkMaxStageBytes;
+        n_seg = (row_bytes + max_stage - 1) / max_stage;
         seg_bytes = static_cast<uint32_t>(round_up((row_bytes + n_seg - 1) / n_seg, 16));
         n_seg = (row_bytes + seg_bytes - 1) / seg_bytes;
     }
     const uint32_t stage_bytes =
         static_cast<uint32_t>(round_up(n_seg == 1 ? static_cast<size_t>(rows_per_item) * row_bytes : seg_bytes, 128));
     const int64_t n_items = (n_seg == 1) ? (T + rows_per_item - 1) / rows_per_item : T * n_seg;
-    const size_t smem = static_cast<size_t>(kBulkStages) * stage_bytes;
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem)));
-    int per_sm = static_cast<int>((220 * 1024) / (smem + 1024));
+
+    if (n_items > 0x7FFFFFFFll) return COBALT_ERR_UNSUPPORTED;
+    if (impl == COBALT_IMPL_BULK) {
+        const size_t smem1 = stage_bytes;
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rows_bulk_oneshot_kernel,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem1)));
+        perm_rows_bulk_oneshot_kernel<<<static_cast<unsigned>(n_items), 32, smem1, stream>>>(
+            static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
+            static_cast<uint8_t*>(send), err_word);
+        COBALT_CUDA_TRY(cudaGetLastError());
+        return COBALT_OK;
+    }
+
+    using Kernel = void (*)(const uint8_t*, const int32_t*, int64_t, int, int64_t, uint32_t, int, int, uint32_t,
+                            uint32_t, int64_t, uint8_t*, uint32_t*);
+    Kernel kernel = nullptr;
+    int stages = tune.rows_stages;
+    const bool hint = tune.rows_hint != 0;
+#define COBALT_BULK_CASE(NS, LAG)                                                                      \
+    case NS:                                                                                           \
+        kernel = hint ? perm_rows_bulk_kernel<NS, LAG, true> : perm_rows_bulk_kernel<NS, LAG, false>;  \
+        break
+    switch (stages) {
+        COBALT_BULK_CASE(3, 1);
+        COBALT_BULK_CASE(4, 2);
+        COBALT_BULK_CASE(8, 4);
+        COBALT_BULK_CASE(12, 6);
+        default:
+            stages = 6;
+            kernel = hint ? perm_rows_bulk_kernel<6, 3, true> : perm_rows_bulk_kernel<6, 3, false>;
+    }
+#undef COBALT_BULK_CASE
+    const size_t smem = static_cast<size_t>(stages) * stage_bytes;
+    if (smem > 224 * 1024) return COBALT_ERR_UNSUPPORTED;
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    int per_sm = static_cast<int>((220 * 1024) / (smem + 2048));
     if (per_sm < 1) per_sm = 1;
     if (per_sm > 8) per_sm = 8;
+    if (tune.rows_per_sm > 0 && tune.rows_per_sm < per_sm) per_sm = tune.rows_per_sm;
     int64_t grid = static_cast<int64_t>(n_sm) * per_sm;
     if (grid > n_items) grid = n_items;
-    perm_rows_bulk_kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
+    kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
         static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
         stage_bytes, n_items, static_cast<uint8_t*>(send), err_word);
     COBALT_CUDA_TRY(cudaGetLastError());
@@ -562,18 +722,27 @@ int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t
     return COBALT_OK;
 }
 
-int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
-                        void* send, uint32_t flags, cobalt_stream_t stream)
+int cobalt_permute_rows_block(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
+                              void* send, int64_t total_rows, uint32_t flags, cobalt_stream_t stream)
 {
-    if (T < 0 || K < 1 || H < 1) return COBALT_ERR_INVALID_ARG;
-    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31))
+    if (T < 0 || K < 1 || H < 1 || total_rows < 0) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31) ||
+        total_rows >= (1ll << 31))
         return COBALT_ERR_UNSUPPORTED;
     if (T == 0) return COBALT_OK;
     if (!x || !row_of_pair || !send) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send) || !aligned16(row_of_pair)) return COBALT_ERR_INVALID_ARG;
     const uint32_t impl = flags & COBALT_IMPL_MASK;
-    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK) return COBALT_ERR_INVALID_ARG;
-    return launch_rows(x, row_of_pair, T, K, H, send, flags, static_cast<cudaStream_t>(stream));
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK && impl != COBALT_IMPL_BULK_RING)
+        return COBALT_ERR_INVALID_ARG;
+    return launch_rows(x, row_of_pair, T, K, H, send, total_rows, flags, static_cast<cudaStream_t>(stream));
+}
+
+int cobalt_permute_rows(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
+                        void* send, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1) return COBALT_ERR_INVALID_ARG;
+    return cobalt_permute_rows_block(x, row_of_pair, T, K, H, send, T * static_cast<int64_t>(K), flags, stream);
 }
 
 int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D, const void* x, int32_t H,
@@ -587,7 +756,8 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
     if (T > 0 && (!x || !send)) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send)) return COBALT_ERR_INVALID_ARG;
     const uint32_t impl = flags & COBALT_IMPL_MASK;
-    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK) return COBALT_ERR_INVALID_ARG;
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK && impl != COBALT_IMPL_BULK_RING)
+        return COBALT_ERR_INVALID_ARG;
     int rc = cobalt_permute_index(assigned_slot, T, K, D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
                                   workspace, workspace_bytes, stream);
     if (rc != COBALT_OK) return rc;

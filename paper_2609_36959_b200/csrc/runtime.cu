@@ -8,6 +8,8 @@
 
 namespace cobalt {
 
+Tuning g_tune;
+
 static thread_local int g_last_cuda_error = 0;
 
 int record_cuda_error(cudaError_t err)
@@ -114,6 +116,7 @@ static int build_tables(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
         ent[en] = (static_cast<uint32_t>(offset[en]) << 8) | static_cast<uint32_t>(count[en]);
     if (primary_in)
         for (int32_t e = 0; e < E; ++e) primary[e] = static_cast<uint32_t>(primary_in[e]);
+    for (int32_t e = 0; e < E; ++e) primary[e] |= (primary[e] / static_cast<uint32_t>(S * Q)) << 24;
     return COBALT_OK;
 }
 
@@ -137,6 +140,21 @@ const char* cobalt_status_string(int status)
 }
 
 int cobalt_version(void) { return COBALT_VERSION; }
+
+// Not part of the public header: sets one of the sweep knobs of cobalt::Tuning by name.
+int cobalt_internal_tune(const char* key, int value)
+{
+    if (!key) return COBALT_ERR_INVALID_ARG;
+    if (!strcmp(key, "rows_item_bytes")) g_tune.rows_item_bytes = value;
+    else if (!strcmp(key, "rows_stages")) g_tune.rows_stages = value;
+    else if (!strcmp(key, "rows_stage_bytes")) g_tune.rows_stage_bytes = value;
+    else if (!strcmp(key, "rows_per_sm")) g_tune.rows_per_sm = value;
+    else if (!strcmp(key, "rows_vec_per_sm")) g_tune.rows_vec_per_sm = value;
+    else if (!strcmp(key, "rows_hint")) g_tune.rows_hint = value;
+    else if (!strcmp(key, "combine_per_sm")) g_tune.combine_per_sm = value;
+    else return COBALT_ERR_INVALID_ARG;
+    return COBALT_OK;
+}
 
 int cobalt_last_cuda_error(void) { return g_last_cuda_error; }
 

@@ -76,17 +76,60 @@ class RouteStep:
     # -- the same step from pinned host memory ----------------------------------------------
     def route_host(self, seed: int, ids_h: torch.Tensor, w_h: torch.Tensor, src_h: torch.Tensor,
                    x_h: torch.Tensor, y_h: torch.Tensor, coact_h: torch.Tensor, load_h: torch.Tensor,
-                   slot_load_h: torch.Tensor, totals_h: torch.Tensor) -> None:
+                   slot_load_h: torch.Tensor, totals_h: torch.Tensor, chunks: int = 8) -> None:
+        """One step with inputs and results in pinned host memory.
+
+        The gating output is small and goes first, so statistics, assignment and the permutation
+        index run while the hidden rows are still on their way.  The rows then move in `chunks`
+        token blocks: block c is copied in on one stream, fanned out to its send rows and (there
+        being no expert computation between dispatch and combine here) combined on the compute
+        stream, and its result copied out on a third stream, so both copy directions and the
+        kernels overlap.  The C entry points take plain pointers, so a block is just an offset.
+        """
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_h2d"):
+            self._h2d, self._d2h = torch.cuda.Stream(), torch.cuda.Stream()
+        h2d, d2h = self._h2d, self._d2h
+        h2d.wait_stream(main)          # the previous step may still be reading x / writing y
+        d2h.wait_stream(main)
+        T, K = self.T, self.K
+        chunks = max(1, min(chunks, T)) if T > 0 else 1
+        # block starts on multiples of 4 tokens keep every offset pointer 16-byte aligned for any K
+        bounds = [min(T, ((T * c) // chunks + 3) // 4 * 4) for c in range(chunks)] + [T]
+        ready = []
+        with torch.cuda.stream(h2d):
+            for c in range(chunks):
+                t0, t1 = bounds[c], bounds[c + 1]
+                self.x[t0:t1].copy_(x_h[t0:t1], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(h2d)
+                ready.append(ev)
         self.topk_ids.copy_(ids_h, non_blocking=True)
         self.gate_w.copy_(w_h, non_blocking=True)
         self.src_rank.copy_(src_h, non_blocking=True)
-        self.x.copy_(x_h, non_blocking=True)
-        self.route(seed)
-        y_h.copy_(self.y, non_blocking=True)
+        self.stats()
+        self.assign(seed)
+        cb.permute_index(self.assigned_slot, self.D, self.dest_counts, self.dest_offsets, self.row_of_pair,
+                         self.pair_of_row, self.workspace)
         coact_h.copy_(self.coact, non_blocking=True)
         load_h.copy_(self.load, non_blocking=True)
         slot_load_h.copy_(self.slot_load, non_blocking=True)
         totals_h.copy_(self.totals, non_blocking=True)
+        for c in range(chunks):
+            t0, t1 = bounds[c], bounds[c + 1]
+            if t1 == t0:
+                continue
+            main.wait_event(ready[c])
+            rop = self.row_of_pair[t0 * K:t1 * K]
+            # rows index the whole send buffer, so the full buffers are passed with a token offset
+            cb.permute_rows_block(self.x, rop, K, self.send, t0, t1)
+            cb.combine_block(self.expert_out, rop, self.gate_w, self.y, t0, t1)
+            done = torch.cuda.Event()
+            done.record(main)
+            with torch.cuda.stream(d2h):
+                d2h.wait_event(done)
+                y_h[t0:t1].copy_(self.y[t0:t1], non_blocking=True)
+        main.wait_stream(d2h)
 
     def h2d_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.topk_ids, self.gate_w, self.src_rank, self.x))

@@ -57,7 +57,7 @@ def test_config_full_elementwise(cb, name):
     r, p = check_index_stages(cb, w, step, w.seed)
 
     x = w.hidden_rows()
-    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR, 0):
+    for impl in (cb.IMPL_BULK, cb.IMPL_BULK_RING, cb.IMPL_VECTOR, 0):
         step.send.zero_()
         step.permute(flags=impl)
         torch.cuda.synchronize()
@@ -145,7 +145,7 @@ def test_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     layout, step = make_step(w, alias_expert_out=False)
     r, p = check_index_stages(cb, w, step, 4242)
     x = w.hidden_rows()
-    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR):
+    for impl in (cb.IMPL_BULK, cb.IMPL_BULK_RING, cb.IMPL_VECTOR):
         step.send.zero_()
         step.permute(flags=impl)
         torch.cuda.synchronize()
@@ -256,6 +256,37 @@ def test_round_trip_identity_and_one_hot(cb):
     torch.cuda.synchronize()
     # one-hot weights select exactly one expert row = the token's own row
     assert torch.equal(step.y.view(torch.int16), step.x.view(torch.int16))
+
+
+@pytest.mark.parametrize("name,T,chunks", [("3", 10001, 5), ("1", 4096, 8), ("2", 37, 8)])
+def test_host_driven_step_matches_the_resident_step(cb, name, T, chunks):
+    """route_host (pinned host buffers, token blocks overlapped with the copies) gives exactly the
+    results of route() on resident data."""
+    w = W.make_config(name, T=T)
+    layout, step = make_step(w)
+    step.route(w.seed)
+    torch.cuda.synchronize()
+    ref = {k: getattr(step, k).clone() for k in ("y", "coact", "load", "slot_load", "totals", "send", "row_of_pair")}
+    ids_h = torch.from_numpy(w.topk_ids).pin_memory()
+    w_h = torch.from_numpy(w.gate_w).pin_memory()
+    src_h = torch.from_numpy(w.src_rank).pin_memory()
+    x_h = bf16_tensor_from_bits(w.hidden_rows(), "cpu").pin_memory()
+    y_h = torch.zeros((w.T, w.H), dtype=torch.bfloat16).pin_memory()
+    coact_h = torch.zeros((w.E, w.E), dtype=torch.int32).pin_memory()
+    load_h = torch.zeros((w.E,), dtype=torch.int32).pin_memory()
+    sl_h = torch.zeros((w.D,), dtype=torch.int32).pin_memory()
+    tot_h = torch.zeros((2,), dtype=torch.int64).pin_memory()
+    for buf in (step.x, step.y, step.send, step.topk_ids, step.coact):
+        buf.zero_()
+    for _ in range(2):       # twice: the second call overlaps with the tail of the first
+        step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h, chunks=chunks)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    assert torch.equal(y_h.view(torch.int16), ref["y"].cpu().view(torch.int16))
+    assert torch.equal(coact_h, ref["coact"].cpu()) and torch.equal(load_h, ref["load"].cpu())
+    assert torch.equal(sl_h, ref["slot_load"].cpu()) and torch.equal(tot_h, ref["totals"].cpu())
+    assert torch.equal(step.send.view(torch.int16), ref["send"].view(torch.int16))
+    assert torch.equal(step.row_of_pair, ref["row_of_pair"])
 
 
 # ---------------------------------------------------------------------------------------------
