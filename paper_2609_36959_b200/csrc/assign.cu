@@ -21,13 +21,19 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
               uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
               uint32_t naive, uint32_t* __restrict__ err_word)
 {
-    extern __shared__ uint32_t smem[];
-    uint32_t* tab = smem;                       // lv.words
-    uint32_t* hist = smem + lv.words;           // lv.D (only when slot_load != nullptr)
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* tab = smem;                               // lv.words, padded to a multiple of 4
+    uint32_t* hist = smem + (lv.words + 3) / 4 * 4;     // lv.D (only when slot_load != nullptr)
     __shared__ unsigned long long cta_totals[2];
 
     const int K = (KT > 0) ? KT : K_rt;
-    for (int i = threadIdx.x; i < lv.words; i += blockDim.x) tab[i] = lv.blob[i];
+    {   // the blob is padded to whole 16-byte vectors
+        const uint4* src = reinterpret_cast<const uint4*>(lv.blob);
+        uint4* dst = reinterpret_cast<uint4*>(tab);
+        const int n_vec = (lv.words + 3) / 4;
+#pragma unroll 4
+        for (int i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = __ldg(src + i);
+    }
     if (slot_load)
         for (int i = threadIdx.x; i < lv.D; i += blockDim.x) hist[i] = 0;
     if (threadIdx.x < 2) cta_totals[threadIdx.x] = 0;
@@ -203,6 +209,7 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
         }
     }
     __syncthreads();
+    wait_for_prior_kernel();   // slot_load / totals may still be being cleared by the kernel before this one
     if (slot_load)
         for (int i = threadIdx.x; i < lv.D; i += blockDim.x)
             if (hist[i]) atomicAdd(&slot_load[i], hist[i]);
@@ -214,19 +221,27 @@ template <int KT>
 static int launch_assign(const LayoutView& lv, const int32_t* ids, const int32_t* src, int32_t src_uniform,
                          int64_t T, int32_t K, uint64_t seed, int32_t* assigned_slot, uint32_t* slot_load,
                          uint8_t* remote_nodes, uint64_t* totals, uint32_t naive, uint32_t* err_word,
-                         cudaStream_t stream)
+                         bool after_zeroing, cudaStream_t stream)
 {
-    const size_t smem = (static_cast<size_t>(lv.words) + (slot_load ? lv.D : 0)) * sizeof(uint32_t);
+    const size_t smem = (static_cast<size_t>(lv.words + 3) / 4 * 4 + (slot_load ? lv.D : 0)) * sizeof(uint32_t);
     auto kernel = assign_kernel<KT>;
     if (smem > 48 * 1024)
         COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(smem)));
     const unsigned grid = static_cast<unsigned>((T + kAssignThreads - 1) / kAssignThreads);
-    kernel<<<grid, kAssignThreads, smem, stream>>>(
-        lv, ids, src, src_uniform, T, K, static_cast<uint32_t>(seed & 0xFFFFFFFFu),
-        static_cast<uint32_t>(seed >> 32), assigned_slot, slot_load, remote_nodes,
-        reinterpret_cast<unsigned long long*>(totals), naive, err_word);
-    COBALT_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kAssignThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    set_programmatic_launch(&attr[0], after_zeroing);
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, ids, src, src_uniform, T, K,
+                                       static_cast<uint32_t>(seed & 0xFFFFFFFFu), static_cast<uint32_t>(seed >> 32),
+                                       assigned_slot, slot_load, remote_nodes,
+                                       reinterpret_cast<unsigned long long*>(totals), naive, err_word));
     return COBALT_OK;
 }
 
@@ -262,18 +277,19 @@ int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids, const 
     if (dev != layout->device) return COBALT_ERR_INVALID_ARG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (slot_load) COBALT_CUDA_TRY(cudaMemsetAsync(slot_load, 0, sizeof(uint32_t) * lv.D, s));
-    if (totals) COBALT_CUDA_TRY(cudaMemsetAsync(totals, 0, sizeof(uint64_t) * 2, s));
+    bool after_zeroing = false;
+    int rc = launch_zero_words(slot_load, lv.D, reinterpret_cast<uint32_t*>(totals), 4, s, &after_zeroing);
+    if (rc != COBALT_OK) return rc;
     if (T == 0) return COBALT_OK;
 
     uint32_t* err_word = nullptr;
-    int rc = device_error_word(&err_word);
+    rc = device_error_word(&err_word);
     if (rc != COBALT_OK) return rc;
     const uint32_t naive = (flags & COBALT_ASSIGN_NAIVE) ? 1u : 0u;
 #define COBALT_ASSIGN_CASE(KT)                                                                          \
     case KT:                                                                                            \
         return launch_assign<KT>(lv, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot,   \
-                                 slot_load, remote_nodes, totals, naive, err_word, s)
+                                 slot_load, remote_nodes, totals, naive, err_word, after_zeroing, s)
     switch (K) {
         COBALT_ASSIGN_CASE(1);
         COBALT_ASSIGN_CASE(2);
@@ -282,7 +298,7 @@ int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids, const 
         COBALT_ASSIGN_CASE(8);
         default:
             return launch_assign<0>(lv, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot,
-                                    slot_load, remote_nodes, totals, naive, err_word, s);
+                                    slot_load, remote_nodes, totals, naive, err_word, after_zeroing, s);
     }
 #undef COBALT_ASSIGN_CASE
 }

@@ -21,7 +21,7 @@ namespace cg = cooperative_groups;
 
 namespace cobalt {
 
-constexpr int kStatsThreads = 512;
+constexpr int kStatsThreads = 1024;
 constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 
 __host__ __device__ inline size_t tri_entries(int E) { return static_cast<size_t>(E) * (E + 1) / 2; }
@@ -111,6 +111,7 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     const int crank = static_cast<int>(cluster.block_rank());
     const int per = (n_vec + csize - 1) / csize;
     const int v0 = crank * per, v1 = min(n_vec, v0 + per);
+    wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
     for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
         uint4 s = make_uint4(0, 0, 0, 0);
         for (int r = 0; r < csize; ++r) {
@@ -138,6 +139,7 @@ __global__ void __launch_bounds__(256)
 coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int E,
                     uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
 {
+    wait_for_prior_kernel();
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
         int32_t id[COBALT_MAX_TOPK];
@@ -151,21 +153,21 @@ coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int 
 
 template <int KT>
 static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                       uint32_t* err_word, int n_sm, cudaStream_t stream)
+                       uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream)
 {
     auto kernel = coact_tile_kernel<KT>;
     const size_t smem = round_up(tri_entries(E) * sizeof(uint32_t), 16);
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
 
-    // about two tokens per thread, never more CTAs than can be co-resident (a second wave of
+    // about one token per thread, never more CTAs than can be co-resident (a second wave of
     // clusters would double the run time), clusters as large as the device schedules well
-    int64_t want = (T + 2 * kStatsThreads - 1) / (2 * kStatsThreads);
+    int64_t want = (T + kStatsThreads - 1) / kStatsThreads;
     if (want < 1) want = 1;
     if (want > n_sm) want = n_sm;
 
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cfg.blockDim = dim3(kStatsThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -225,6 +227,8 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     if (best_cs == 0) return COBALT_ERR_UNSUPPORTED;
     attr[0].val.clusterDim.x = best_cs;
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
+    set_programmatic_launch(&attr[1], after_zeroing);
+    cfg.numAttrs = 2;
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, coact, load, err_word));
     return COBALT_OK;
 }
@@ -254,14 +258,16 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     if (!aligned16(topk_ids) || !aligned16(coact) || !aligned16(load)) return COBALT_ERR_INVALID_ARG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int rc = COBALT_OK;
+    bool after_zeroing = false;
     if (!(flags & COBALT_STATS_ACCUMULATE)) {
-        COBALT_CUDA_TRY(cudaMemsetAsync(coact, 0, sizeof(uint32_t) * static_cast<size_t>(E) * E, s));
-        COBALT_CUDA_TRY(cudaMemsetAsync(load, 0, sizeof(uint32_t) * static_cast<size_t>(E), s));
+        rc = launch_zero_words(coact, E * E, load, E, s, &after_zeroing);
+        if (rc != COBALT_OK) return rc;
     }
     if (T == 0) return COBALT_OK;
 
     uint32_t* err_word = nullptr;
-    int rc = device_error_word(&err_word);
+    rc = device_error_word(&err_word);
     if (rc != COBALT_OK) return rc;
     int n_sm = 0;
     rc = sm_count(&n_sm);
@@ -270,17 +276,25 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     if (tri_entries(E) * sizeof(uint32_t) > kStatsMaxTileBytes) {
         int64_t want = (T + 255) / 256;
         const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
-        coact_global_kernel<<<grid, 256, 0, s>>>(topk_ids, T, K, E, coact, load, err_word);
-        COBALT_CUDA_TRY(cudaGetLastError());
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        set_programmatic_launch(&attr[0], after_zeroing);
+        COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, coact_global_kernel, topk_ids, T, static_cast<int>(K),
+                                           static_cast<int>(E), coact, load, err_word));
         return COBALT_OK;
     }
     switch (K) {
-        case 1: return launch_tile<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
-        case 2: return launch_tile<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
-        case 4: return launch_tile<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
-        case 6: return launch_tile<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
-        case 8: return launch_tile<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
-        default: return launch_tile<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, s);
+        case 1: return launch_tile<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        case 2: return launch_tile<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        case 4: return launch_tile<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        case 6: return launch_tile<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        case 8: return launch_tile<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        default: return launch_tile<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
     }
 }
 

@@ -116,6 +116,46 @@ __device__ __forceinline__ void st_stream16(void* p, uint4 v)
                  : "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with launch_after_zeroing() may start while
+// the zeroing kernel before it is still running; it must call wait_for_prior_kernel() before it
+// first touches memory the zeroing kernel writes.
+__device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Clears up to two small accumulator arrays (32-bit words) in one launch.
+static __global__ void zero_words_kernel(uint32_t* a, int n_a, uint32_t* b, int n_b)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start right away
+    const int stride = gridDim.x * blockDim.x;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_a; i += stride) a[i] = 0;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_b; i += stride) b[i] = 0;
+}
+
+// *launched tells the caller whether a zeroing kernel now precedes its own kernel in the stream:
+// only then may that kernel be launched programmatically (it would otherwise overlap with a
+// foreign kernel that may still be producing its inputs).
+static inline int launch_zero_words(uint32_t* a, int n_a, uint32_t* b, int n_b, cudaStream_t stream, bool* launched)
+{
+    *launched = false;
+    if (!a) n_a = 0;
+    if (!b) n_b = 0;
+    if (n_a + n_b == 0) return COBALT_OK;
+    *launched = true;
+    const int n = n_a > n_b ? n_a : n_b;
+    int grid = (n + 255) / 256;
+    if (grid > 296) grid = 296;
+    zero_words_kernel<<<grid, 256, 0, stream>>>(a, n_a, b, n_b);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
+// Fills a launch attribute that lets the kernel overlap with the tail of the previous kernel
+// in the stream (see wait_for_prior_kernel).
+static inline void set_programmatic_launch(cudaLaunchAttribute* attr, bool allowed)
+{
+    attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr->val.programmaticStreamSerializationAllowed = allowed ? 1 : 0;
+}
+
 #endif  // __CUDACC__
 
 }  // namespace cobalt

@@ -48,6 +48,7 @@ perm_hist_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
                  uint32_t* __restrict__ ws, uint32_t* __restrict__ err_word)
 {
     extern __shared__ uint32_t hist[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the scan kernel may be scheduled early
     for (int d = threadIdx.x; d < D; d += blockDim.x) hist[d] = 0;
     __syncthreads();
     const int64_t p0 = static_cast<int64_t>(blockIdx.x) * chunk;
@@ -70,6 +71,8 @@ perm_scan_kernel(uint32_t* __restrict__ ws, int D, int n_chunks, uint32_t* __res
 {
     const int d = blockIdx.x * kPermWarps + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    wait_for_prior_kernel();        // the histograms of the kernel before this one
     if (d >= D) return;
     uint32_t* row = ws + static_cast<size_t>(d) * n_chunks;
     uint32_t running = 0;
@@ -123,6 +126,8 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     __shared__ uint32_t warp_sums[kPermWarps];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < kPermWarps * D; i += kPermThreads) wcnt[i] = 0;
+    wait_for_prior_kernel();        // dest_counts and the scanned histograms of the kernel before this one
 
     // exclusive scan of dest_counts over d: thread-contiguous segments, then a block scan
     const int per = (D + kPermThreads - 1) / kPermThreads;
@@ -136,7 +141,6 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
         if (lane >= off) incl += up;
     }
     if (lane == 31) warp_sums[warp] = incl;
-    for (int i = tid; i < kPermWarps * D; i += kPermThreads) wcnt[i] = 0;
     __syncthreads();
     uint32_t before = incl - local;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
@@ -159,6 +163,7 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     const int n_super = (sub + 32 * kRankSteps - 1) / (32 * kRankSteps);
     const int key_bits = 32 - __clz(D);      // keys 0..D (D marks "no destination")
     int32_t dreg[kRankSteps];
+    uint32_t preg[kRankSteps];     // lanes sharing each step's destination (kept from pass A)
     auto load_super = [&](int ss) {
 #pragma unroll
         for (int s = 0; s < kRankSteps; ++s) {
@@ -175,6 +180,7 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
         for (int s = 0; s < kRankSteps; ++s) {
             const int32_t d = dreg[s];
             const uint32_t peers = peers_of(static_cast<uint32_t>(d < 0 ? D : d), key_bits);
+            preg[s] = peers;
             if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
             __syncwarp();
         }
@@ -193,12 +199,17 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     __syncthreads();
     // pass C: stable rank inside the warp's sub-range
     for (int ss = 0; ss < n_super; ++ss) {
-        if (n_super > 1) load_super(ss);     // a single super-step still holds its slots in registers
+        if (n_super > 1) {                   // a single super-step still holds its slots and peers
+            load_super(ss);
+#pragma unroll
+            for (int s = 0; s < kRankSteps; ++s)
+                preg[s] = peers_of(static_cast<uint32_t>(dreg[s] < 0 ? D : dreg[s]), key_bits);
+        }
 #pragma unroll
         for (int s = 0; s < kRankSteps; ++s) {
             const int64_t p = w0 + static_cast<int64_t>(ss) * 32 * kRankSteps + s * 32 + lane;
             const int32_t d = dreg[s];
-            const uint32_t peers = peers_of(static_cast<uint32_t>(d < 0 ? D : d), key_bits);
+            const uint32_t peers = preg[s];
             if (d >= 0) {
                 const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
                 row_of_pair[p] = static_cast<int32_t>(row);
@@ -591,6 +602,34 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     return COBALT_OK;
 }
 
+// K2 and K3, each launched programmatically after the kernel before it (their prologues overlap
+// with its tail; both wait for it before reading its results).
+static int launch_scan_and_rank(const int32_t* assigned_slot, int64_t P, int D, const ChunkPlan& c, uint32_t* ws,
+                                uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                                int32_t* pair_of_row, cudaStream_t s)
+{
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    set_programmatic_launch(&attr[0], true);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.stream = s;
+    cfg.blockDim = dim3(kPermThreads);
+    cfg.gridDim = dim3((D + kPermWarps - 1) / kPermWarps);
+    cfg.dynamicSmemBytes = 0;
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, perm_scan_kernel, ws, D, c.n_chunks, dest_counts));
+    const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
+    if (smem > 48 * 1024)
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem)));
+    cfg.gridDim = dim3(c.n_chunks);
+    cfg.dynamicSmemBytes = smem;
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, perm_rank_kernel, assigned_slot, P, D, c.chunk, c.n_chunks,
+                                       static_cast<const uint32_t*>(ws), static_cast<const uint32_t*>(dest_counts),
+                                       dest_offsets, row_of_pair, pair_of_row));
+    return COBALT_OK;
+}
+
 static int check_index_args(int64_t T, int32_t K, int32_t D)
 {
     if (T < 0 || K < 1 || D < 1) return COBALT_ERR_INVALID_ARG;
@@ -638,16 +677,7 @@ int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int
     perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
                                                                             c.n_chunks, ws, err_word);
     COBALT_CUDA_TRY(cudaGetLastError());
-    perm_scan_kernel<<<(D + kPermWarps - 1) / kPermWarps, kPermThreads, 0, s>>>(ws, D, c.n_chunks, dest_counts);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
-    if (smem > 48 * 1024)
-        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem)));
-    perm_rank_kernel<<<c.n_chunks, kPermThreads, smem, s>>>(assigned_slot, P, D, c.chunk, c.n_chunks, ws,
-                                                            dest_counts, dest_offsets, row_of_pair, pair_of_row);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    return COBALT_OK;
+    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, s);
 }
 
 // ---- no-allocation variant of the index half ------------------------------------------------
@@ -710,16 +740,7 @@ int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t
     perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
                                                                             c.n_chunks, ws, err_word);
     COBALT_CUDA_TRY(cudaGetLastError());
-    perm_scan_kernel<<<(D + kPermWarps - 1) / kPermWarps, kPermThreads, 0, s>>>(ws, D, c.n_chunks, dest_counts);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
-    if (smem > 48 * 1024)
-        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem)));
-    perm_rank_kernel<<<c.n_chunks, kPermThreads, smem, s>>>(assigned_slot, P, D, c.chunk, c.n_chunks, ws,
-                                                            dest_counts, dest_offsets, row_of_pair, pair_of_row);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    return COBALT_OK;
+    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, s);
 }
 
 int cobalt_permute_rows_block(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,

@@ -95,7 +95,7 @@ static int build_tables(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
     view->blob = nullptr;
     if (!blob) return COBALT_OK;
 
-    blob->assign(static_cast<size_t>(view->words), 0u);
+    blob->assign(static_cast<size_t>(view->words + 3) / 4 * 4, 0u);   // whole 16-byte vectors
     uint32_t* ent = blob->data() + view->ent_off();
     uint32_t* primary = blob->data() + view->primary_off();
     uint32_t* rlist = blob->data() + view->rlist_off();

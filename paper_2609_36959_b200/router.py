@@ -76,7 +76,7 @@ class RouteStep:
     # -- the same step from pinned host memory ----------------------------------------------
     def route_host(self, seed: int, ids_h: torch.Tensor, w_h: torch.Tensor, src_h: torch.Tensor,
                    x_h: torch.Tensor, y_h: torch.Tensor, coact_h: torch.Tensor, load_h: torch.Tensor,
-                   slot_load_h: torch.Tensor, totals_h: torch.Tensor, chunks: int = 8) -> None:
+                   slot_load_h: torch.Tensor, totals_h: torch.Tensor, chunks: int = 16) -> None:
         """One step with inputs and results in pinned host memory.
 
         The gating output is small and goes first, so statistics, assignment and the permutation
@@ -96,25 +96,35 @@ class RouteStep:
         chunks = max(1, min(chunks, T)) if T > 0 else 1
         # block starts on multiples of 4 tokens keep every offset pointer 16-byte aligned for any K
         bounds = [min(T, ((T * c) // chunks + 3) // 4 * 4) for c in range(chunks)] + [T]
+        # All copies of one direction go through one stream, the gating output ahead of the hidden
+        # rows: copies in a direction share a copy engine, and a small copy issued from another
+        # stream can end up queued behind every row block that is ready at the same moment.
         ready = []
         with torch.cuda.stream(h2d):
+            self.topk_ids.copy_(ids_h, non_blocking=True)
+            self.gate_w.copy_(w_h, non_blocking=True)
+            self.src_rank.copy_(src_h, non_blocking=True)
+            gating_ready = torch.cuda.Event()
+            gating_ready.record(h2d)
             for c in range(chunks):
                 t0, t1 = bounds[c], bounds[c + 1]
                 self.x[t0:t1].copy_(x_h[t0:t1], non_blocking=True)
                 ev = torch.cuda.Event()
                 ev.record(h2d)
                 ready.append(ev)
-        self.topk_ids.copy_(ids_h, non_blocking=True)
-        self.gate_w.copy_(w_h, non_blocking=True)
-        self.src_rank.copy_(src_h, non_blocking=True)
+        main.wait_event(gating_ready)
         self.stats()
         self.assign(seed)
         cb.permute_index(self.assigned_slot, self.D, self.dest_counts, self.dest_offsets, self.row_of_pair,
                          self.pair_of_row, self.workspace)
-        coact_h.copy_(self.coact, non_blocking=True)
-        load_h.copy_(self.load, non_blocking=True)
-        slot_load_h.copy_(self.slot_load, non_blocking=True)
-        totals_h.copy_(self.totals, non_blocking=True)
+        index_done = torch.cuda.Event()
+        index_done.record(main)
+        with torch.cuda.stream(d2h):
+            d2h.wait_event(index_done)
+            coact_h.copy_(self.coact, non_blocking=True)
+            load_h.copy_(self.load, non_blocking=True)
+            slot_load_h.copy_(self.slot_load, non_blocking=True)
+            totals_h.copy_(self.totals, non_blocking=True)
         for c in range(chunks):
             t0, t1 = bounds[c], bounds[c + 1]
             if t1 == t0:
