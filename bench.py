@@ -35,7 +35,7 @@ KERNELS_PER_STEP = 7               # stats 1, assign 1, permute 4 (hist, scan, r
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes per pair, measured on a reduced token count and scaled by the pairs of a launch)
-NCU_TRAFFIC_BYTES_PER_PAIR = {}
+NCU_TRAFFIC_BYTES_PER_PAIR = {"permute_rows": 15683.4, "combine": 15972.4}   # profiles/perm_rows_and_combine_T16384.md
 
 
 def parse_args():
