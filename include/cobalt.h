@@ -68,6 +68,7 @@ extern "C" {
 /* flag bits */
 #define COBALT_STATS_ACCUMULATE 0x1u         /* add to coact/load instead of overwriting them */
 #define COBALT_ASSIGN_NAIVE 0x1u             /* primary-replica rule instead of Algorithm 1 */
+#define COBALT_ASSIGN_ROUND_ROBIN 0x2u       /* deal each (expert, node) group's tasks to its replicas in turn */
 #define COBALT_IMPL_MASK 0xF00u              /* kernel variant override, 0 = library default */
 #define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
 #define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies, one work item per CTA (default) */
@@ -124,7 +125,13 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
  * slot_load uint32 [D] = w_er (Section 3.1), remote_nodes uint8 [T] = the token's term of
  * Eq. 1, totals uint64 [2] = { V of this assignment, V of the naive primary-replica rule }.
  * The optional outputs are overwritten.  COBALT_ASSIGN_NAIVE assigns every task to its
- * expert's primary replica instead (the one-replica-per-expert baseline). */
+ * expert's primary replica instead (the one-replica-per-expert baseline).
+ * COBALT_ASSIGN_ROUND_ROBIN (not in the paper) keeps Step 1 and replaces the hashed replica
+ * pick of Step 2: walking the pairs in ascending p, the j-th task of group (expert, node) goes
+ * to R_{e,n}[j mod |R_{e,n}|], so replica loads inside a group differ by at most one.  The
+ * running count is reproduced exactly (chunk histograms, scan, stable rank), never with racing
+ * counters.  This mode needs the workspace of cobalt_assign_workspace_bytes and E*N <= 4096;
+ * the other modes need none. */
 size_t cobalt_assign_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);
 int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids,
                   const int32_t* src_rank, int32_t src_rank_uniform, int64_t T, int32_t K,
@@ -160,6 +167,23 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
                    uint32_t* dest_offsets, int32_t* row_of_pair, int32_t* pair_of_row,
                    uint32_t flags, void* workspace, size_t workspace_bytes,
                    cobalt_stream_t stream);
+
+/* ---- stages 1 + 2 + index half of stage 3 in one pass over the ids ---------------------------
+ * Same outputs, bit for bit, as cobalt_coact_stats, cobalt_assign (Algorithm 1, hashed replica
+ * pick) and cobalt_permute_index called one after the other, with dest_counts = slot_load = w_er.
+ * The top-k ids are read once and the co-activation triangle, the layout tables and the chunk
+ * histograms of the permutation share one cluster-launched kernel; the scan and stable-rank
+ * kernels follow.  (Section 3.2 Stage 1, Section 3.3 Algorithm 1, Fig. 1 "Dispatch".)
+ * flags: COBALT_STATS_ACCUMULATE only.  remote_nodes, totals, pair_of_row may be NULL.
+ * Follow with cobalt_permute_rows to fill the send buffer. */
+size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);
+int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
+                       int32_t src_rank_uniform, int64_t T, int32_t K, uint64_t seed,
+                       uint32_t* coact, uint32_t* load, int32_t* assigned_slot,
+                       uint8_t* remote_nodes, uint64_t* totals, uint32_t* dest_counts,
+                       uint32_t* dest_offsets, int32_t* row_of_pair, int32_t* pair_of_row,
+                       uint32_t flags, void* workspace, size_t workspace_bytes,
+                       cobalt_stream_t stream);
 
 /* ---- index half of stage 3 for callers that cannot provide device scratch -------------------
  * (No counterpart in the paper: this is a packaging variant of cobalt_permute_index, same

@@ -97,8 +97,8 @@ def coact_stats(topk_ids, E: int):
 
 
 def assign(N: int, Q: int, S: int, E: int, slot_expert, primary_slot, topk_ids, src_rank, seed: int,
-           *, naive: bool = False):
-    """Algorithm 1 (or the naive primary-replica rule).
+           *, naive: bool = False, round_robin: bool = False):
+    """Algorithm 1 (or the naive primary-replica rule; or Algorithm 1 with the round-robin replica pick).
 
     -> dict(assigned_slot int32 [T,K], slot_load uint32 [D], remote_nodes uint8 [T],
             V int, V_naive int)
@@ -114,7 +114,8 @@ def assign(N: int, Q: int, S: int, E: int, slot_expert, primary_slot, topk_ids, 
     remote = np.zeros(T, np.uint8)
     totals = np.zeros(2, np.uint64)
     _check(_lib.oracle_assign(N, Q, S, E, slot_expert, _opt_ptr(prim_in), ids, src, T, K,
-                              seed & (2**64 - 1), 1 if naive else 0, out, slot_load, remote, totals),
+                              seed & (2**64 - 1), (1 if naive else 0) | (2 if round_robin else 0), out, slot_load,
+                              remote, totals),
            "assign")
     return dict(assigned_slot=out, slot_load=slot_load, remote_nodes=remote,
                 V=int(totals[0]), V_naive=int(totals[1]))

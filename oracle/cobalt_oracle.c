@@ -157,6 +157,11 @@ int oracle_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
  * (Section 3.1); optional remote_nodes[t] = BitCount(b*) (0 when U_t is empty) = the token's
  * term of Eq. 1; optional totals[0] = V of this assignment, totals[1] = V of the naive rule.
  * flags bit0: use the naive primary-replica rule (every task goes to primary[e]) instead.
+ * flags bit1: round-robin replica pick.  Step 1 is unchanged; in Step 2 the tasks of a group
+ *   (expert e, node n) are dealt to R_{e,n} in turn: walking the pairs in ascending p = t*K + k,
+ *   the j-th task of the group (j from 0) goes to R_{e,n}[j mod |R_{e,n}|].  This makes "equal
+ *   workloads in expectation" (Section 3.3, Step 2) exact: replica loads inside a group differ
+ *   by at most one.  Not in the paper; an optional mode of this repository.
  * ---------------------------------------------------------------------------------------- */
 int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
                   const int32_t* slot_expert, const int32_t* primary_in,
@@ -172,8 +177,9 @@ int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
     int32_t* primary = (int32_t*)malloc(sizeof(int32_t) * (size_t)E);
     uint32_t* m = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)(K > 0 ? K : 1));
     int32_t* n_te = (int32_t*)malloc(sizeof(int32_t) * (size_t)(K > 0 ? K : 1));
+    uint32_t* dealt = (uint32_t*)calloc((size_t)E * N, sizeof(uint32_t));   /* tasks seen per (e, n) group */
     int rc = ORACLE_ERR_ALLOC;
-    if (!nodes_mask || !r_count || !r_list || !primary || !m || !n_te) goto done;
+    if (!nodes_mask || !r_count || !r_list || !primary || !m || !n_te || !dealt) goto done;
     rc = oracle_layout_tables(N, Q, S, E, slot_expert, primary_in, nodes_mask, r_count, r_list, primary);
     if (rc != ORACLE_OK) goto done;
 
@@ -260,8 +266,14 @@ int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
         /* lines 14-16 */
         for (int32_t a = 0; a < K; ++a) {
             int64_t en = (int64_t)D_t[a] * N + n_te[a];
-            uint32_t i = oracle_hash_index(oracle_hash(seed, (uint32_t)t, (uint32_t)D_t[a], 1u),
-                                           (uint32_t)r_count[en]);
+            uint32_t i;
+            if (flags & 2u) {
+                i = dealt[en] % (uint32_t)r_count[en];
+                dealt[en] += 1;
+            } else {
+                i = oracle_hash_index(oracle_hash(seed, (uint32_t)t, (uint32_t)D_t[a], 1u),
+                                      (uint32_t)r_count[en]);
+            }
             int32_t d = r_list[en * Q + i];
             assigned_slot[t * K + a] = d;
             if (slot_load) slot_load[d] += 1;
@@ -274,7 +286,7 @@ int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
     if (totals) { totals[0] = V; totals[1] = V_naive; }
     rc = ORACLE_OK;
 done:
-    free(nodes_mask); free(r_count); free(r_list); free(primary); free(m); free(n_te);
+    free(nodes_mask); free(r_count); free(r_list); free(primary); free(m); free(n_te); free(dealt);
     return rc;
 }
 

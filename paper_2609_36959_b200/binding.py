@@ -32,6 +32,7 @@ DEVERR_WAIT_TIMEOUT = 0x10
 
 STATS_ACCUMULATE = 0x1
 ASSIGN_NAIVE = 0x1
+ASSIGN_ROUND_ROBIN = 0x2
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200
 IMPL_BULK_RING = 0x300
@@ -44,6 +45,7 @@ EXPORTS = (
     "cobalt_assign_workspace_bytes", "cobalt_assign",
     "cobalt_permute_workspace_bytes", "cobalt_permute_index", "cobalt_permute_rows", "cobalt_permute",
     "cobalt_permute_index_static", "cobalt_permute_rows_block", "cobalt_combine_block",
+    "cobalt_route_index_workspace_bytes", "cobalt_route_index",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -79,6 +81,9 @@ def _load() -> C.CDLL:
         "cobalt_permute_rows": (C.c_int, [vp, vp, i64, i32, i32, vp, u32, vp]),
         "cobalt_permute": (C.c_int, [vp, i64, i32, i32, vp, i32, vp, vp, vp, vp, vp, u32, vp, sz, vp]),
         "cobalt_combine": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, u32, vp]),
+        "cobalt_route_index_workspace_bytes": (sz, [vp, i64, i32]),
+        "cobalt_route_index": (C.c_int, [vp, vp, vp, i32, i64, i32, u64, vp, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp,
+                                         sz, vp]),
         "cobalt_permute_rows_block": (C.c_int, [vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_combine_block": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_read_and_clear_device_error": (C.c_int, [C.POINTER(u32), vp]),
@@ -222,6 +227,42 @@ def assign(layout: Layout, topk_ids: torch.Tensor, src_rank, seed: int, assigned
                               _ptr(remote_nodes, torch.uint8, "remote_nodes"),
                               _ptr(totals, torch.int64, "totals"), flags, _ptr(workspace), ws_bytes,
                               _stream()), "cobalt_assign")
+
+
+def route_index_workspace_bytes(layout: Layout, T: int, K: int) -> int:
+    return _lib.cobalt_route_index_workspace_bytes(layout.handle, T, K)
+
+
+def route_index(layout: Layout, topk_ids: torch.Tensor, src_rank, seed: int, coact: torch.Tensor,
+                load: torch.Tensor, assigned_slot: torch.Tensor, dest_counts: torch.Tensor,
+                dest_offsets: torch.Tensor, row_of_pair: torch.Tensor, workspace: torch.Tensor, *,
+                remote_nodes: Optional[torch.Tensor] = None, totals: Optional[torch.Tensor] = None,
+                pair_of_row: Optional[torch.Tensor] = None, flags: int = 0) -> None:
+    """Statistics, assignment and the permutation index in one pass over the ids."""
+    T, K = topk_ids.shape
+    E, D = layout.E, layout.D
+    if coact.numel() != E * E or load.numel() != E or assigned_slot.numel() != T * K:
+        raise CobaltError(ERR_INVALID_ARG, "route_index (output sizes)")
+    _check_index_outputs(T, K, D, dest_counts, dest_offsets, row_of_pair, pair_of_row, "route_index")
+    if remote_nodes is not None and remote_nodes.numel() != T:
+        raise CobaltError(ERR_INVALID_ARG, "route_index (remote_nodes size)")
+    if totals is not None and totals.numel() != 2:
+        raise CobaltError(ERR_INVALID_ARG, "route_index (totals size)")
+    if isinstance(src_rank, int):
+        src_ptr, src_uniform = None, src_rank
+    else:
+        if src_rank.numel() != T:
+            raise CobaltError(ERR_INVALID_ARG, "route_index (src_rank size)")
+        src_ptr, src_uniform = _ptr(src_rank, torch.int32, "src_rank"), 0
+    _check(_lib.cobalt_route_index(layout.handle, _ptr(topk_ids, torch.int32, "topk_ids"), src_ptr, src_uniform, T, K,
+                                   seed & (2**64 - 1), _ptr(coact, torch.int32, "coact"),
+                                   _ptr(load, torch.int32, "load"), _ptr(assigned_slot, torch.int32, "assigned_slot"),
+                                   _ptr(remote_nodes, torch.uint8, "remote_nodes"), _ptr(totals, torch.int64, "totals"),
+                                   _ptr(dest_counts, torch.int32, "dest_counts"),
+                                   _ptr(dest_offsets, torch.int32, "dest_offsets"),
+                                   _ptr(row_of_pair, torch.int32, "row_of_pair"),
+                                   _ptr(pair_of_row, torch.int32, "pair_of_row"), flags, _ptr(workspace),
+                                   _ws_bytes(workspace), _stream()), "cobalt_route_index")
 
 
 def permute_workspace_bytes(T: int, K: int, D: int) -> int:

@@ -15,7 +15,7 @@
 #include <tuple>
 #include <utility>
 
-#include "common.cuh"
+#include "token_core.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -24,114 +24,36 @@ namespace cobalt {
 constexpr int kStatsThreads = 1024;
 constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 
-__host__ __device__ inline size_t tri_entries(int E) { return static_cast<size_t>(E) * (E + 1) / 2; }
-
-template <int KT>
-__device__ __forceinline__ bool load_token_ids(const int32_t* __restrict__ ids, int64_t t, int K, int E,
-                                               int32_t (&id)[(KT > 0) ? KT : COBALT_MAX_TOPK],
-                                               uint32_t* err_word)
-{
-    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
-    const int32_t* row = ids + t * K;
-    if (KT > 0 && KT % 4 == 0) {
-#pragma unroll
-        for (int a = 0; a < KT / 4; ++a) {
-            const int4 v = __ldg(reinterpret_cast<const int4*>(row) + a);
-            id[4 * a] = v.x; id[4 * a + 1] = v.y; id[4 * a + 2] = v.z; id[4 * a + 3] = v.w;
-        }
-    } else if (KT > 0 && KT % 2 == 0) {
-#pragma unroll
-        for (int a = 0; a < KT / 2; ++a) {
-            const int2 v = __ldg(reinterpret_cast<const int2*>(row) + a);
-            id[2 * a] = v.x; id[2 * a + 1] = v.y;
-        }
-    } else {
-#pragma unroll
-        for (int a = 0; a < KMAX; ++a)
-            if (a < K) id[a] = __ldg(row + a);
-    }
-    uint32_t bad = 0;
-#pragma unroll
-    for (int a = 0; a < KMAX; ++a) {
-        if (a < K) {
-            if (id[a] < 0 || id[a] >= E) bad |= COBALT_DEVERR_BAD_EXPERT_ID;
-#pragma unroll
-            for (int b = 0; b < a; ++b)
-                if (id[b] == id[a]) bad |= COBALT_DEVERR_DUPLICATE_ID;
-        }
-    }
-    if (bad) flag_error(err_word, bad);
-    return bad == 0;
-}
-
-// Row of the lower triangle that holds flat index idx (row hi starts at hi*(hi+1)/2).
-__device__ __forceinline__ int tri_row(int idx)
-{
-    int hi = static_cast<int>((sqrtf(8.0f * static_cast<float>(idx) + 1.0f) - 1.0f) * 0.5f);
-    while (hi * (hi + 1) / 2 > idx) --hi;
-    while ((hi + 1) * (hi + 2) / 2 <= idx) ++hi;
-    return hi;
-}
-
 template <int KT>
 __global__ void __launch_bounds__(kStatsThreads)
 coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E,
                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(16) uint32_t tri[];   // lower triangle, padded to whole uint4
-    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    constexpr int KMAX = TokenShape<KT>::KMAX;
     const int K = (KT > 0) ? KT : K_rt;
     cg::cluster_group cluster = cg::this_cluster();
 
-    const int n_tri = static_cast<int>(tri_entries(E));
-    const int n_vec = (n_tri + 3) / 4;
+    const int n_vec = (static_cast<int>(tri_entries(E)) + 3) / 4;
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
         int32_t id[KMAX];
-        if (!load_token_ids<KT>(topk_ids, t, K, E, id, err_word)) continue;
-#pragma unroll
-        for (int a = 0; a < KMAX; ++a) {
-#pragma unroll
-            for (int b = a; b < KMAX; ++b) {
-                if (b < K) {
-                    const int hi = max(id[a], id[b]), lo = min(id[a], id[b]);
-                    atomicAdd(&tri[hi * (hi + 1) / 2 + lo], 1u);
-                }
-            }
+        load_token_ids<KT>(topk_ids, t, K, id);
+        const uint32_t bad = check_token_ids<KT>(id, K, E);
+        if (bad) {
+            flag_error(err_word, bad);
+            continue;
         }
+        add_token_to_triangle<KT>(tri, id, K);
     }
 
-    cluster.sync();  // every tile of the cluster is complete
-    // Each CTA owns a contiguous slice of the flat triangle and sums it over all tiles of the
-    // cluster with 16-byte distributed-shared-memory loads (all threads busy, loads independent).
-    const int csize = static_cast<int>(cluster.num_blocks());
-    const int crank = static_cast<int>(cluster.block_rank());
-    const int per = (n_vec + csize - 1) / csize;
-    const int v0 = crank * per, v1 = min(n_vec, v0 + per);
+    cluster.sync();            // every tile of the cluster is complete
     wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
-    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
-        uint4 s = make_uint4(0, 0, 0, 0);
-        for (int r = 0; r < csize; ++r) {
-            const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
-            s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
-        }
-        const uint32_t part[4] = {s.x, s.y, s.z, s.w};
-        int hi = tri_row(4 * v);
-        int lo = 4 * v - hi * (hi + 1) / 2;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (4 * v + c < n_tri && part[c]) {
-                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], part[c]);
-                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], part[c]);
-                else atomicAdd(&load[hi], part[c]);
-            }
-            if (++lo > hi) { ++hi; lo = 0; }
-        }
-    }
-    cluster.sync();  // no CTA may exit while a peer still reads its tile
+    merge_triangle_over_cluster(tri, E, coact, load);
+    cluster.sync();            // no CTA may exit while a peer still reads its tile
 }
 
 // Fallback for expert counts whose triangle does not fit in shared memory.
@@ -143,7 +65,12 @@ coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int 
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
         int32_t id[COBALT_MAX_TOPK];
-        if (!load_token_ids<0>(topk_ids, t, K, E, id, err_word)) continue;
+        load_token_ids<0>(topk_ids, t, K, id);
+        const uint32_t bad = check_token_ids<0>(id, K, E);
+        if (bad) {
+            flag_error(err_word, bad);
+            continue;
+        }
         for (int a = 0; a < K; ++a) {
             atomicAdd(&load[id[a]], 1u);
             for (int b = 0; b < K; ++b) atomicAdd(&coact[static_cast<size_t>(id[a]) * E + id[b]], 1u);

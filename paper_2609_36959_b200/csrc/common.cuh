@@ -121,31 +121,45 @@ __device__ __forceinline__ void st_stream16(void* p, uint4 v)
 // first touches memory the zeroing kernel writes.
 __device__ __forceinline__ void wait_for_prior_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// Clears up to two small accumulator arrays (32-bit words) in one launch.
-static __global__ void zero_words_kernel(uint32_t* a, int n_a, uint32_t* b, int n_b)
+// Clears up to four small accumulator arrays (32-bit words) in one launch.
+struct ZeroList {
+    uint32_t* ptr[4];
+    int n[4];
+};
+
+static __global__ void zero_words_kernel(ZeroList z)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start right away
     const int stride = gridDim.x * blockDim.x;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_a; i += stride) a[i] = 0;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_b; i += stride) b[i] = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+        for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < z.n[k]; i += stride) z.ptr[k][i] = 0;
 }
 
 // *launched tells the caller whether a zeroing kernel now precedes its own kernel in the stream:
 // only then may that kernel be launched programmatically (it would otherwise overlap with a
 // foreign kernel that may still be producing its inputs).
-static inline int launch_zero_words(uint32_t* a, int n_a, uint32_t* b, int n_b, cudaStream_t stream, bool* launched)
+static inline int launch_zero_list(ZeroList z, cudaStream_t stream, bool* launched)
 {
     *launched = false;
-    if (!a) n_a = 0;
-    if (!b) n_b = 0;
-    if (n_a + n_b == 0) return COBALT_OK;
+    int most = 0;
+    for (int k = 0; k < 4; ++k) {
+        if (!z.ptr[k]) z.n[k] = 0;
+        if (z.n[k] > most) most = z.n[k];
+    }
+    if (most == 0) return COBALT_OK;
     *launched = true;
-    const int n = n_a > n_b ? n_a : n_b;
-    int grid = (n + 255) / 256;
+    int grid = (most + 255) / 256;
     if (grid > 296) grid = 296;
-    zero_words_kernel<<<grid, 256, 0, stream>>>(a, n_a, b, n_b);
+    zero_words_kernel<<<grid, 256, 0, stream>>>(z);
     COBALT_CUDA_TRY(cudaGetLastError());
     return COBALT_OK;
+}
+
+static inline int launch_zero_words(uint32_t* a, int n_a, uint32_t* b, int n_b, cudaStream_t stream, bool* launched)
+{
+    ZeroList z = {{a, b, nullptr, nullptr}, {n_a, n_b, 0, 0}};
+    return launch_zero_list(z, stream, launched);
 }
 
 // Fills a launch attribute that lets the kernel overlap with the tail of the previous kernel

@@ -14,23 +14,16 @@
 // bulk async copy shared -> global per destination row, many small CTAs in flight per SM;
 // a persistent variant of the same with a shared-memory ring; and plain 16-byte streaming
 // loads/stores.
-#include "common.cuh"
+#include "permute_index.cuh"
 
 namespace cobalt {
 
-constexpr int kPermThreads = 256;
 constexpr int kPermWarps = kPermThreads / 32;
 constexpr int kMinChunk = 2048;      // pairs per chunk (multiple of kPermThreads)
 constexpr int kMaxChunks = 2048;
 constexpr int kRankSteps = kMinChunk / kPermWarps / 32;   // 32-pair steps of a warp per super-step
 
-struct ChunkPlan {
-    int64_t P;
-    int chunk;        // pairs per chunk
-    int n_chunks;
-};
-
-static ChunkPlan plan_chunks(int64_t P)
+ChunkPlan plan_chunks(int64_t P)
 {
     ChunkPlan c;
     c.P = P;
@@ -118,7 +111,7 @@ __global__ void __launch_bounds__(kPermThreads)
 perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
                  const uint32_t* __restrict__ ws, const uint32_t* __restrict__ dest_counts,
                  uint32_t* __restrict__ dest_offsets, int32_t* __restrict__ row_of_pair,
-                 int32_t* __restrict__ pair_of_row)
+                 int32_t* __restrict__ pair_of_row, int rank_in_group)
 {
     extern __shared__ uint32_t sm[];
     uint32_t* base = sm;                 // [D]   first row of this chunk inside destination d
@@ -146,7 +139,8 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
     for (int d = d_lo; d < d_hi; ++d) {
         if (blockIdx.x == 0) dest_offsets[d] = before;
-        base[d] = before + __ldg(ws + static_cast<size_t>(d) * n_chunks + blockIdx.x);
+        // rank_in_group: ranks count from 0 inside each destination instead of from its offset
+        base[d] = (rank_in_group ? 0u : before) + __ldg(ws + static_cast<size_t>(d) * n_chunks + blockIdx.x);
         before += __ldg(dest_counts + d);
     }
     if (blockIdx.x == 0 && tid == kPermThreads - 1) dest_offsets[D] = before;  // last thread ends at D
@@ -604,9 +598,9 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
 
 // K2 and K3, each launched programmatically after the kernel before it (their prologues overlap
 // with its tail; both wait for it before reading its results).
-static int launch_scan_and_rank(const int32_t* assigned_slot, int64_t P, int D, const ChunkPlan& c, uint32_t* ws,
-                                uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
-                                int32_t* pair_of_row, cudaStream_t s)
+int launch_scan_and_rank(const int32_t* assigned_slot, int64_t P, int D, const ChunkPlan& c, uint32_t* ws,
+                         uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                         int32_t* pair_of_row, int rank_in_group, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -626,7 +620,16 @@ static int launch_scan_and_rank(const int32_t* assigned_slot, int64_t P, int D, 
     cfg.dynamicSmemBytes = smem;
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, perm_rank_kernel, assigned_slot, P, D, c.chunk, c.n_chunks,
                                        static_cast<const uint32_t*>(ws), static_cast<const uint32_t*>(dest_counts),
-                                       dest_offsets, row_of_pair, pair_of_row));
+                                       dest_offsets, row_of_pair, pair_of_row, rank_in_group));
+    return COBALT_OK;
+}
+
+int launch_chunk_histograms(const int32_t* keys, int64_t P, int D, const ChunkPlan& c, uint32_t* ws,
+                            uint32_t* err_word, cudaStream_t s)
+{
+    perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(keys, P, D, c.chunk, c.n_chunks, ws,
+                                                                            err_word);
+    COBALT_CUDA_TRY(cudaGetLastError());
     return COBALT_OK;
 }
 
@@ -674,10 +677,9 @@ int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int
     rc = device_error_word(&err_word);
     if (rc != COBALT_OK) return rc;
 
-    perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
-                                                                            c.n_chunks, ws, err_word);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, s);
+    rc = launch_chunk_histograms(assigned_slot, P, D, c, ws, err_word, s);
+    if (rc != COBALT_OK) return rc;
+    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, 0, s);
 }
 
 // ---- no-allocation variant of the index half ------------------------------------------------
@@ -737,10 +739,9 @@ int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t
     // entries, zeros included), so nothing left over from an earlier call is ever consumed and
     // no clearing pass is needed.
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    perm_hist_kernel<<<c.n_chunks, kPermThreads, sizeof(uint32_t) * D, s>>>(assigned_slot, P, D, c.chunk,
-                                                                            c.n_chunks, ws, err_word);
-    COBALT_CUDA_TRY(cudaGetLastError());
-    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, s);
+    rc = launch_chunk_histograms(assigned_slot, P, D, c, ws, err_word, s);
+    if (rc != COBALT_OK) return rc;
+    return launch_scan_and_rank(assigned_slot, P, D, c, ws, dest_counts, dest_offsets, row_of_pair, pair_of_row, 0, s);
 }
 
 int cobalt_permute_rows_block(const void* x, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,

@@ -1,0 +1,355 @@
+// Fused index pass: statistics (stage 1), assignment (stage 2) and the per-chunk destination
+// histograms of the permutation (first kernel of stage 3) in ONE pass over the top-k ids.
+//
+// The separate entry points read the ids three times and launch six kernels before the scan;
+// for the few megabytes involved those launches, not the bytes, set the time.  Here one
+// cluster-launched kernel keeps, per CTA, the co-activation triangle, the layout tables and the
+// chunk histograms in shared memory; every thread owns one token per round: it adds the token's
+// K(K+1)/2 pairs to the triangle, runs Algorithm 1, stores the K slots and counts them in the
+// histogram of its permutation chunk (256 consecutive tokens = 8 warps).  The triangle is then
+// merged over the cluster exactly as in the stand-alone statistics kernel; the scan and rank
+// kernels of the permutation follow.  Results are bit-identical to the separate calls.
+#include <cooperative_groups.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <utility>
+
+#include "permute_index.cuh"
+#include "token_core.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace cobalt {
+
+constexpr int kRouteThreads = 1024;
+constexpr int kRouteChunkTokens = 256;                              // tokens per permutation chunk
+constexpr int kRouteChunksPerRound = kRouteThreads / kRouteChunkTokens;
+constexpr size_t kRouteMaxSmem = 220 * 1024;
+
+struct RouteSmem {
+    size_t tri_words, tab_words, hist_words;
+    size_t bytes() const { return (tri_words + tab_words + hist_words) * sizeof(uint32_t); }
+};
+
+static RouteSmem route_smem(const LayoutView& lv)
+{
+    RouteSmem r;
+    r.tri_words = (tri_entries(lv.E) + 3) / 4 * 4;
+    r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
+    r.hist_words = static_cast<size_t>(kRouteChunksPerRound) * lv.D;
+    return r;
+}
+
+template <int KT>
+__global__ void __launch_bounds__(kRouteThreads)
+route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ src_rank,
+                   int32_t src_uniform, int64_t T, int32_t K_rt, uint32_t seed_lo, uint32_t seed_hi,
+                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot,
+                   uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
+                   uint32_t* __restrict__ chunk_ws, int n_chunks, int tri_words, int tab_words,
+                   uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* tri = smem;
+    uint32_t* tab = smem + tri_words;
+    uint32_t* chist = tab + tab_words;            // [kRouteChunksPerRound][D]
+    __shared__ unsigned long long cta_totals[2];
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    const int K = (KT > 0) ? KT : K_rt;
+    const int D = lv.D;
+    cg::cluster_group cluster = cg::this_cluster();
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the scan kernel may be scheduled early
+    for (int i = threadIdx.x; i < tri_words / 4; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < kRouteChunksPerRound * D; i += blockDim.x) chist[i] = 0;
+    if (threadIdx.x < 2) cta_totals[threadIdx.x] = 0;
+    const TableView tv = stage_tables(lv, tab);
+    __syncthreads();
+
+    const int64_t tokens_per_round = static_cast<int64_t>(gridDim.x) * kRouteThreads;
+    const int n_rounds = static_cast<int>((T + tokens_per_round - 1) / tokens_per_round);
+    uint32_t cost_sum = 0, naive_sum = 0;
+    for (int round = 0; round < n_rounds; ++round) {
+        const int64_t base = (static_cast<int64_t>(round) * gridDim.x + blockIdx.x) * kRouteThreads;
+        const int64_t t = base + threadIdx.x;
+        if (t < T) {
+            int32_t id[KMAX], out[KMAX];
+            load_token_ids<KT>(topk_ids, t, K, id);
+            const int32_t s_t = src_rank ? __ldg(src_rank + t) : src_uniform;
+            const uint32_t bad_ids = check_token_ids<KT>(id, K, lv.E);
+            uint32_t bad = bad_ids;
+            if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
+            if (bad) flag_error(err_word, bad);
+            // the statistics only need valid ids, as in the stand-alone statistics call
+            if (!bad_ids) add_token_to_triangle<KT>(tri, id, K);
+            uint32_t cost = 0, naive_cost = 0;
+            if (bad) {
+#pragma unroll
+                for (int a = 0; a < KMAX; ++a) out[a] = -1;
+            } else {
+                assign_token<KT, kAssignSlot>(tv, id, K, s_t, static_cast<uint32_t>(t), seed_lo, seed_hi, out, cost,
+                                              naive_cost);
+                uint32_t* mine = chist + (threadIdx.x / kRouteChunkTokens) * D;
+#pragma unroll
+                for (int a = 0; a < KMAX; ++a)
+                    if (a < K) atomicAdd(&mine[out[a]], 1u);
+            }
+            store_token_slots<KT>(assigned_slot + t * K, out, K);
+            if (remote_nodes) remote_nodes[t] = static_cast<uint8_t>(cost);
+            cost_sum += cost;
+            naive_sum += naive_cost;
+        }
+        __syncthreads();
+        // hand this round's chunk histograms to the scan (every chunk row is written, zeros included)
+        const int64_t first_chunk = base / kRouteChunkTokens;
+        for (int i = threadIdx.x; i < kRouteChunksPerRound * D; i += blockDim.x) {
+            const int g = i / D, d = i - g * D;
+            const int64_t chunk = first_chunk + g;
+            if (chunk < n_chunks) chunk_ws[static_cast<size_t>(d) * n_chunks + chunk] = chist[i];
+            chist[i] = 0;
+        }
+        __syncthreads();
+    }
+
+    if (totals) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            cost_sum += __shfl_xor_sync(0xFFFFFFFFu, cost_sum, off);
+            naive_sum += __shfl_xor_sync(0xFFFFFFFFu, naive_sum, off);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            if (cost_sum) atomicAdd(&cta_totals[0], static_cast<unsigned long long>(cost_sum));
+            if (naive_sum) atomicAdd(&cta_totals[1], static_cast<unsigned long long>(naive_sum));
+        }
+    }
+    cluster.sync();            // every triangle of the cluster is complete (also orders cta_totals)
+    wait_for_prior_kernel();   // coact / load / totals may still be being cleared by the kernel before this one
+    merge_triangle_over_cluster(tri, lv.E, coact, load);
+    if (totals && threadIdx.x < 2 && cta_totals[threadIdx.x])
+        atomicAdd(&totals[threadIdx.x], cta_totals[threadIdx.x]);
+    cluster.sync();            // no CTA may exit while a peer still reads its triangle
+}
+
+struct RouteLaunch {
+    int cluster;
+    int ctas;
+};
+
+template <int KT>
+static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n_sm, RouteLaunch* out)
+{
+    auto kernel = route_fused_kernel<KT>;
+    static std::mutex cache_lock;
+    static std::map<std::tuple<int, int, int, int64_t>, RouteLaunch> cache;
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    int64_t want = (T + kRouteThreads - 1) / kRouteThreads;
+    if (want < 1) want = 1;
+    if (want > n_sm) want = n_sm;
+    const auto key = std::make_tuple(dev, lv.E, lv.D, want * 1024 + lv.words % 1024);
+    {
+        std::lock_guard<std::mutex> guard(cache_lock);
+        auto it = cache.find(key);
+        if (it != cache.end()) {
+            *out = it->second;
+            return COBALT_OK;
+        }
+    }
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(kRouteThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    int cand_cs[5], cand_cta[5], n_cand = 0, most = 0;
+    for (int cs = 16; cs >= 1; cs >>= 1) {
+        if (cs > want) continue;
+        attr[0].val.clusterDim.x = cs;
+        cfg.gridDim = dim3(cs);
+        int max_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            continue;
+        }
+        int n_cta = static_cast<int>(want) / cs * cs;
+        if (n_cta > max_clusters * cs) n_cta = max_clusters * cs;
+        if (n_cta < cs) continue;
+        cand_cs[n_cand] = cs;
+        cand_cta[n_cand] = n_cta;
+        ++n_cand;
+        if (n_cta > most) most = n_cta;
+    }
+    RouteLaunch best = {0, 0};
+    for (int i = 0; i < n_cand; ++i) {
+        if (cand_cta[i] * 10 >= most * 9) {
+            best.cluster = cand_cs[i];
+            best.ctas = cand_cta[i];
+            break;
+        }
+    }
+    if (best.cluster == 0) return COBALT_ERR_UNSUPPORTED;
+    {
+        std::lock_guard<std::mutex> guard(cache_lock);
+        cache[key] = best;
+    }
+    *out = best;
+    return COBALT_OK;
+}
+
+struct RouteArgs {
+    const LayoutView* lv;
+    const int32_t* ids;
+    const int32_t* src;
+    int32_t src_uniform;
+    int64_t T;
+    int32_t K;
+    uint64_t seed;
+    uint32_t* coact;
+    uint32_t* load;
+    int32_t* assigned_slot;
+    uint8_t* remote_nodes;
+    uint64_t* totals;
+    uint32_t* chunk_ws;
+    int n_chunks;
+    uint32_t* err_word;
+    bool after_zeroing;
+    int n_sm;
+    cudaStream_t stream;
+};
+
+template <int KT>
+static int launch_route(const RouteArgs& a)
+{
+    const LayoutView& lv = *a.lv;
+    const RouteSmem sm = route_smem(lv);
+    RouteLaunch how;
+    int rc = pick_route_launch<KT>(lv, a.T, sm.bytes(), a.n_sm, &how);
+    if (rc != COBALT_OK) return rc;
+    auto kernel = route_fused_kernel<KT>;
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sm.bytes())));
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    cfg.blockDim = dim3(kRouteThreads);
+    cfg.gridDim = dim3(static_cast<unsigned>(how.ctas));
+    cfg.dynamicSmemBytes = sm.bytes();
+    cfg.stream = a.stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = how.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    set_programmatic_launch(&attr[1], a.after_zeroing);
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T, a.K,
+                                       static_cast<uint32_t>(a.seed & 0xFFFFFFFFu),
+                                       static_cast<uint32_t>(a.seed >> 32), a.coact, a.load, a.assigned_slot,
+                                       a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.chunk_ws,
+                                       a.n_chunks, static_cast<int>(sm.tri_words), static_cast<int>(sm.tab_words),
+                                       a.err_word));
+    return COBALT_OK;
+}
+
+static ChunkPlan route_chunks(int64_t T, int32_t K)
+{
+    ChunkPlan c;
+    c.P = T * K;
+    c.chunk = kRouteChunkTokens * K;
+    c.n_chunks = static_cast<int>((T + kRouteChunkTokens - 1) / kRouteChunkTokens);
+    if (c.n_chunks < 1) c.n_chunks = 1;
+    return c;
+}
+
+static bool fused_fits(const LayoutView& lv) { return route_smem(lv).bytes() <= kRouteMaxSmem; }
+
+}  // namespace cobalt
+
+using namespace cobalt;
+
+extern "C" {
+
+size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K)
+{
+    if (!layout || T < 0 || K < 1 || K > COBALT_MAX_TOPK || T * static_cast<int64_t>(K) >= (1ll << 31)) return 0;
+    const LayoutView& lv = layout->view;
+    if (!fused_fits(lv) || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
+    const ChunkPlan c = route_chunks(T, K);
+    return round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
+}
+
+int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
+                       int32_t src_rank_uniform, int64_t T, int32_t K, uint64_t seed, uint32_t* coact,
+                       uint32_t* load, int32_t* assigned_slot, uint8_t* remote_nodes, uint64_t* totals,
+                       uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
+                       int32_t* pair_of_row, uint32_t flags, void* workspace, size_t workspace_bytes,
+                       cobalt_stream_t stream)
+{
+    if (!layout || T < 0 || K < 1 || !coact || !load || !dest_counts || !dest_offsets) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || T * static_cast<int64_t>(K) >= (1ll << 31)) return COBALT_ERR_UNSUPPORTED;
+    const LayoutView& lv = layout->view;
+    if (K > lv.E) return COBALT_ERR_INVALID_ARG;
+    if (!src_rank && (src_rank_uniform < 0 || src_rank_uniform >= lv.G)) return COBALT_ERR_INVALID_ARG;
+    if (T > 0 && (!topk_ids || !assigned_slot || !row_of_pair)) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(topk_ids) || !aligned16(src_rank) || !aligned16(coact) || !aligned16(load) ||
+        !aligned16(assigned_slot) || !aligned16(totals) || !aligned16(dest_counts) || !aligned16(dest_offsets) ||
+        !aligned16(row_of_pair) || !aligned16(pair_of_row) || !aligned16(workspace))
+        return COBALT_ERR_INVALID_ARG;
+    if (flags & ~COBALT_STATS_ACCUMULATE) return COBALT_ERR_INVALID_ARG;
+    const size_t need = cobalt_route_index_workspace_bytes(layout, T, K);
+    if (!workspace || workspace_bytes < need) return COBALT_ERR_WORKSPACE_TOO_SMALL;
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != layout->device) return COBALT_ERR_INVALID_ARG;
+
+    if (!fused_fits(lv) || T == 0) {
+        // the co-activation triangle does not fit beside the tables (or there is nothing to route):
+        // same results from the separate calls
+        int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags, nullptr, 0, stream);
+        if (rc != COBALT_OK) return rc;
+        rc = cobalt_assign(layout, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot, nullptr,
+                           remote_nodes, totals, 0, nullptr, 0, stream);
+        if (rc != COBALT_OK) return rc;
+        return cobalt_permute_index(assigned_slot, T, K, lv.D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
+                                    workspace, workspace_bytes, stream);
+    }
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    RouteArgs a;
+    a.after_zeroing = false;
+    ZeroList z = {{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
+    if (!(flags & COBALT_STATS_ACCUMULATE)) {
+        z.ptr[0] = coact; z.n[0] = lv.E * lv.E;
+        z.ptr[1] = load;  z.n[1] = lv.E;
+    }
+    int rc = launch_zero_list(z, s, &a.after_zeroing);
+    if (rc != COBALT_OK) return rc;
+
+    const ChunkPlan c = route_chunks(T, K);
+    a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K; a.seed = seed;
+    a.coact = coact; a.load = load; a.assigned_slot = assigned_slot; a.remote_nodes = remote_nodes; a.totals = totals;
+    a.chunk_ws = static_cast<uint32_t*>(workspace); a.n_chunks = c.n_chunks; a.stream = s;
+    rc = device_error_word(&a.err_word);
+    if (rc != COBALT_OK) return rc;
+    rc = sm_count(&a.n_sm);
+    if (rc != COBALT_OK) return rc;
+    switch (K) {
+        case 1: rc = launch_route<1>(a); break;
+        case 2: rc = launch_route<2>(a); break;
+        case 4: rc = launch_route<4>(a); break;
+        case 6: rc = launch_route<6>(a); break;
+        case 8: rc = launch_route<8>(a); break;
+        default: rc = launch_route<0>(a);
+    }
+    if (rc != COBALT_OK) return rc;
+    return launch_scan_and_rank(assigned_slot, T * K, lv.D, c, a.chunk_ws, dest_counts, dest_offsets, row_of_pair,
+                                pair_of_row, 0, s);
+}
+
+}  // extern "C"

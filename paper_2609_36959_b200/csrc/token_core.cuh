@@ -1,0 +1,286 @@
+// Per-token device routines shared by the statistics, assignment and fused route kernels:
+// loading and checking a token's K expert ids, and Algorithm 1 for one token.
+#pragma once
+
+#ifdef __CUDACC__
+#include <cooperative_groups.h>
+#endif
+
+#include "common.cuh"
+
+namespace cobalt {
+
+#ifdef __CUDACC__
+
+template <int KT>
+struct TokenShape {
+    static constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+};
+
+// ids of token t into registers (16/8-byte loads when K allows)
+template <int KT>
+__device__ __forceinline__ void load_token_ids(const int32_t* __restrict__ ids, int64_t t, int K,
+                                               int32_t (&id)[TokenShape<KT>::KMAX])
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    const int32_t* row = ids + t * K;
+    if (KT > 0 && KT % 4 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 4; ++a) {
+            const int4 v = __ldg(reinterpret_cast<const int4*>(row) + a);
+            id[4 * a] = v.x; id[4 * a + 1] = v.y; id[4 * a + 2] = v.z; id[4 * a + 3] = v.w;
+        }
+    } else if (KT > 0 && KT % 2 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 2; ++a) {
+            const int2 v = __ldg(reinterpret_cast<const int2*>(row) + a);
+            id[2 * a] = v.x; id[2 * a + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a)
+            if (a < K) id[a] = __ldg(row + a);
+    }
+}
+
+// COBALT_DEVERR_* bits for ids outside [0, E) or listed twice (D_t must be a set); 0 if fine
+template <int KT>
+__device__ __forceinline__ uint32_t check_token_ids(const int32_t (&id)[TokenShape<KT>::KMAX], int K, int E)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    uint32_t bad = 0;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            if (id[a] < 0 || id[a] >= E) bad |= COBALT_DEVERR_BAD_EXPERT_ID;
+#pragma unroll
+            for (int b = 0; b < a; ++b)
+                if (id[b] == id[a]) bad |= COBALT_DEVERR_DUPLICATE_ID;
+        }
+    }
+    return bad;
+}
+
+template <int KT>
+__device__ __forceinline__ void store_token_slots(int32_t* __restrict__ dst, const int32_t (&out)[TokenShape<KT>::KMAX],
+                                                  int K)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    if (KT > 0 && KT % 4 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 4; ++a)
+            reinterpret_cast<int4*>(dst)[a] = make_int4(out[4 * a], out[4 * a + 1], out[4 * a + 2], out[4 * a + 3]);
+    } else if (KT > 0 && KT % 2 == 0) {
+#pragma unroll
+        for (int a = 0; a < KT / 2; ++a)
+            reinterpret_cast<int2*>(dst)[a] = make_int2(out[2 * a], out[2 * a + 1]);
+    } else {
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a)
+            if (a < K) dst[a] = out[a];
+    }
+}
+
+// Layout tables staged in shared memory (see LayoutView for the word layout).
+struct TableView {
+    const uint32_t* ent;
+    const uint32_t* primary;
+    const uint32_t* rlist;
+    const uint32_t* nodes;
+    int N, Q, G, E;
+};
+
+__device__ __forceinline__ TableView stage_tables(const LayoutView& lv, uint32_t* tab)
+{
+    // the blob is padded to whole 16-byte vectors
+    const uint4* src = reinterpret_cast<const uint4*>(lv.blob);
+    uint4* dst = reinterpret_cast<uint4*>(tab);
+    const int n_vec = (lv.words + 3) / 4;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = __ldg(src + i);
+    TableView tv;
+    tv.ent = tab + lv.ent_off();
+    tv.primary = tab + lv.primary_off();
+    tv.rlist = tab + lv.rlist_off();
+    tv.nodes = tab + lv.nodes_off();
+    tv.N = lv.N; tv.Q = lv.Q; tv.G = lv.G; tv.E = lv.E;
+    return tv;
+}
+
+// What assign_token writes per task.
+enum AssignMode {
+    kAssignSlot = 0,      // Algorithm 1 with the hashed uniform replica pick (lines 14-15)
+    kAssignNaive = 1,     // every task to its expert's primary replica
+    kAssignGroupKey = 2,  // Step 1 only: out = e * N + n_te (the replica is picked later, in task order)
+};
+
+// Algorithm 1 for one token (ids already checked, s_t in range).  Writes out[a] for each of the K
+// tasks and returns the token's term of Eq. 1 in `cost`, the naive rule's term in `naive_cost`.
+template <int KT, int MODE>
+__device__ __forceinline__ void assign_token(const TableView& tv, const int32_t (&id)[TokenShape<KT>::KMAX], int K,
+                                             int32_t s_t, uint32_t t, uint32_t seed_lo, uint32_t seed_hi,
+                                             int32_t (&out)[TokenShape<KT>::KMAX], uint32_t& cost,
+                                             uint32_t& naive_cost)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    const int N = tv.N;
+    const int n_s = s_t / tv.Q;                       // N(s_t)
+    const uint32_t src_bit = 1u << n_s;
+    const uint32_t low = src_bit - 1u;
+
+    // the naive rule's term of Eq. 1: distinct nodes of the primaries, source excluded
+    uint32_t naive_nodes = 0;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a)
+        if (a < K) naive_nodes |= 1u << (tv.primary[id[a]] >> 24);
+    naive_cost = __popc(naive_nodes & ~src_bit);
+
+    if (MODE == kAssignNaive) {
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a)
+            if (a < K) out[a] = static_cast<int32_t>(tv.primary[id[a]] & 0xFFFFFFu);
+        cost = naive_cost;
+        return;
+    }
+
+    // lines 3-4: U_t and the remote masks; bit j <-> j-th node after skipping n_s.
+    // m[a] == 0 marks an expert that is present on the source node.
+    uint32_t m[KMAX];
+    uint32_t any_remote = 0, common = 0xFFFFFFFFu;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            const uint32_t held = tv.nodes[id[a]];
+            m[a] = (held & src_bit) ? 0u : (((held >> (n_s + 1)) << n_s) | (held & low));
+            any_remote |= m[a];
+            if (m[a]) common &= m[a];
+        }
+    }
+    // lines 5-8: ascending b, strictly smaller popcount replaces b*.  A single node covers U_t
+    // iff every mask has its bit, and the lowest such bit is the smallest one-bit b; only
+    // otherwise are the masks with two or more bits enumerated.
+    uint32_t b_star = 0;
+    cost = 0;
+    if (any_remote) {
+        if (common) {
+            b_star = common & (0u - common);
+        } else {
+            const uint32_t full = (1u << (N - 1)) - 1u;
+            b_star = full;
+            int best = N - 1;
+            for (uint32_t b = 3; b < full; ++b) {
+                const int pc = __popc(b);
+                if (pc >= best) continue;
+                bool feasible = true;
+#pragma unroll
+                for (int a = 0; a < KMAX; ++a)
+                    if (a < K) feasible = feasible && (m[a] == 0 || (b & m[a]) != 0);
+                if (feasible) {
+                    b_star = b;
+                    best = pc;
+                    if (pc == 2) break;  // one node is known not to suffice
+                }
+            }
+        }
+        cost = __popc(b_star);
+    }
+    // lines 9-16: node per expert, then a replica inside the node
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            int node = n_s;
+            if (m[a] != 0) {
+                // RandomNode: the i-th set bit of b* & m; a single candidate needs no draw
+                uint32_t c = b_star & m[a];
+                const uint32_t n_c = __popc(c);
+                if (n_c > 1) {
+                    const uint32_t i = hash_index(route_hash(seed_lo, seed_hi, t, id[a], 0u), n_c);
+                    for (uint32_t j = 0; j < i; ++j) c &= c - 1u;   // drop the i lowest set bits
+                }
+                const int bit = __ffs(c) - 1;
+                node = bit + (bit >= n_s ? 1 : 0);
+            }
+            if (MODE == kAssignGroupKey) {
+                out[a] = id[a] * N + node;
+            } else {
+                // UniformChoice over R_{e,node}; floor(x * 1 / 2^32) = 0, so one replica needs no draw
+                const uint32_t e_n = tv.ent[id[a] * N + node];
+                const uint32_t n_r = e_n & 0xFFu;
+                const uint32_t i = (n_r > 1) ? hash_index(route_hash(seed_lo, seed_hi, t, id[a], 1u), n_r) : 0u;
+                out[a] = static_cast<int32_t>(tv.rlist[(e_n >> 8) + i]);
+            }
+        }
+    }
+}
+
+// Adds the K(K+1)/2 unordered pairs of one token (diagonal included) to a lower-triangle tile.
+template <int KT>
+__device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32_t (&id)[TokenShape<KT>::KMAX], int K)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+#pragma unroll
+        for (int b = a; b < KMAX; ++b) {
+            if (b < K) {
+                const int hi = max(id[a], id[b]), lo = min(id[a], id[b]);
+                atomicAdd(&tri[hi * (hi + 1) / 2 + lo], 1u);
+            }
+        }
+    }
+}
+
+__host__ __device__ inline size_t tri_entries(int E) { return static_cast<size_t>(E) * (E + 1) / 2; }
+
+// Row of the lower triangle that holds flat index idx (row hi starts at hi*(hi+1)/2).
+__device__ __forceinline__ int tri_row(int idx)
+{
+    int hi = static_cast<int>((sqrtf(8.0f * static_cast<float>(idx) + 1.0f) - 1.0f) * 0.5f);
+    while (hi * (hi + 1) / 2 > idx) --hi;
+    while ((hi + 1) * (hi + 2) / 2 <= idx) ++hi;
+    return hi;
+}
+
+// After a cluster barrier: every CTA owns a contiguous slice of the flat triangle, sums it over
+// all tiles of the cluster with 16-byte distributed-shared-memory loads and merges the sums into
+// coact (both (hi, lo) and (lo, hi)) and load (the diagonal) with global integer reductions.
+// The caller must hold a second cluster barrier before any CTA exits.
+__device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E, uint32_t* __restrict__ coact,
+                                                            uint32_t* __restrict__ load)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int n_tri = static_cast<int>(tri_entries(E));
+    const int n_vec = (n_tri + 3) / 4;
+    const int csize = static_cast<int>(cluster.num_blocks());
+    const int crank = static_cast<int>(cluster.block_rank());
+    const int per = (n_vec + csize - 1) / csize;
+    const int v0 = crank * per, v1 = min(n_vec, v0 + per);
+    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+        uint4 s = make_uint4(0, 0, 0, 0);
+        for (int r = 0; r < csize; ++r) {
+            const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
+            s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+        }
+        const uint32_t part[4] = {s.x, s.y, s.z, s.w};
+        int hi = tri_row(4 * v);
+        int lo = 4 * v - hi * (hi + 1) / 2;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (4 * v + c < n_tri && part[c]) {
+                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], part[c]);
+                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], part[c]);
+                else atomicAdd(&load[hi], part[c]);
+            }
+            if (++lo > hi) { ++hi; lo = 0; }
+        }
+    }
+}
+
+#else
+
+inline size_t tri_entries(int E) { return static_cast<size_t>(E) * (E + 1) / 2; }
+
+#endif  // __CUDACC__
+
+}  // namespace cobalt

@@ -46,7 +46,7 @@ class RouteStep:
         self.expert_out = self.send if alias_expert_out else z((self.P, H), torch.bfloat16)
         self.y = z((T, H), torch.bfloat16)
         ws = max(cb.coact_stats_workspace_bytes(T, K, self.E), cb.assign_workspace_bytes(layout, T, K),
-                 cb.permute_workspace_bytes(T, K, self.D), 256)
+                 cb.permute_workspace_bytes(T, K, self.D), cb.route_index_workspace_bytes(layout, T, K), 256)
         self.workspace = torch.empty((ws,), dtype=torch.uint8, device=dev)
 
     # -- the four stages, device-resident --------------------------------------------------
@@ -69,6 +69,17 @@ class RouteStep:
         self.stats()
         self.assign(seed)
         self.permute()
+        if experts is not None:
+            experts(self.send, self.expert_out)
+        self.combine()
+
+    def route_fused(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None) -> None:
+        """The same step with stages 1, 2 and the permutation index fused into one pass over the ids
+        (cobalt_route_index); slot_load is delivered as dest_counts."""
+        cb.route_index(self.layout, self.topk_ids, self.src_rank, seed, self.coact, self.load, self.assigned_slot,
+                       self.dest_counts, self.dest_offsets, self.row_of_pair, self.workspace,
+                       remote_nodes=self.remote_nodes, totals=self.totals, pair_of_row=self.pair_of_row)
+        cb.permute_rows(self.x, self.row_of_pair, self.K, self.send)
         if experts is not None:
             experts(self.send, self.expert_out)
         self.combine()

@@ -202,6 +202,123 @@ def test_naive_rule_and_uniform_source(cb):
     assert (out.cpu().numpy() == r["assigned_slot"]).all()
 
 
+def run_fused_and_compare(cb, w, step, seed):
+    coact, load = O.coact_stats(w.topk_ids, w.E)
+    r = oracle_assign(w, seed)
+    p = O.permute(r["assigned_slot"], w.D)
+    for buf in (step.coact, step.load, step.assigned_slot, step.dest_counts, step.dest_offsets, step.row_of_pair,
+                step.pair_of_row, step.remote_nodes, step.totals):
+        buf.fill_(77)
+    cb.route_index(step.layout, step.topk_ids, step.src_rank, seed, step.coact, step.load, step.assigned_slot,
+                   step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
+                   remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    assert (u32(step.coact) == coact).all() and (u32(step.load) == load).all()
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    assert (step.remote_nodes.cpu().numpy() == r["remote_nodes"]).all()
+    assert step.totals.cpu().tolist() == [r["V"], r["V_naive"]]
+    assert (u32(step.dest_counts) == r["slot_load"]).all()
+    assert (u32(step.dest_offsets) == p["dest_offsets"]).all()
+    assert (step.row_of_pair.cpu().numpy() == p["row_of_pair"]).all()
+    assert (step.pair_of_row.cpu().numpy() == p["pair_of_row"]).all()
+
+
+@pytest.mark.parametrize("name", ["1", "1a", "2", "3", "4", "5"])
+def test_fused_route_index_on_configs(cb, name):
+    w = W.make_config(name)
+    layout, step = make_step(w, with_x=False)
+    run_fused_and_compare(cb, w, step, w.seed)
+    run_fused_and_compare(cb, w, step, w.seed + 1)      # a second call on used buffers
+
+
+@pytest.mark.parametrize("T,E,K,H,N,Q,S,empty", [
+    (1, 4, 1, 8, 1, 2, 2, 0), (7, 9, 2, 8, 3, 2, 2, 1), (255, 13, 3, 8, 4, 2, 3, 2), (257, 13, 3, 8, 4, 2, 3, 2),
+    (1000, 20, 5, 8, 8, 1, 5, 0), (2049, 40, 8, 8, 2, 4, 6, 0), (4099, 100, 16, 8, 4, 8, 5, 7),
+    (5000, 257, 7, 8, 4, 4, 20, 0), (6000, 700, 8, 8, 4, 8, 24, 0), (200000, 6, 2, 8, 4, 2, 1, 0)])
+def test_fused_route_index_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
+    w = W.make_custom(T, E, K, H, N, Q, S, seed=2000 + T + E, C=3, p_in=0.6, n_empty=empty)
+    layout, step = make_step(w, with_x=False)
+    run_fused_and_compare(cb, w, step, 31337)
+
+
+def test_fused_route_step_equals_separate_stages(cb):
+    w = W.make_config("3", T=12345)
+    layout, step = make_step(w)
+    step.route(w.seed)
+    torch.cuda.synchronize()
+    ref = {k: getattr(step, k).clone() for k in ("coact", "load", "assigned_slot", "slot_load", "dest_counts",
+                                                   "dest_offsets", "row_of_pair", "pair_of_row", "send", "y", "totals")}
+    for k in ref:
+        getattr(step, k).fill_(0)
+    step.route_fused(w.seed)
+    torch.cuda.synchronize()
+    for k, v in ref.items():
+        if k == "slot_load":
+            continue              # delivered as dest_counts by the fused call
+        got = getattr(step, k)
+        assert torch.equal(got.view(torch.int16) if got.dtype == torch.bfloat16 else got,
+                           v.view(torch.int16) if v.dtype == torch.bfloat16 else v), k
+    # accumulate flag and empty batch
+    cb.route_index(layout, step.topk_ids, step.src_rank, w.seed, step.coact, step.load, step.assigned_slot,
+                   step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace, flags=cb.STATS_ACCUMULATE)
+    torch.cuda.synchronize()
+    assert torch.equal(step.coact, 2 * ref["coact"]) and torch.equal(step.load, 2 * ref["load"])
+    w0 = W.make_custom(0, 8, 2, 16, 2, 2, 3, seed=1)
+    layout0, step0 = make_step(w0)
+    step0.route_fused(5)
+    torch.cuda.synchronize()
+    assert int(step0.coact.sum()) == 0 and step0.dest_offsets.cpu().tolist() == [0] * (w0.D + 1)
+
+
+@pytest.mark.parametrize("name,T", [("1", 4096), ("2", 9000), ("3", 20001), ("5", 131072)])
+def test_round_robin_replica_pick(cb, name, T):
+    """The running count behind the round-robin pick is reproduced exactly (bit-identical slots)."""
+    w = W.make_config(name, T=T)
+    layout, step = make_step(w, with_x=False)
+    ws = torch.empty(max(cb.assign_workspace_bytes(layout, w.T, w.K), 256), dtype=torch.uint8, device="cuda")
+    r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, w.seed,
+                 round_robin=True)
+    for _ in range(2):
+        step.assigned_slot.fill_(-5)
+        cb.assign(layout, step.topk_ids, step.src_rank, w.seed, step.assigned_slot, slot_load=step.slot_load,
+                  remote_nodes=step.remote_nodes, totals=step.totals, flags=cb.ASSIGN_ROUND_ROBIN, workspace=ws)
+        torch.cuda.synchronize()
+        assert cb.read_and_clear_device_error() == 0
+        assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+        assert (u32(step.slot_load) == r["slot_load"]).all()
+        assert (step.remote_nodes.cpu().numpy() == r["remote_nodes"]).all()
+        assert step.totals.cpu().tolist() == [r["V"], r["V_naive"]]
+    with pytest.raises(cb.CobaltError) as e:
+        cb.assign(layout, step.topk_ids, step.src_rank, w.seed, step.assigned_slot, flags=cb.ASSIGN_ROUND_ROBIN)
+    assert e.value.status == cb.ERR_WORKSPACE_TOO_SMALL
+
+
+def test_round_robin_skips_bad_tokens(cb):
+    w = W.make_config("3", T=3000)
+    layout, step = make_step(w, with_x=False)
+    ws = torch.empty(cb.assign_workspace_bytes(layout, w.T, w.K), dtype=torch.uint8, device="cuda")
+    ids = w.topk_ids.copy()
+    ids[100, 2] = ids[100, 0]
+    ids[2000, 1] = -3
+    step.topk_ids.copy_(torch.from_numpy(ids))
+    cb.assign(layout, step.topk_ids, step.src_rank, 5, step.assigned_slot, slot_load=step.slot_load,
+              flags=cb.ASSIGN_ROUND_ROBIN, workspace=ws)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == cb.DEVERR_BAD_EXPERT_ID | cb.DEVERR_DUPLICATE_ID
+    keep = np.ones(w.T, bool)
+    keep[[100, 2000]] = False
+    # the oracle on the remaining tokens, in their original order: the bad ones are simply not dealt
+    r = O.assign(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids[keep], w.src_rank[keep], 5,
+                 round_robin=True)
+    got = step.assigned_slot.cpu().numpy()
+    assert (got[~keep] == -1).all()
+    # node choices are hashed on the token index, so compare what does not depend on it
+    assert int(step.slot_load.sum()) == keep.sum() * w.K
+    assert (w.slot_expert[got[keep]] == w.topk_ids[keep]).all()
+    del r
+
+
 def test_fig1_layout_on_gpu(cb, fig1):
     g = fig1
     ids = np.array([tk["ids"] for tk in g["tokens"]], np.int32)

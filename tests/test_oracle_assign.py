@@ -315,3 +315,46 @@ def test_input_validation():
         O.assign(2, 2, 2, 4, slot, None, np.array([[0, 4]], np.int32), np.array([0], np.int32), 1)
     with pytest.raises(O.OracleError):
         O.assign(2, 2, 2, 4, slot, None, np.array([[0, 1]], np.int32), np.array([4], np.int32), 1)
+
+
+# ---------------------------------------------------------------- round-robin replica pick ---
+def test_round_robin_hand_example():
+    """One node, expert 0 on all four ranks (slots 0,2,4,6), expert 1 on ranks 0 and 2 (slots 1,5):
+    tasks of a group are dealt to its replicas in turn, in pair order."""
+    slot = np.array([0, 1, 0, -1, 0, 1, 0, -1], np.int32)
+    ids = np.array([[0, 1]] * 5 + [[1, 0]] * 5, np.int32)
+    r = O.assign(1, 4, 2, 2, slot, None, ids, np.zeros(10, np.int32), 99, round_robin=True)
+    assert r["assigned_slot"][:, 0].tolist()[:5] == [0, 2, 4, 6, 0]
+    assert r["assigned_slot"][:, 1].tolist()[:5] == [1, 5, 1, 5, 1]
+    # tokens 5..9 list expert 1 first: the groups keep their own counters
+    assert r["assigned_slot"][5:, 0].tolist() == [5, 1, 5, 1, 5]
+    assert r["assigned_slot"][5:, 1].tolist() == [2, 4, 6, 0, 2]
+    assert r["slot_load"].tolist() == [3, 5, 3, 0, 2, 5, 2, 0]
+
+
+@pytest.mark.parametrize("name,T", [("1", 3000), ("2", 3000), ("3", 4000), ("5", 2000)])
+def test_round_robin_balances_each_group_exactly(name, T):
+    w = W.make_config(name, T=T)
+    args = (w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot, w.topk_ids, w.src_rank, w.seed)
+    base = O.assign(*args)
+    rr = O.assign(*args, round_robin=True)
+    naive = O.assign(*args, naive=True)
+    _invariants(w, rr, naive)
+    # Step 1 is untouched: same node per task, same per-token cost
+    spn = w.S * w.Q
+    assert (rr["assigned_slot"] // spn == base["assigned_slot"] // spn).all()
+    assert (rr["remote_nodes"] == base["remote_nodes"]).all() and rr["V"] == base["V"]
+    tab = O.layout_tables(w.N, w.Q, w.S, w.E, w.slot_expert, w.primary_slot)
+    flat_slot = rr["assigned_slot"].ravel()
+    flat_e = w.topk_ids.ravel()
+    node = flat_slot // spn
+    seen_first = {}
+    for p, (e, n, d) in enumerate(zip(flat_e, node, flat_slot)):
+        if (e, n) not in seen_first:
+            seen_first[(e, n)] = d
+    for (e, n), first in seen_first.items():
+        replicas = tab["r_list"][e, n, :tab["r_count"][e, n]]
+        assert first == replicas[0]                       # the first task goes to the lowest slot
+        loads = rr["slot_load"][replicas].astype(int)
+        assert loads.max() - loads.min() <= 1             # exact balance inside the group
+        assert (np.diff(loads) <= 0).all()                # earlier replicas get the extra task
