@@ -259,6 +259,30 @@ def extra_measurements(args, w, step, cb, torch):
         out["index_stages_graph_replay_warm_us"] = None
         out["graph_replay_error"] = str(exc)[:200]
 
+    # the same step with stages 1, 2 and the permutation index fused into one pass over the ids
+    try:
+        n = max(5, min(args.steps, 30))
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n)]
+        for _ in range(3):
+            step.route_fused(w.seed)
+        torch.cuda.synchronize()
+        for i in range(n):
+            ev[i][0].record()
+            cb.route_index(step.layout, step.topk_ids, step.src_rank, w.seed, step.coact, step.load,
+                           step.assigned_slot, step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
+                           remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+            ev[i][1].record()
+            cb.permute_rows(step.x, step.row_of_pair, w.K, step.send)
+            step.combine()
+            ev[i][2].record()
+        torch.cuda.synchronize()
+        out["fused_route_index_us"] = sum(e[0].elapsed_time(e[1]) for e in ev) / n * 1e3
+        out["fused_step_ms"] = ev[0][0].elapsed_time(ev[-1][2]) / n
+        out["fused_step_pairs_per_s"] = w.P / (out["fused_step_ms"] * 1e-3)
+    except Exception as exc:
+        out["fused_route_index_us"] = None
+        out["fused_error"] = str(exc)[:200]
+
     # Eq. 1 under a layout that co-locates each co-activation cluster (what the paper's global
     # planner aims for), same ids: reported as context, not judged
     try:

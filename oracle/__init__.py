@@ -46,6 +46,13 @@ _lib.oracle_combine.argtypes = [_u16p, _i32p, _f32p, C.c_int64, C.c_int32, C.c_i
                                 C.c_int64, _f32p]
 
 
+_f64p = np.ctypeslib.ndpointer(np.float64, flags="C_CONTIGUOUS")
+_lib.oracle_permute_backward.restype = C.c_int
+_lib.oracle_permute_backward.argtypes = [_u16p, _i32p, C.c_int64, C.c_int32, C.c_int32, _f64p]
+_lib.oracle_combine_backward.restype = C.c_int
+_lib.oracle_combine_backward.argtypes = [_u16p, _u16p, _i32p, _f32p, C.c_int64, C.c_int32, C.c_int32, _f64p, _f64p]
+
+
 class OracleError(ValueError):
     pass
 
@@ -166,3 +173,26 @@ def combine(expert_out_bits, row_of_pair, gate_w, tokens: Optional[Sequence[int]
     y = np.zeros((n, H), np.float32)
     _check(_lib.oracle_combine(out, rop, w, T, K, H, _opt_ptr(tok), n, y), "combine")
     return y
+
+
+def permute_backward(grad_send_bits, row_of_pair, T: int, K: int) -> np.ndarray:
+    """float64 grad_x [T,H] = sum over a token's K send rows of grad_send."""
+    g = np.ascontiguousarray(grad_send_bits, dtype=np.uint16)
+    H = g.shape[1]
+    out = np.zeros((T, H), np.float64)
+    _check(_lib.oracle_permute_backward(g, _i32(row_of_pair).reshape(-1), T, K, H, out), "permute_backward")
+    return out
+
+
+def combine_backward(grad_y_bits, expert_out_bits, row_of_pair, gate_w):
+    """-> (float64 grad_expert_out [P,H], float64 grad_gate_w [T,K])."""
+    gy = np.ascontiguousarray(grad_y_bits, dtype=np.uint16)
+    out = np.ascontiguousarray(expert_out_bits, dtype=np.uint16)
+    w = np.ascontiguousarray(gate_w, dtype=np.float32)
+    T, K = w.shape
+    H = gy.shape[1]
+    grad_out = np.zeros((T * K, H), np.float64)
+    grad_w = np.zeros((T, K), np.float64)
+    _check(_lib.oracle_combine_backward(gy, out, _i32(row_of_pair).reshape(-1), w, T, K, H, grad_out, grad_w),
+           "combine_backward")
+    return grad_out, grad_w

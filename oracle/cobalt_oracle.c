@@ -394,3 +394,46 @@ int oracle_combine(const uint16_t* expert_out, const int32_t* row_of_pair, const
     }
     return ORACLE_OK;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Backward of the two row stages (the method is a training method: Section 1, "MoE training").
+ * With rows r(t,k) = row_of_pair[t*K+k], the forward maps are linear:
+ *   dispatch  send[r(t,k)] = x[t]                       combine  y[t] = sum_k g[t][k] * out[r(t,k)]
+ * so their adjoints are
+ *   grad_x[t]        = sum_k grad_send[r(t,k)]           (permute backward)
+ *   grad_out[r(t,k)] = g[t][k] * grad_y[t]               (combine backward, data)
+ *   grad_g[t][k]     = sum_h grad_y[t][h] * out[r(t,k)][h]   (combine backward, gate weights)
+ * Inputs are 16-bit bfloat patterns; results are left in double precision (no rounding), so
+ * that tolerances against them measure the CUDA path alone.
+ * ---------------------------------------------------------------------------------------- */
+int oracle_permute_backward(const uint16_t* grad_send, const int32_t* row_of_pair, int64_t T, int32_t K,
+                            int32_t H, double* grad_x)
+{
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int32_t k = 0; k < K; ++k)
+                acc += (double)f32_from_bf16(grad_send[(size_t)row_of_pair[t * K + k] * H + h]);
+            grad_x[(size_t)t * H + h] = acc;
+        }
+    return ORACLE_OK;
+}
+
+int oracle_combine_backward(const uint16_t* grad_y, const uint16_t* expert_out, const int32_t* row_of_pair,
+                            const float* gate_w, int64_t T, int32_t K, int32_t H, double* grad_out,
+                            double* grad_gate_w)
+{
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t k = 0; k < K; ++k) {
+            size_t row = (size_t)row_of_pair[t * K + k];
+            double g = (double)gate_w[t * K + k];
+            double dot = 0.0;
+            for (int32_t h = 0; h < H; ++h) {
+                double gy = (double)f32_from_bf16(grad_y[(size_t)t * H + h]);
+                grad_out[row * H + h] = g * gy;
+                dot += gy * (double)f32_from_bf16(expert_out[row * H + h]);
+            }
+            grad_gate_w[t * K + k] = dot;
+        }
+    return ORACLE_OK;
+}
