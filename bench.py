@@ -283,6 +283,23 @@ def extra_measurements(args, w, step, cb, torch):
         out["fused_route_index_us"] = None
         out["fused_error"] = str(exc)[:200]
 
+    # backward of the two row stages (adjoints), same buffers: grad_send := send, grad_y := y
+    try:
+        peak, _ = hbm_peak()
+        grad_x = torch.empty_like(step.x)
+        grad_out = torch.empty_like(step.send)
+        grad_w = torch.empty_like(step.gate_w)
+        T, K, H, P = w.T, w.K, w.H, w.P
+        ms = timed(lambda: cb.permute_backward(step.send, step.row_of_pair, K, grad_x), 10)
+        b = 2 * P * H + 2 * T * H + 4 * P
+        out["permute_backward"] = {"ms": ms, "bytes": b, "gbs": b / ms / 1e6, "frac": b / ms / 1e6 / peak}
+        ms = timed(lambda: cb.combine_backward(step.y, step.send, step.row_of_pair, step.gate_w, grad_out, grad_w), 10)
+        b = 2 * T * H + 4 * P * H + 12 * P
+        out["combine_backward"] = {"ms": ms, "bytes": b, "gbs": b / ms / 1e6, "frac": b / ms / 1e6 / peak}
+        del grad_x, grad_out, grad_w
+    except Exception as exc:
+        out["backward_error"] = str(exc)[:200]
+
     # Eq. 1 under a layout that co-locates each co-activation cluster (what the paper's global
     # planner aims for), same ids: reported as context, not judged
     try:

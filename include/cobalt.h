@@ -222,6 +222,23 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
                          int64_t T, int32_t K, int32_t H, void* y, int64_t total_rows,
                          uint32_t flags, cobalt_stream_t stream);
 
+/* ---- backward of the two row stages (the method is used in training: Section 1) --------------
+ * The forward maps are linear, send[r(t,k)] = x[t] and y[t] = sum_k g[t][k] * out[r(t,k)] with
+ * r(t,k) = row_of_pair[t*K+k]; these are their adjoints.
+ * cobalt_permute_backward: grad_x[t] = bf16( sum_k float(grad_send[r(t,k)]) ), fp32 accumulation in
+ *   ascending k.  grad_send bf16 [P, H], grad_x bf16 [T, H].
+ * cobalt_combine_backward: grad_expert_out[r(t,k)] = bf16( g[t][k] * float(grad_y[t]) ) and
+ *   grad_gate_w[t*K+k] = sum_h float(grad_y[t][h]) * float(expert_out[r(t,k)][h]) in fp32 (a fixed
+ *   reduction tree: results do not vary from run to run).  Either output may be NULL (expert_out
+ *   is only read for grad_gate_w).  grad_y bf16 [T, H], grad_expert_out bf16 [P, H], grad_gate_w
+ *   fp32 [P]. */
+int cobalt_permute_backward(const void* grad_send, const int32_t* row_of_pair, int64_t T, int32_t K,
+                            int32_t H, void* grad_x, uint32_t flags, cobalt_stream_t stream);
+int cobalt_combine_backward(const void* grad_y, const void* expert_out, const int32_t* row_of_pair,
+                            const float* gate_w, int64_t T, int32_t K, int32_t H,
+                            void* grad_expert_out, float* grad_gate_w, uint32_t flags,
+                            cobalt_stream_t stream);
+
 /* ---- device error word -------------------------------------------------------------------
  * Waits for `stream`, copies the COBALT_DEVERR_* bits set by kernels on the current device
  * since the last call into *out_bits_host and clears them. */

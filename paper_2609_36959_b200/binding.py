@@ -46,6 +46,7 @@ EXPORTS = (
     "cobalt_permute_workspace_bytes", "cobalt_permute_index", "cobalt_permute_rows", "cobalt_permute",
     "cobalt_permute_index_static", "cobalt_permute_rows_block", "cobalt_combine_block",
     "cobalt_route_index_workspace_bytes", "cobalt_route_index",
+    "cobalt_permute_backward", "cobalt_combine_backward",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -84,6 +85,8 @@ def _load() -> C.CDLL:
         "cobalt_route_index_workspace_bytes": (sz, [vp, i64, i32]),
         "cobalt_route_index": (C.c_int, [vp, vp, vp, i32, i64, i32, u64, vp, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp,
                                          sz, vp]),
+        "cobalt_permute_backward": (C.c_int, [vp, vp, i64, i32, i32, vp, u32, vp]),
+        "cobalt_combine_backward": (C.c_int, [vp, vp, vp, vp, i64, i32, i32, vp, vp, u32, vp]),
         "cobalt_permute_rows_block": (C.c_int, [vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_combine_block": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_read_and_clear_device_error": (C.c_int, [C.POINTER(u32), vp]),
@@ -377,6 +380,39 @@ def combine_block(expert_out: torch.Tensor, row_of_pair_block: torch.Tensor, gat
     _check(_lib.cobalt_combine_block(expert_out.data_ptr(), _ptr(row_of_pair_block, torch.int32, "row_of_pair"),
                                      _elem_ptr(gate_w, t0 * K), t1 - t0, K, H, _elem_ptr(y, t0 * H), T * K, flags,
                                      _stream()), "cobalt_combine_block")
+
+
+def permute_backward(grad_send: torch.Tensor, row_of_pair: torch.Tensor, K: int, grad_x: torch.Tensor, *,
+                     flags: int = 0) -> None:
+    """grad_x[t] = sum of the K rows of grad_send that token t was sent to."""
+    T, H = grad_x.shape
+    if row_of_pair.numel() != T * K or grad_send.numel() != T * K * H:
+        raise CobaltError(ERR_INVALID_ARG, "permute_backward (sizes)")
+    _check(_lib.cobalt_permute_backward(_ptr(grad_send, torch.bfloat16, "grad_send"),
+                                        _ptr(row_of_pair, torch.int32, "row_of_pair"), T, K, H,
+                                        _ptr(grad_x, torch.bfloat16, "grad_x"), flags, _stream()),
+           "cobalt_permute_backward")
+
+
+def combine_backward(grad_y: torch.Tensor, expert_out: Optional[torch.Tensor], row_of_pair: torch.Tensor,
+                     gate_w: torch.Tensor, grad_expert_out: Optional[torch.Tensor],
+                     grad_gate_w: Optional[torch.Tensor], *, flags: int = 0) -> None:
+    T, K = gate_w.shape
+    H = grad_y.shape[1]
+    if grad_y.shape[0] != T or row_of_pair.numel() != T * K:
+        raise CobaltError(ERR_INVALID_ARG, "combine_backward (sizes)")
+    for name, t in (("expert_out", expert_out), ("grad_expert_out", grad_expert_out)):
+        if t is not None and t.numel() != T * K * H:
+            raise CobaltError(ERR_INVALID_ARG, f"combine_backward ({name} size)")
+    if grad_gate_w is not None and grad_gate_w.numel() != T * K:
+        raise CobaltError(ERR_INVALID_ARG, "combine_backward (grad_gate_w size)")
+    _check(_lib.cobalt_combine_backward(_ptr(grad_y, torch.bfloat16, "grad_y"),
+                                        _ptr(expert_out, torch.bfloat16, "expert_out"),
+                                        _ptr(row_of_pair, torch.int32, "row_of_pair"),
+                                        _ptr(gate_w, torch.float32, "gate_w"), T, K, H,
+                                        _ptr(grad_expert_out, torch.bfloat16, "grad_expert_out"),
+                                        _ptr(grad_gate_w, torch.float32, "grad_gate_w"), flags, _stream()),
+           "cobalt_combine_backward")
 
 
 def read_and_clear_device_error() -> int:

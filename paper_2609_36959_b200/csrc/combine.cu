@@ -26,7 +26,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-template <int KT>
+// kUnit: no gate weights, the plain sum of the K rows (the adjoint of the dispatch gather).
+template <int KT, bool kUnit>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const uint4* __restrict__ out, const int32_t* __restrict__ row_of_pair,
                const float* __restrict__ gate_w, int64_t T, int K_rt, int n_vec, int64_t P,
@@ -43,7 +44,7 @@ combine_kernel(const uint4* __restrict__ out, const int32_t* __restrict__ row_of
                 const int32_t r = __ldg(row_of_pair + t * K + k);
                 const bool valid = (r >= 0 && r < P);
                 row[k] = valid ? static_cast<int64_t>(r) * n_vec : -1;
-                w[k] = valid ? __ldg(gate_w + t * K + k) : 0.0f;
+                w[k] = valid ? (kUnit ? 1.0f : __ldg(gate_w + t * K + k)) : 0.0f;
                 if (!valid && threadIdx.x == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
             }
         }
@@ -72,6 +73,97 @@ combine_kernel(const uint4* __restrict__ out, const int32_t* __restrict__ row_of
     }
 }
 
+// Backward of the combine for one token per CTA: grad_out[r(t,k)] = g[t][k] * grad_y[t] (bf16, one
+// rounding) and grad_g[t][k] = <grad_y[t], out[r(t,k)]> (fp32; per-thread partial sums, then a fixed
+// warp-shuffle tree and a fixed-order sum over the warps, so the result does not depend on timing).
+template <int KT>
+__global__ void __launch_bounds__(kCombineThreads)
+combine_backward_kernel(const uint4* __restrict__ grad_y, const uint4* __restrict__ out,
+                        const int32_t* __restrict__ row_of_pair, const float* __restrict__ gate_w, int64_t T,
+                        int K_rt, int n_vec, int64_t P, uint4* __restrict__ grad_out, float* __restrict__ grad_w,
+                        uint32_t* __restrict__ err_word)
+{
+    constexpr int KMAX = (KT > 0) ? KT : COBALT_MAX_TOPK;
+    constexpr int kWarps = kCombineThreads / 32;
+    const int K = (KT > 0) ? KT : K_rt;
+    __shared__ float partial[kWarps][KMAX];
+    const int64_t t = blockIdx.x;
+    if (t >= T) return;
+
+    int64_t row[KMAX];
+    float w[KMAX], dot[KMAX];
+#pragma unroll
+    for (int k = 0; k < KMAX; ++k) {
+        dot[k] = 0.0f;
+        if (k < K) {
+            const int32_t r = __ldg(row_of_pair + t * K + k);
+            const bool valid = (r >= 0 && r < P);
+            row[k] = valid ? static_cast<int64_t>(r) * n_vec : -1;
+            w[k] = __ldg(gate_w + t * K + k);
+            if (!valid && threadIdx.x == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+        }
+    }
+    for (int v = threadIdx.x; v < n_vec; v += blockDim.x) {
+        const uint4 g = ld_stream16(grad_y + t * n_vec + v);
+        const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+        float gf[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            gf[2 * i] = __uint_as_float(gw[i] << 16);
+            gf[2 * i + 1] = __uint_as_float(gw[i] & 0xFFFF0000u);
+        }
+        if (grad_w) {
+            uint4 val[KMAX];
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k)
+                if (k < K) val[k] = (row[k] >= 0) ? ld_stream16(out + row[k] + v) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) {
+                if (k < K) {
+                    const uint32_t ow[4] = {val[k].x, val[k].y, val[k].z, val[k].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        dot[k] = fmaf(gf[2 * i], __uint_as_float(ow[i] << 16), dot[k]);
+                        dot[k] = fmaf(gf[2 * i + 1], __uint_as_float(ow[i] & 0xFFFF0000u), dot[k]);
+                    }
+                }
+            }
+        }
+        if (grad_out) {
+#pragma unroll
+            for (int k = 0; k < KMAX; ++k) {
+                if (k < K && row[k] >= 0) {
+                    uint4 o;
+                    o.x = pack_bf16x2(w[k] * gf[0], w[k] * gf[1]);
+                    o.y = pack_bf16x2(w[k] * gf[2], w[k] * gf[3]);
+                    o.z = pack_bf16x2(w[k] * gf[4], w[k] * gf[5]);
+                    o.w = pack_bf16x2(w[k] * gf[6], w[k] * gf[7]);
+                    st_stream16(grad_out + row[k] + v, o);
+                }
+            }
+        }
+    }
+    if (grad_w) {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+        for (int k = 0; k < KMAX; ++k) {
+            if (k < K) {
+                float d = dot[k];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xFFFFFFFFu, d, off);
+                if (lane == 0) partial[warp][k] = d;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < K) {
+            float d = 0.0f;
+#pragma unroll
+            for (int wi = 0; wi < kWarps; ++wi) d += partial[wi][threadIdx.x];
+            grad_w[t * K + threadIdx.x] = d;
+        }
+    }
+}
+
 }  // namespace cobalt
 
 using namespace cobalt;
@@ -87,7 +179,8 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
         total_rows >= (1ll << 31))
         return COBALT_ERR_UNSUPPORTED;
     if (T == 0) return COBALT_OK;
-    if (!expert_out || !row_of_pair || !gate_w || !y) return COBALT_ERR_INVALID_ARG;
+    // gate_w == NULL means unit weights (the plain sum of the K rows), used by cobalt_permute_backward
+    if (!expert_out || !row_of_pair || !y) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(expert_out) || !aligned16(y) || !aligned16(row_of_pair) || !aligned16(gate_w))
         return COBALT_ERR_INVALID_ARG;
     const uint32_t impl = flags & COBALT_IMPL_MASK;
@@ -111,7 +204,12 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
     uint4* dst = static_cast<uint4*>(y);
 #define COBALT_COMBINE_CASE(KT)                                                                         \
     case KT:                                                                                            \
-        combine_kernel<KT><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, err_word); \
+        if (gate_w)                                                                                     \
+            combine_kernel<KT, false><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, \
+                                                                       err_word);                       \
+        else                                                                                            \
+            combine_kernel<KT, true><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,  \
+                                                                      err_word);                        \
         break
     switch (K) {
         COBALT_COMBINE_CASE(1);
@@ -120,7 +218,12 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
         COBALT_COMBINE_CASE(6);
         COBALT_COMBINE_CASE(8);
         default:
-            combine_kernel<0><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, err_word);
+            if (gate_w)
+                combine_kernel<0, false><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
+                                                                          err_word);
+            else
+                combine_kernel<0, true><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
+                                                                         err_word);
     }
 #undef COBALT_COMBINE_CASE
     COBALT_CUDA_TRY(cudaGetLastError());
@@ -133,6 +236,58 @@ int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const flo
     if (T < 0 || K < 1) return COBALT_ERR_INVALID_ARG;
     return cobalt_combine_block(expert_out, row_of_pair, gate_w, T, K, H, y, T * static_cast<int64_t>(K), flags,
                                 stream);
+}
+
+int cobalt_permute_backward(const void* grad_send, const int32_t* row_of_pair, int64_t T, int32_t K, int32_t H,
+                            void* grad_x, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1) return COBALT_ERR_INVALID_ARG;
+    // the adjoint of the gather is the sum of the token's K rows: the combine with unit weights
+    return cobalt_combine_block(grad_send, row_of_pair, nullptr, T, K, H, grad_x, T * static_cast<int64_t>(K), flags,
+                                stream);
+}
+
+int cobalt_combine_backward(const void* grad_y, const void* expert_out, const int32_t* row_of_pair,
+                            const float* gate_w, int64_t T, int32_t K, int32_t H, void* grad_expert_out,
+                            float* grad_gate_w, uint32_t flags, cobalt_stream_t stream)
+{
+    if (T < 0 || K < 1 || H < 1) return COBALT_ERR_INVALID_ARG;
+    if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31)) return COBALT_ERR_UNSUPPORTED;
+    if ((flags & COBALT_IMPL_MASK) != 0 && (flags & COBALT_IMPL_MASK) != COBALT_IMPL_VECTOR) return COBALT_ERR_INVALID_ARG;
+    if (!grad_expert_out && !grad_gate_w) return COBALT_ERR_INVALID_ARG;
+    if (T == 0) return COBALT_OK;
+    if (!grad_y || !row_of_pair || !gate_w || (grad_gate_w && !expert_out)) return COBALT_ERR_INVALID_ARG;
+    if (!aligned16(grad_y) || !aligned16(expert_out) || !aligned16(row_of_pair) || !aligned16(gate_w) ||
+        !aligned16(grad_expert_out) || !aligned16(grad_gate_w))
+        return COBALT_ERR_INVALID_ARG;
+    uint32_t* err_word = nullptr;
+    int rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n_vec = H / 8;
+    const int64_t P = T * K;
+    const unsigned grid = static_cast<unsigned>(T);
+    const uint4* gy = static_cast<const uint4*>(grad_y);
+    const uint4* out = static_cast<const uint4*>(expert_out);
+    uint4* go = static_cast<uint4*>(grad_expert_out);
+#define COBALT_CBWD_CASE(KT)                                                                                   \
+    case KT:                                                                                                   \
+        combine_backward_kernel<KT><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go, \
+                                                                     grad_gate_w, err_word);                   \
+        break
+    switch (K) {
+        COBALT_CBWD_CASE(1);
+        COBALT_CBWD_CASE(2);
+        COBALT_CBWD_CASE(4);
+        COBALT_CBWD_CASE(6);
+        COBALT_CBWD_CASE(8);
+        default:
+            combine_backward_kernel<0><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go,
+                                                                        grad_gate_w, err_word);
+    }
+#undef COBALT_CBWD_CASE
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
 }
 
 }  // extern "C"
