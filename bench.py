@@ -214,6 +214,7 @@ def whole_job_value(world: int, pairs_per_rank: int, ms_per_step: float) -> floa
 # traffic model on a layout whose co-activation clusters share a node
 # ---------------------------------------------------------------------------------------------
 def extra_measurements(args, w, step, cb, torch):
+    import numpy as np
     out = {}
 
     def timed(fn, n, warm=3):
@@ -299,6 +300,22 @@ def extra_measurements(args, w, step, cb, torch):
         del grad_x, grad_out, grad_w
     except Exception as exc:
         out["backward_error"] = str(exc)[:200]
+
+    # Stage 2 of the planner closed on one box: this step's w_er -> greedy intra-node rebalancing ->
+    # the same tokens assigned over the new layout (rank-load imbalance = max / mean, as in the paper)
+    try:
+        load = step.slot_load.cpu().numpy().astype(np.float32)
+        new_layout, moved, kept = cb.rebalance_intra_node(w.N, w.Q, w.S, w.E, w.slot_expert.tolist(), load.tolist())
+        lay2 = cb.Layout(w.N, w.Q, w.S, w.E, new_layout)
+        slots2 = torch.zeros_like(step.assigned_slot)
+        load2 = torch.zeros_like(step.slot_load)
+        cb.assign(lay2, step.topk_ids, step.src_rank, w.seed, slots2, slot_load=load2)
+        before = load.reshape(w.G, w.S).sum(axis=1)
+        after = load2.cpu().numpy().astype(np.float64).reshape(w.G, w.S).sum(axis=1)
+        out["stage2_rebalance"] = {"imbalance_before": float(before.max() / before.mean()),
+                                   "imbalance_after": float(after.max() / after.mean()), "nodes_kept": kept}
+    except Exception as exc:
+        out["stage2_rebalance"] = {"error": str(exc)[:200]}
 
     # Eq. 1 under a layout that co-locates each co-activation cluster (what the paper's global
     # planner aims for), same ids: reported as context, not judged

@@ -239,6 +239,29 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
                             void* grad_expert_out, float* grad_gate_w, uint32_t flags,
                             cobalt_stream_t stream);
 
+/* ---- statistics epilogue and Stage 2 of the layout planner (Section 3.2) ---------------------
+ * cobalt_ema_update: ema[i] = decay * ema[i] + (1 - decay) * counts[i] for n entries (device arrays;
+ *   counts uint32, ema fp32), the moving averages w^_e, c^_ij and w_er the planner reads.  The paper
+ *   gives no decay constant: it is the caller's.  COBALT_EMA_INITIALISE sets ema = counts instead.
+ * cobalt_ochiai: ochiai[i*E+j] = coact[i*E+j] / sqrt(coact[i*E+i] * coact[j*E+j]), 0 where either
+ *   expert was never selected (the similarity of Section 1's footnote).  fp32 [E*E] on the device.
+ * cobalt_rebalance_intra_node (host arrays only, no device work): per node, re-partitions the
+ *   replicas among the node's ranks by greedy bin packing on slot_load_host (fp32 [G*S], the EMA of
+ *   w_er): longest first (ties: lower expert id, then lower old slot), each to the least-loaded
+ *   rank of its node that has a free slot and does not hold that expert yet (ties: lower rank);
+ *   slots of a rank fill in placement order.  A node where some replica finds no admissible rank
+ *   keeps its placement.  Outputs: new_slot_expert_host [G*S]; moved_from_host [G*S] (old slot
+ *   of every new slot, -1 for empty; may be NULL); *nodes_kept_host (may be NULL).  Replicas never
+ *   leave their node, so no cross-node parameter movement is implied. */
+#define COBALT_EMA_INITIALISE 0x1u
+int cobalt_ema_update(const uint32_t* counts, float* ema, int64_t n, float decay, uint32_t flags,
+                      cobalt_stream_t stream);
+int cobalt_ochiai(const uint32_t* coact, int32_t E, float* ochiai, cobalt_stream_t stream);
+int cobalt_rebalance_intra_node(int32_t num_nodes, int32_t ranks_per_node, int32_t slots_per_rank,
+                                int32_t num_experts, const int32_t* slot_expert_host,
+                                const float* slot_load_host, int32_t* new_slot_expert_host,
+                                int32_t* moved_from_host, int32_t* nodes_kept_host);
+
 /* ---- device error word -------------------------------------------------------------------
  * Waits for `stream`, copies the COBALT_DEVERR_* bits set by kernels on the current device
  * since the last call into *out_bits_host and clears them. */

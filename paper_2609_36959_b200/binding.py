@@ -33,6 +33,7 @@ DEVERR_WAIT_TIMEOUT = 0x10
 STATS_ACCUMULATE = 0x1
 ASSIGN_NAIVE = 0x1
 ASSIGN_ROUND_ROBIN = 0x2
+EMA_INITIALISE = 0x1
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200
 IMPL_BULK_RING = 0x300
@@ -47,6 +48,7 @@ EXPORTS = (
     "cobalt_permute_index_static", "cobalt_permute_rows_block", "cobalt_combine_block",
     "cobalt_route_index_workspace_bytes", "cobalt_route_index",
     "cobalt_permute_backward", "cobalt_combine_backward",
+    "cobalt_ema_update", "cobalt_ochiai", "cobalt_rebalance_intra_node",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -87,6 +89,9 @@ def _load() -> C.CDLL:
                                          sz, vp]),
         "cobalt_permute_backward": (C.c_int, [vp, vp, i64, i32, i32, vp, u32, vp]),
         "cobalt_combine_backward": (C.c_int, [vp, vp, vp, vp, i64, i32, i32, vp, vp, u32, vp]),
+        "cobalt_ema_update": (C.c_int, [vp, vp, i64, C.c_float, u32, vp]),
+        "cobalt_ochiai": (C.c_int, [vp, i32, vp, vp]),
+        "cobalt_rebalance_intra_node": (C.c_int, [i32, i32, i32, i32, vp, vp, vp, vp, vp]),
         "cobalt_permute_rows_block": (C.c_int, [vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_combine_block": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_read_and_clear_device_error": (C.c_int, [C.POINTER(u32), vp]),
@@ -413,6 +418,37 @@ def combine_backward(grad_y: torch.Tensor, expert_out: Optional[torch.Tensor], r
                                         _ptr(grad_expert_out, torch.bfloat16, "grad_expert_out"),
                                         _ptr(grad_gate_w, torch.float32, "grad_gate_w"), flags, _stream()),
            "cobalt_combine_backward")
+
+
+def ema_update(counts: torch.Tensor, ema: torch.Tensor, decay: float, *, flags: int = 0) -> None:
+    """ema = decay * ema + (1 - decay) * counts, element-wise on the device (counts int32, ema float32)."""
+    if counts.numel() != ema.numel():
+        raise CobaltError(ERR_INVALID_ARG, "ema_update (sizes)")
+    _check(_lib.cobalt_ema_update(_ptr(counts, torch.int32, "counts"), _ptr(ema, torch.float32, "ema"),
+                                  counts.numel(), decay, flags, _stream()), "cobalt_ema_update")
+
+
+def ochiai(coact: torch.Tensor, out: torch.Tensor) -> None:
+    E = coact.shape[0]
+    if coact.numel() != E * E or out.numel() != E * E:
+        raise CobaltError(ERR_INVALID_ARG, "ochiai (sizes)")
+    _check(_lib.cobalt_ochiai(_ptr(coact, torch.int32, "coact"), E, _ptr(out, torch.float32, "ochiai"), _stream()),
+           "cobalt_ochiai")
+
+
+def rebalance_intra_node(N: int, Q: int, S: int, E: int, slot_expert, slot_load):
+    """Stage-2 greedy rebalancing on host arrays -> (new_slot_expert, moved_from, nodes_kept) as Python lists/int."""
+    D = N * Q * S
+    se = _host_i32(slot_expert)
+    ld = (C.c_float * D)(*[float(v) for v in slot_load])
+    if len(se) != D:
+        raise CobaltError(ERR_INVALID_ARG, "rebalance_intra_node (slot_expert size)")
+    new = (C.c_int32 * D)()
+    moved = (C.c_int32 * D)()
+    kept = C.c_int32(0)
+    _check(_lib.cobalt_rebalance_intra_node(N, Q, S, E, se, ld, new, moved, C.byref(kept)),
+           "cobalt_rebalance_intra_node")
+    return list(new), list(moved), int(kept.value)
 
 
 def read_and_clear_device_error() -> int:

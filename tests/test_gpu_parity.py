@@ -319,6 +319,27 @@ def test_round_robin_skips_bad_tokens(cb):
     del r
 
 
+def test_ema_and_ochiai(cb):
+    w = W.make_config("5", T=20000)
+    layout, step = make_step(w, with_x=False)
+    step.stats()
+    och = torch.zeros((w.E, w.E), dtype=torch.float32, device="cuda")
+    cb.ochiai(step.coact, och)
+    ema = torch.zeros((w.E, w.E), dtype=torch.float32, device="cuda")
+    cb.ema_update(step.coact, ema, 0.9, flags=cb.EMA_INITIALISE)
+    for _ in range(3):
+        cb.ema_update(step.coact, ema, 0.9)
+    ema2 = torch.full((w.E,), 5.0, dtype=torch.float32, device="cuda")
+    cb.ema_update(step.load, ema2, 0.75)
+    torch.cuda.synchronize()
+    coact, load = O.coact_stats(w.topk_ids, w.E)
+    assert np.allclose(och.cpu().numpy(), O.ochiai(coact), rtol=2e-6, atol=1e-7)
+    assert np.allclose(ema.cpu().numpy(), coact, rtol=1e-6)            # an EMA of a constant stays there
+    assert np.allclose(ema2.cpu().numpy(), O.ema_update(np.full(w.E, 5.0), load, 0.75), rtol=1e-6)
+    with pytest.raises(cb.CobaltError):
+        cb.ema_update(step.load, ema2, 1.5)
+
+
 def test_fig1_layout_on_gpu(cb, fig1):
     g = fig1
     ids = np.array([tk["ids"] for tk in g["tokens"]], np.int32)
