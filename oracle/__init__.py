@@ -14,6 +14,7 @@ import numpy as np
 
 from . import build as _build
 from .bruteforce import min_remote_nodes_bruteforce  # noqa: F401
+from .dedup import dedup_index, dedup_rows, forward_rows  # noqa: F401
 from .epilogue import ema_update, ochiai, rebalance_intra_node  # noqa: F401
 
 _lib = C.CDLL(_build.build())
