@@ -301,6 +301,39 @@ def extra_measurements(args, w, step, cb, torch):
     except Exception as exc:
         out["backward_error"] = str(exc)[:200]
 
+    # node-deduplicated send layout: one row per (token, destination node) instead of per pair
+    try:
+        peak, _ = hbm_peak()
+        T, K, H, P, N = w.T, w.K, w.H, w.P, w.N
+        node_counts = torch.zeros(N, dtype=torch.int32, device="cuda")
+        node_offsets = torch.zeros(N + 1, dtype=torch.int32, device="cuda")
+        node_row = torch.zeros(T * N, dtype=torch.int32, device="cuda")
+        fwd = torch.zeros(P, dtype=torch.int32, device="cuda")
+        cross = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ws = torch.empty(cb.dedup_workspace_bytes(T, K, N), dtype=torch.uint8, device="cuda")
+
+        def index():
+            cb.dedup_index(step.assigned_slot, step.src_rank, N, w.Q, w.S, node_counts, node_offsets, node_row, fwd, ws,
+                           cross_node_rows=cross)
+        ms_index = timed(index, 20)
+        rows = int(node_offsets[-1])
+        dedup_send = torch.empty((rows, H), dtype=torch.bfloat16, device="cuda")
+        ms_rows = timed(lambda: cb.dedup_rows(step.x, node_row, N, dedup_send), 10)
+        recv = torch.empty_like(step.send)
+        ms_fwd = timed(lambda: cb.forward_rows(dedup_send, fwd, step.row_of_pair, recv), 10)
+        b_rows = 2 * T * H + 2 * rows * H + 4 * T * N
+        b_fwd = 2 * rows * H + 2 * P * H + 8 * P      # every buffer row read once, every pair row written
+        out["dedup_layout"] = {
+            "n_rows": rows, "pairs": P, "rows_per_pair": rows / P, "cross_node_rows": int(cross[0]),
+            "buffer_bytes": rows * H * 2, "plain_buffer_bytes": P * H * 2, "bytes_saved_frac": 1 - rows / P,
+            "index_us": ms_index * 1e3,
+            "fill": {"ms": ms_rows, "gbs": b_rows / ms_rows / 1e6, "frac": b_rows / ms_rows / 1e6 / peak},
+            "forward": {"ms": ms_fwd, "gbs": b_fwd / ms_fwd / 1e6, "frac": b_fwd / ms_fwd / 1e6 / peak},
+            "recv_equals_send": bool(torch.equal(recv.view(torch.int16), step.send.view(torch.int16)))}
+        del dedup_send, recv
+    except Exception as exc:
+        out["dedup_layout"] = {"error": str(exc)[:200]}
+
     # Stage 2 of the planner closed on one box: this step's w_er -> greedy intra-node rebalancing ->
     # the same tokens assigned over the new layout (rank-load imbalance = max / mean, as in the paper)
     try:

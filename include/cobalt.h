@@ -262,6 +262,32 @@ int cobalt_rebalance_intra_node(int32_t num_nodes, int32_t ranks_per_node, int32
                                 const float* slot_load_host, int32_t* new_slot_expert_host,
                                 int32_t* moved_from_host, int32_t* nodes_kept_host);
 
+/* ---- node-deduplicated send layout (Section 3.1, Eq. 1; Section 1 on node-level dedup) -------
+ * When ranks of one node need the same token it crosses the network once and is forwarded inside
+ * the node; Eq. 1 counts exactly those crossings.  cobalt_dedup_index lays the send buffer out
+ * accordingly: ONE row per (token, destination node), grouped by destination node in ascending
+ * token order.
+ *   node_counts[n]              rows for node n                                uint32 [N]
+ *   node_offsets                exclusive scan, last = total rows              uint32 [N+1]
+ *   node_row_of_token[t*N+n]    row of token t in node n's group, -1 if none   int32 [T*N]
+ *   fwd_src_row[p]              row pair p is forwarded from on arrival        int32 [P]
+ *   cross_node_rows[0]          rows whose node differs from the source node = V of Eq. 1
+ *                               (uint64 [1]; may be NULL)
+ * Fill the buffer with cobalt_permute_rows_block(x, node_row_of_token, T, N, H, dedup_send,
+ * capacity_rows, ...) (N "copies" per token, absent nodes skipped; T*min(K,N) rows always
+ * suffice).  cobalt_forward_rows is the receiving side's expansion,
+ * recv[row_of_pair[p]] = dedup_send[fwd_src_row[p]], which reproduces the buffer of
+ * cobalt_permute bit for bit.  src_rows / dst_rows bound the two index arrays. */
+size_t cobalt_dedup_workspace_bytes(int64_t T, int32_t K, int32_t num_nodes);
+int cobalt_dedup_index(const int32_t* assigned_slot, const int32_t* src_rank, int32_t src_rank_uniform,
+                       int64_t T, int32_t K, int32_t num_nodes, int32_t ranks_per_node,
+                       int32_t slots_per_rank, uint32_t* node_counts, uint32_t* node_offsets,
+                       int32_t* node_row_of_token, int32_t* fwd_src_row, uint64_t* cross_node_rows,
+                       void* workspace, size_t workspace_bytes, cobalt_stream_t stream);
+int cobalt_forward_rows(const void* dedup_send, const int32_t* fwd_src_row, const int32_t* row_of_pair,
+                        int64_t P, int32_t H, void* recv, int64_t src_rows, int64_t dst_rows,
+                        cobalt_stream_t stream);
+
 /* ---- device error word -------------------------------------------------------------------
  * Waits for `stream`, copies the COBALT_DEVERR_* bits set by kernels on the current device
  * since the last call into *out_bits_host and clears them. */

@@ -49,6 +49,7 @@ EXPORTS = (
     "cobalt_route_index_workspace_bytes", "cobalt_route_index",
     "cobalt_permute_backward", "cobalt_combine_backward",
     "cobalt_ema_update", "cobalt_ochiai", "cobalt_rebalance_intra_node",
+    "cobalt_dedup_workspace_bytes", "cobalt_dedup_index", "cobalt_forward_rows",
     "cobalt_combine", "cobalt_read_and_clear_device_error",
 )
 
@@ -92,6 +93,9 @@ def _load() -> C.CDLL:
         "cobalt_ema_update": (C.c_int, [vp, vp, i64, C.c_float, u32, vp]),
         "cobalt_ochiai": (C.c_int, [vp, i32, vp, vp]),
         "cobalt_rebalance_intra_node": (C.c_int, [i32, i32, i32, i32, vp, vp, vp, vp, vp]),
+        "cobalt_dedup_workspace_bytes": (sz, [i64, i32, i32]),
+        "cobalt_dedup_index": (C.c_int, [vp, vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]),
+        "cobalt_forward_rows": (C.c_int, [vp, vp, vp, i64, i32, vp, i64, i64, vp]),
         "cobalt_permute_rows_block": (C.c_int, [vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_combine_block": (C.c_int, [vp, vp, vp, i64, i32, i32, vp, i64, u32, vp]),
         "cobalt_read_and_clear_device_error": (C.c_int, [C.POINTER(u32), vp]),
@@ -449,6 +453,57 @@ def rebalance_intra_node(N: int, Q: int, S: int, E: int, slot_expert, slot_load)
     _check(_lib.cobalt_rebalance_intra_node(N, Q, S, E, se, ld, new, moved, C.byref(kept)),
            "cobalt_rebalance_intra_node")
     return list(new), list(moved), int(kept.value)
+
+
+def dedup_workspace_bytes(T: int, K: int, N: int) -> int:
+    return _lib.cobalt_dedup_workspace_bytes(T, K, N)
+
+
+def dedup_index(assigned_slot: torch.Tensor, src_rank, N: int, Q: int, S: int, node_counts: torch.Tensor,
+                node_offsets: torch.Tensor, node_row_of_token: torch.Tensor, fwd_src_row: torch.Tensor,
+                workspace: torch.Tensor, *, cross_node_rows: Optional[torch.Tensor] = None) -> None:
+    """One row per (token, destination node): see cobalt_dedup_index."""
+    T, K = assigned_slot.shape
+    if (node_counts.numel() != N or node_offsets.numel() != N + 1 or node_row_of_token.numel() != T * N or
+            fwd_src_row.numel() != T * K or (cross_node_rows is not None and cross_node_rows.numel() != 1)):
+        raise CobaltError(ERR_INVALID_ARG, "dedup_index (output sizes)")
+    if isinstance(src_rank, int):
+        src_ptr, src_uniform = None, src_rank
+    else:
+        src_ptr, src_uniform = _ptr(src_rank, torch.int32, "src_rank"), 0
+    _check(_lib.cobalt_dedup_index(_ptr(assigned_slot, torch.int32, "assigned_slot"), src_ptr, src_uniform, T, K,
+                                   N, Q, S, _ptr(node_counts, torch.int32, "node_counts"),
+                                   _ptr(node_offsets, torch.int32, "node_offsets"),
+                                   _ptr(node_row_of_token, torch.int32, "node_row_of_token"),
+                                   _ptr(fwd_src_row, torch.int32, "fwd_src_row"),
+                                   _ptr(cross_node_rows, torch.int64, "cross_node_rows"), _ptr(workspace),
+                                   _ws_bytes(workspace), _stream()), "cobalt_dedup_index")
+
+
+def dedup_rows(x: torch.Tensor, node_row_of_token: torch.Tensor, N: int, dedup_send: torch.Tensor, *,
+               flags: int = 0) -> None:
+    """Fill the deduplicated buffer: the row mover with N optional copies per token."""
+    T, H = x.shape
+    if node_row_of_token.numel() != T * N or dedup_send.shape[1] != H:
+        raise CobaltError(ERR_INVALID_ARG, "dedup_rows (sizes)")
+    _check(_lib.cobalt_permute_rows_block(_ptr(x, torch.bfloat16, "x"),
+                                          _ptr(node_row_of_token, torch.int32, "node_row_of_token"), T, N, H,
+                                          _ptr(dedup_send, torch.bfloat16, "dedup_send"), dedup_send.shape[0], flags,
+                                          _stream()), "cobalt_permute_rows_block")
+
+
+def forward_rows(dedup_send: torch.Tensor, fwd_src_row: torch.Tensor, row_of_pair: torch.Tensor,
+                 recv: torch.Tensor) -> None:
+    """recv[row_of_pair[p]] = dedup_send[fwd_src_row[p]]."""
+    P = fwd_src_row.numel()
+    H = dedup_send.shape[1]
+    if row_of_pair.numel() != P or recv.shape[1] != H:
+        raise CobaltError(ERR_INVALID_ARG, "forward_rows (sizes)")
+    _check(_lib.cobalt_forward_rows(_ptr(dedup_send, torch.bfloat16, "dedup_send"),
+                                    _ptr(fwd_src_row, torch.int32, "fwd_src_row"),
+                                    _ptr(row_of_pair, torch.int32, "row_of_pair"), P, H,
+                                    _ptr(recv, torch.bfloat16, "recv"), dedup_send.shape[0], recv.shape[0], _stream()),
+           "cobalt_forward_rows")
 
 
 def read_and_clear_device_error() -> int:

@@ -492,6 +492,66 @@ perm_rows_bulk_oneshot_kernel(const uint8_t* __restrict__ x, const int32_t* __re
     }
 }
 
+// Row gather-scatter: dst[dst_row[i]] = src[src_row[i]] for i < n (rows of row_bytes bytes, cut into
+// column segments of at most seg_bytes).  One (row, segment) per single-warp CTA: a bulk async copy
+// global -> shared, then one shared -> global.  Negative indices are skipped.
+__global__ void __launch_bounds__(32)
+row_gather_scatter_kernel(const uint8_t* __restrict__ src, const int32_t* __restrict__ src_row,
+                          const int32_t* __restrict__ dst_row, int64_t n, int64_t src_rows, int64_t dst_rows,
+                          uint32_t row_bytes, int n_seg, uint32_t seg_bytes, uint8_t* __restrict__ dst,
+                          uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(128) uint8_t buf[];
+    __shared__ __align__(8) uint64_t full;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) / n_seg;
+    const uint32_t col = static_cast<uint32_t>(blockIdx.x % n_seg) * seg_bytes;
+    const uint32_t bytes = min(seg_bytes, row_bytes - col);
+    if (i >= n) return;
+    const int32_t from = __ldg(src_row + i), to = __ldg(dst_row + i);
+    if (from < 0 || to < 0) return;
+    if (from >= src_rows || to >= dst_rows) {
+        if (threadIdx.x == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+        return;
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(&full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_expect_tx(&full, bytes);
+        bulk_load(buf, src + static_cast<size_t>(from) * row_bytes + col, bytes, &full);
+        const bool ok = mbar_wait(&full, 0);
+        if (ok) bulk_store(dst + static_cast<size_t>(to) * row_bytes + col, buf, bytes);
+        else flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
+        bulk_commit();
+        bulk_wait_all();
+        if (!ok) (void)mbar_wait(&full, 0);
+    }
+}
+
+int launch_row_gather_scatter(const void* src, const int32_t* src_row, const int32_t* dst_row, int64_t n,
+                              int64_t src_rows, int64_t dst_rows, int H, void* dst, cudaStream_t stream)
+{
+    uint32_t* err_word = nullptr;
+    int rc = device_error_word(&err_word);
+    if (rc != COBALT_OK) return rc;
+    const uint32_t row_bytes = static_cast<uint32_t>(H) * 2u;
+    const int max_seg = g_tune.rows_item_bytes;
+    int n_seg = (row_bytes + max_seg - 1) / max_seg;
+    uint32_t seg_bytes = static_cast<uint32_t>(round_up((row_bytes + n_seg - 1) / n_seg, 16));
+    n_seg = (row_bytes + seg_bytes - 1) / seg_bytes;
+    const int64_t grid = n * n_seg;
+    if (grid > 0x7FFFFFFFll) return COBALT_ERR_UNSUPPORTED;
+    if (grid == 0) return COBALT_OK;
+    const size_t smem = round_up(seg_bytes, 128);
+    COBALT_CUDA_TRY(cudaFuncSetAttribute(row_gather_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem)));
+    row_gather_scatter_kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
+        static_cast<const uint8_t*>(src), src_row, dst_row, n, src_rows, dst_rows, row_bytes, n_seg, seg_bytes,
+        static_cast<uint8_t*>(dst), err_word);
+    COBALT_CUDA_TRY(cudaGetLastError());
+    return COBALT_OK;
+}
+
 // P bounds the row indices (rows of the whole send buffer), which may exceed T*K when the call
 // covers only a block of tokens.
 static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int K, int H, void* send,

@@ -28,4 +28,9 @@ int launch_scan_and_rank(const int32_t* keys, int64_t P, int D, const ChunkPlan&
                          uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
                          int32_t* pair_of_row, int rank_in_group, cudaStream_t s);
 
+// dst[dst_row[i]] = src[src_row[i]] for i < n, rows of H 16-bit elements; negative indices are skipped,
+// indices beyond src_rows / dst_rows are flagged and skipped.
+int launch_row_gather_scatter(const void* src, const int32_t* src_row, const int32_t* dst_row, int64_t n,
+                              int64_t src_rows, int64_t dst_rows, int H, void* dst, cudaStream_t stream);
+
 }  // namespace cobalt
