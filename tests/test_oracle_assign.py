@@ -358,3 +358,42 @@ def test_round_robin_balances_each_group_exactly(name, T):
         loads = rr["slot_load"][replicas].astype(int)
         assert loads.max() - loads.min() <= 1             # exact balance inside the group
         assert (np.diff(loads) <= 0).all()                # earlier replicas get the extra task
+
+
+def test_random_node_is_uniform_over_three_nodes():
+    """b* = 111 (three singles force all remote nodes); an expert held by all three picks each a third of the time."""
+    N, S = 4, 4
+    slot = _layout_from_nodes([[1], [2], [3], [1, 2, 3]], N)
+    T = 6000
+    ids = np.tile(np.array([[0, 1, 2, 3]], np.int32), (T, 1))
+    r = O.assign(N, 1, S, 4, slot, None, ids, np.zeros(T, np.int32), 321)
+    assert (r["remote_nodes"] == 3).all()
+    nodes = r["assigned_slot"][:, 3] // S
+    counts = np.bincount(nodes, minlength=4)[1:]
+    assert counts.sum() == T and (counts > 0).all()
+    assert (((counts - T / 3) ** 2) / (T / 3)).sum() < 25.0        # chi2, 2 dof
+
+
+def test_node_pick_and_replica_pick_are_independent_draws():
+    """RandomNode and UniformChoice use separate hash streams: with two nodes and two replicas on each,
+    the chosen node says nothing about which of the two replicas is chosen."""
+    # nodes 1 and 2 each have two ranks holding expert 2; experts 0 and 1 force b* = 011 from source node 0
+    N, Q, S = 3, 2, 3
+    slot = np.full(N * Q * S, -1, np.int32)
+    slot[0] = 3                                   # node 0 needs something: expert 3 lives there
+    slot[1 * Q * S + 0], slot[1 * Q * S + 1] = 0, 2          # node 1, rank 2: experts 0, 2
+    slot[1 * Q * S + S + 0] = 2                                # node 1, rank 3: expert 2
+    slot[2 * Q * S + 0], slot[2 * Q * S + 1] = 1, 2          # node 2, rank 4: experts 1, 2
+    slot[2 * Q * S + S + 0] = 2                                # node 2, rank 5: expert 2
+    T = 8000
+    ids = np.tile(np.array([[0, 1, 2]], np.int32), (T, 1))
+    r = O.assign(N, Q, S, 4, slot, None, ids, np.zeros(T, np.int32), 77)
+    d = r["assigned_slot"][:, 2]
+    node_bit = (d // (Q * S)) - 1                 # 0 for node 1, 1 for node 2
+    rank_bit = (d // S) % Q                       # which of the node's two ranks
+    table = np.zeros((2, 2))
+    for a, b in zip(node_bit, rank_bit):
+        table[a, b] += 1
+    assert (table > T / 8).all()                  # all four combinations occur often
+    expected = np.outer(table.sum(1), table.sum(0)) / T
+    assert (((table - expected) ** 2) / expected).sum() < 20.0     # chi2 independence, 1 dof
