@@ -120,6 +120,17 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
  * ascending order (first minimum wins), each such expert picks a node of that set and every
  * expert picks a replica inside its node, both uniformly through a counter hash of
  * (seed, t, e) so that results do not depend on launch shape.
+ * The counter hash (arithmetic modulo 2^32; seed_lo / seed_hi = low / high half of seed;
+ * stream 0 = node pick, 1 = replica pick):
+ *     x = seed_lo ^ 0x6A09E667
+ *     x = (x ^ t) * 0x9E3779B9;              x ^= x >> 16
+ *     x = (x ^ seed_hi) * 0xBB67AE85;        x ^= x >> 15
+ *     x = (x ^ (2*e + stream)) * 0x9E3779B9; x ^= x >> 16
+ *     x = x * 0xBB67AE85;                    x ^= x >> 15
+ *     x = x * 0x6A09E667;                    x ^= x >> 16
+ *     index among n candidates = (x * n) >> 32
+ * Node candidates are the set bits of b* & m counted from bit 0 (bit j = j-th remote node in
+ * ascending node id, source node skipped); replica candidates are R_{e,n} in ascending slot id.
  * src_rank: int32 [T], or NULL to use src_rank_uniform for every token.
  * Outputs: assigned_slot int32 [T*K] (r_te as global slot id); optional (NULL to skip)
  * slot_load uint32 [D] = w_er (Section 3.1), remote_nodes uint8 [T] = the token's term of
