@@ -35,18 +35,22 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
     constexpr bool kCountSlots = (MODE != kAssignGroupKey);   // group keys are not slots yet
 
     const int K = (KT > 0) ? KT : K_rt;
+    // the token's own loads go out first so that their latency overlaps the table staging
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    int32_t id[KMAX], out[KMAX];
+    int32_t s_t = src_uniform;
+    if (t < T) {
+        load_token_ids<KT>(topk_ids, t, K, id);
+        if (src_rank) s_t = __ldg(src_rank + t);
+    }
     const TableView tv = stage_tables(lv, tab);
     if (kCountSlots && slot_load)
         for (int i = threadIdx.x; i < lv.D; i += blockDim.x) hist[i] = 0;
     if (threadIdx.x < 2) cta_totals[threadIdx.x] = 0;
     __syncthreads();
 
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     uint32_t cost = 0, naive_cost = 0;
     if (t < T) {
-        int32_t id[KMAX], out[KMAX];
-        load_token_ids<KT>(topk_ids, t, K, id);
-        const int32_t s_t = src_rank ? __ldg(src_rank + t) : src_uniform;
         uint32_t bad = check_token_ids<KT>(id, K, lv.E);
         if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
         if (bad) {

@@ -34,20 +34,21 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     const int K = (KT > 0) ? KT : K_rt;
     cg::cluster_group cluster = cg::this_cluster();
 
+    // the first token's ids are requested before the tile is cleared so that the two overlap
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    int32_t id[KMAX];
+    if (t < T) load_token_ids<KT>(topk_ids, t, K, id);
     const int n_vec = (static_cast<int>(tri_entries(E)) + 3) / 4;
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
-        int32_t id[KMAX];
-        load_token_ids<KT>(topk_ids, t, K, id);
+    while (t < T) {
         const uint32_t bad = check_token_ids<KT>(id, K, E);
-        if (bad) {
-            flag_error(err_word, bad);
-            continue;
-        }
-        add_token_to_triangle<KT>(tri, id, K);
+        if (bad) flag_error(err_word, bad);
+        else add_token_to_triangle<KT>(tri, id, K);
+        t += stride;
+        if (t < T) load_token_ids<KT>(topk_ids, t, K, id);
     }
 
     cluster.sync();            // every tile of the cluster is complete

@@ -62,22 +62,33 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
     cg::cluster_group cluster = cg::this_cluster();
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the scan kernel may be scheduled early
+    const int64_t tokens_per_round = static_cast<int64_t>(gridDim.x) * kRouteThreads;
+    const int n_rounds = static_cast<int>((T + tokens_per_round - 1) / tokens_per_round);
+    // the first round's loads go out before the shared-memory set-up so that the two overlap
+    int32_t id[KMAX], out[KMAX];
+    int32_t s_t = src_uniform;
+    {
+        const int64_t t0 = static_cast<int64_t>(blockIdx.x) * kRouteThreads + threadIdx.x;
+        if (n_rounds > 0 && t0 < T) {
+            load_token_ids<KT>(topk_ids, t0, K, id);
+            if (src_rank) s_t = __ldg(src_rank + t0);
+        }
+    }
     for (int i = threadIdx.x; i < tri_words / 4; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     for (int i = threadIdx.x; i < kRouteChunksPerRound * D; i += blockDim.x) chist[i] = 0;
     if (threadIdx.x < 2) cta_totals[threadIdx.x] = 0;
     const TableView tv = stage_tables(lv, tab);
     __syncthreads();
 
-    const int64_t tokens_per_round = static_cast<int64_t>(gridDim.x) * kRouteThreads;
-    const int n_rounds = static_cast<int>((T + tokens_per_round - 1) / tokens_per_round);
     uint32_t cost_sum = 0, naive_sum = 0;
     for (int round = 0; round < n_rounds; ++round) {
         const int64_t base = (static_cast<int64_t>(round) * gridDim.x + blockIdx.x) * kRouteThreads;
         const int64_t t = base + threadIdx.x;
         if (t < T) {
-            int32_t id[KMAX], out[KMAX];
-            load_token_ids<KT>(topk_ids, t, K, id);
-            const int32_t s_t = src_rank ? __ldg(src_rank + t) : src_uniform;
+            if (round > 0) {
+                load_token_ids<KT>(topk_ids, t, K, id);
+                if (src_rank) s_t = __ldg(src_rank + t);
+            }
             const uint32_t bad_ids = check_token_ids<KT>(id, K, lv.E);
             uint32_t bad = bad_ids;
             if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
