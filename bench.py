@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 METRIC = "routed token-expert pairs/sec"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
-KERNELS_PER_STEP = 7               # stats 1, assign 1, permute 4 (hist, scan, rank, rows), combine 1
+KERNELS_PER_STEP = 9               # stats 2 (clear + tile), assign 2 (clear + assign), permute 4 (hist, scan, rank, rows), combine 1
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes per pair, measured on a reduced token count and scaled by the pairs of a launch)
@@ -512,7 +512,8 @@ def run_cobalt(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 rows, u32 counts, f32 accumulate",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "dtype_detail": "bf16 rows moved bit-exactly, fp32 accumulation in the combine, u32 counts, i32 indices",
             "data": "synthetic",
             "config": {"workload": workload_name(w), "seed": int(w.seed),
                        "l2": "no explicit flush: each step streams the 15 GB send buffer through L2 twice, "

@@ -34,6 +34,8 @@ struct Tuning {
     int rows_per_sm = 0;            // cap on CTAs per SM (0 = as many as shared memory allows)
     int rows_vec_per_sm = 0;        // vector row mover: CTAs per SM (0 = one CTA per token)
     int rows_hint = 0;              // 1 = evict-first L2 hints on the bulk copies
+    int stats_max_ctas = 0;         // statistics kernel: cap on CTAs (0 = one per 1024 tokens, at most the SM count)
+    int stats_cluster = 0;          // statistics kernel: force this cluster size (0 = pick)
     int combine_per_sm = 0;         // CTAs per SM of the combine kernel's grid (0 = one CTA per token)
 };
 extern Tuning g_tune;

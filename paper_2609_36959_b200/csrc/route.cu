@@ -199,7 +199,7 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
     }
     RouteLaunch best = {0, 0};
     for (int i = 0; i < n_cand; ++i) {
-        if (cand_cta[i] * 10 >= most * 9) {
+        if (cand_cta[i] * 4 >= most * 3) {
             best.cluster = cand_cs[i];
             best.ctas = cand_cta[i];
             break;
