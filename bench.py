@@ -389,7 +389,7 @@ def run_cobalt(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the routing path has no CPU fallback")
     torch.cuda.set_device(local_rank)
-    distributed = world > 1
+    distributed = world > 1 or "TORCHELASTIC_RUN_ID" in os.environ   # under torchrun: always through NCCL
     if distributed:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
