@@ -96,10 +96,12 @@ perm_scan_kernel(uint32_t* __restrict__ ws, int D, int n_chunks, uint32_t* __res
 // ---- K3 -----------------------------------------------------------------------------------
 // Lanes of the warp holding the same key, built from one ballot per key bit (the hardware
 // match instruction is far slower than a dozen votes for keys this narrow).
-__device__ __forceinline__ uint32_t peers_of(uint32_t key, int key_bits)
+template <int kKeyBits>
+__device__ __forceinline__ uint32_t peers_of(uint32_t key)
 {
     uint32_t peers = 0xFFFFFFFFu;
-    for (int b = 0; b < key_bits; ++b) {
+#pragma unroll
+    for (int b = 0; b < kKeyBits; ++b) {
         const uint32_t bit = (key >> b) & 1u;
         const uint32_t vote = __ballot_sync(0xFFFFFFFFu, bit);
         peers &= bit ? vote : ~vote;
@@ -107,6 +109,8 @@ __device__ __forceinline__ uint32_t peers_of(uint32_t key, int key_bits)
     return peers;
 }
 
+// kKeyBits >= bits of D (keys 0..D, D marking "no destination"); the votes are fully unrolled
+template <int kKeyBits>
 __global__ void __launch_bounds__(kPermThreads)
 perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
                  const uint32_t* __restrict__ ws, const uint32_t* __restrict__ dest_counts,
@@ -155,7 +159,6 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
     // The warp's sub-range is walked in super-steps of kRankSteps x 32 pairs whose slots are
     // loaded back to back into registers (one exposed memory latency per super-step, not per step).
     const int n_super = (sub + 32 * kRankSteps - 1) / (32 * kRankSteps);
-    const int key_bits = 32 - __clz(D);      // keys 0..D (D marks "no destination")
     int32_t dreg[kRankSteps];
     uint32_t preg[kRankSteps];     // lanes sharing each step's destination (kept from pass A)
     auto load_super = [&](int ss) {
@@ -173,7 +176,7 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
 #pragma unroll
         for (int s = 0; s < kRankSteps; ++s) {
             const int32_t d = dreg[s];
-            const uint32_t peers = peers_of(static_cast<uint32_t>(d < 0 ? D : d), key_bits);
+            const uint32_t peers = peers_of<kKeyBits>(static_cast<uint32_t>(d < 0 ? D : d));
             preg[s] = peers;
             if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
             __syncwarp();
@@ -197,7 +200,7 @@ perm_rank_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, 
             load_super(ss);
 #pragma unroll
             for (int s = 0; s < kRankSteps; ++s)
-                preg[s] = peers_of(static_cast<uint32_t>(dreg[s] < 0 ? D : dreg[s]), key_bits);
+                preg[s] = peers_of<kKeyBits>(static_cast<uint32_t>(dreg[s] < 0 ? D : dreg[s]));
         }
 #pragma unroll
         for (int s = 0; s < kRankSteps; ++s) {
@@ -673,12 +676,22 @@ int launch_scan_and_rank(const int32_t* assigned_slot, int64_t P, int D, const C
     cfg.dynamicSmemBytes = 0;
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, perm_scan_kernel, ws, D, c.n_chunks, dest_counts));
     const size_t smem = sizeof(uint32_t) * static_cast<size_t>(D) * (1 + kPermWarps);
+    using RankKernel = void (*)(const int32_t*, int64_t, int, int, int, const uint32_t*, const uint32_t*, uint32_t*,
+                                int32_t*, int32_t*, int);
+    int need_bits = 1;
+    while ((1 << need_bits) <= D) ++need_bits;       // keys 0..D
+    RankKernel kernel = perm_rank_kernel<13>;
+    if (need_bits <= 4) kernel = perm_rank_kernel<4>;
+    else if (need_bits <= 6) kernel = perm_rank_kernel<6>;
+    else if (need_bits <= 8) kernel = perm_rank_kernel<8>;
+    else if (need_bits <= 9) kernel = perm_rank_kernel<9>;
+    else if (need_bits <= 10) kernel = perm_rank_kernel<10>;
+    else if (need_bits <= 11) kernel = perm_rank_kernel<11>;
     if (smem > 48 * 1024)
-        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem)));
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     cfg.gridDim = dim3(c.n_chunks);
     cfg.dynamicSmemBytes = smem;
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, perm_rank_kernel, assigned_slot, P, D, c.chunk, c.n_chunks,
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, assigned_slot, P, D, c.chunk, c.n_chunks,
                                        static_cast<const uint32_t*>(ws), static_cast<const uint32_t*>(dest_counts),
                                        dest_offsets, row_of_pair, pair_of_row, rank_in_group));
     return COBALT_OK;
