@@ -284,8 +284,17 @@ def extra_measurements(args, w, step, cb, torch):
         out["fused_route_index_us"] = None
         out["fused_error"] = str(exc)[:200]
 
+    # the next two blocks allocate one more buffer of the send buffer's size: only with room to spare
+    send_bytes = step.send.numel() * 2
+
+    def has_room():
+        free, _ = torch.cuda.mem_get_info()
+        return free > 1.5 * send_bytes + (2 << 30)
+
     # backward of the two row stages (adjoints), same buffers: grad_send := send, grad_y := y
     try:
+        if not has_room():
+            raise RuntimeError("skipped: not enough free device memory for another send-sized buffer")
         peak, _ = hbm_peak()
         grad_x = torch.empty_like(step.x)
         grad_out = torch.empty_like(step.send)
@@ -303,6 +312,9 @@ def extra_measurements(args, w, step, cb, torch):
 
     # node-deduplicated send layout: one row per (token, destination node) instead of per pair
     try:
+        torch.cuda.empty_cache()
+        if not has_room():
+            raise RuntimeError("skipped: not enough free device memory for another send-sized buffer")
         peak, _ = hbm_peak()
         T, K, H, P, N = w.T, w.K, w.H, w.P, w.N
         node_counts = torch.zeros(N, dtype=torch.int32, device="cuda")
