@@ -413,6 +413,11 @@ def run_cobalt(args):
     w = W.make_config(args.config, T=args.tokens)
     if args.hidden is not None:
         w.H = args.hidden
+    need = 2 * w.P * w.H + 4 * w.T * w.H + 64 * w.P + (1 << 28)     # send + x + y + index arrays + slack
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        raise SystemExit(f"bench.py: {workload_name(w)} needs about {need / 2**30:.1f} GiB of device memory, "
+                         f"only {free / 2**30:.1f} GiB are free on cuda:{local_rank}")
     layout = cb.Layout(w.N, w.Q, w.S, w.E, w.slot_expert.tolist(), w.primary_slot.tolist())
     step = RouteStep(layout, w.T, w.K, w.H)
 
