@@ -7,7 +7,8 @@
 // all CTAs of the cluster through distributed shared memory and merges the result into global
 // memory with integer reductions, mirroring (hi, lo) to (lo, hi) and writing the diagonal to
 // `load` as well.  Only integer adds are used, so the result is independent of scheduling.
-// Experts counts whose triangle does not fit in shared memory take a direct global-atomic path.
+// Expert counts whose triangle does not fit in one CTA's shared memory spread it over the CTAs
+// of a cluster (coact_spread_kernel).
 #include <cooperative_groups.h>
 
 #include <map>
@@ -77,6 +78,114 @@ coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int 
             for (int b = 0; b < K; ++b) atomicAdd(&coact[static_cast<size_t>(id[a]) * E + id[b]], 1u);
         }
     }
+}
+
+// Expert counts whose triangle exceeds one CTA's shared memory: the triangle of a CLUSTER is
+// spread over its CTAs (flat index idx lives in CTA idx mod C at word idx / C, so that the hot
+// low-numbered entries do not pile onto one CTA) and every CTA adds its own tokens' pairs with
+// shared-memory atomics that may land in a peer's shared memory.  After a cluster barrier each CTA
+// merges the words it owns into global memory.  E = 1024 needs 2.1 MB per cluster: 16 CTAs x 131 KB.
+template <int KT>
+__global__ void __launch_bounds__(kStatsThreads)
+coact_spread_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int log2_c, int words_per_cta,
+                    uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(16) uint32_t part[];   // this CTA's share of the cluster's triangle
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    const int K = (KT > 0) ? KT : K_rt;
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t c_mask = (1u << log2_c) - 1u;
+
+    for (int i = threadIdx.x; i < words_per_cta; i += blockDim.x) part[i] = 0;
+    cluster.sync();            // every share is cleared before any peer adds to it
+
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
+        int32_t id[KMAX];
+        load_token_ids<KT>(topk_ids, t, K, id);
+        const uint32_t bad = check_token_ids<KT>(id, K, E);
+        if (bad) {
+            flag_error(err_word, bad);
+            continue;
+        }
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a) {
+#pragma unroll
+            for (int b = a; b < KMAX; ++b) {
+                if (b < K) {
+                    const uint32_t hi = max(id[a], id[b]), lo = min(id[a], id[b]);
+                    const uint32_t idx = hi * (hi + 1) / 2 + lo;
+                    atomicAdd(cluster.map_shared_rank(part, idx & c_mask) + (idx >> log2_c), 1u);
+                }
+            }
+        }
+    }
+    cluster.sync();            // all adds of the cluster have landed
+    wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
+    const uint32_t n_tri = static_cast<uint32_t>(tri_entries(E));
+    const uint32_t crank = cluster.block_rank();
+    for (int l = threadIdx.x; l < words_per_cta; l += blockDim.x) {
+        const uint32_t v = part[l];
+        const uint32_t idx = (static_cast<uint32_t>(l) << log2_c) | crank;
+        if (v && idx < n_tri) {
+            const int hi = tri_row(static_cast<int>(idx));
+            const int lo = static_cast<int>(idx) - hi * (hi + 1) / 2;
+            atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], v);
+            if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], v);
+            else atomicAdd(&load[hi], v);
+        }
+    }
+}
+
+template <int KT>
+static int launch_spread(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
+                         uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
+{
+    *launched = false;
+    auto kernel = coact_spread_kernel<KT>;
+    const size_t n_tri = tri_entries(E);
+    int log2_c = 1;
+    while (log2_c < 4 && round_up((n_tri + (1u << log2_c) - 1) >> log2_c, 4) * sizeof(uint32_t) > kStatsMaxTileBytes / 2)
+        ++log2_c;                                    // shares of <= 100 KB when possible (two CTAs per SM)
+    while (log2_c <= 4 && round_up((n_tri + (1u << log2_c) - 1) >> log2_c, 4) * sizeof(uint32_t) > kStatsMaxTileBytes)
+        ++log2_c;
+    if (log2_c > 3) return COBALT_OK;   // 16 shares measured slower than plain global atomics: caller falls back
+    const int c = 1 << log2_c;
+    const int words = static_cast<int>(round_up((n_tri + c - 1) / c, 4));
+    const size_t smem = static_cast<size_t>(words) * sizeof(uint32_t);
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return COBALT_OK;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    cfg.blockDim = dim3(kStatsThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(c);
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
+        (void)cudaGetLastError();
+        return COBALT_OK;
+    }
+    int64_t want = (T + kStatsThreads - 1) / kStatsThreads;      // about one token per thread
+    int64_t clusters = (want + c - 1) / c;
+    if (clusters > max_clusters) clusters = max_clusters;
+    if (clusters * c > 2ll * n_sm) clusters = 2ll * n_sm / c;
+    if (clusters < 1) clusters = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(clusters * c));
+    set_programmatic_launch(&attr[1], after_zeroing);
+    cfg.numAttrs = 2;
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, log2_c, words, coact, load, err_word));
+    *launched = true;
+    return COBALT_OK;
 }
 
 template <int KT>
@@ -206,6 +315,16 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     if (rc != COBALT_OK) return rc;
 
     if (tri_entries(E) * sizeof(uint32_t) > kStatsMaxTileBytes) {
+        bool launched = false;
+        switch (K) {
+            case 2: rc = launch_spread<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 4: rc = launch_spread<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 6: rc = launch_spread<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 8: rc = launch_spread<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            default: rc = launch_spread<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
+        }
+        if (rc != COBALT_OK || launched) return rc;
+        // last resort (clusters unavailable): every pair straight to global memory
         int64_t want = (T + 255) / 256;
         const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
         cudaLaunchConfig_t cfg = {};

@@ -166,6 +166,24 @@ def test_large_expert_count_takes_global_path(cb):
     check_index_stages(cb, w, step, 9)
 
 
+@pytest.mark.parametrize("E,K,T", [(320, 8, 20000), (384, 8, 131072), (451, 7, 9999), (512, 6, 30000),
+                                   (1024, 8, 50000), (1024, 16, 3000)])
+def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
+    """E > 316: the co-activation triangle no longer fits one CTA and is spread over the cluster."""
+    model = W.configs.ClusterModel(E, K, 8, 0.7, np.full(8, 1 / 8), np.ones(E))
+    ids = W.sample_topk_ids(model, T, seed=E + K)
+    ids_d = torch.from_numpy(ids).cuda()
+    coact = torch.full((E, E), 9, dtype=torch.int32, device="cuda")
+    load = torch.full((E,), 9, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        cb.coact_stats(ids_d, E, coact, load)
+    cb.coact_stats(ids_d, E, coact, load, flags=cb.STATS_ACCUMULATE)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    ref_coact, ref_load = O.coact_stats(ids, E)
+    assert (u32(coact) == 2 * ref_coact).all() and (u32(load) == 2 * ref_load).all()
+
+
 def test_empty_batch(cb):
     w = W.make_custom(0, 8, 2, 16, 2, 2, 3, seed=1)
     layout, step = make_step(w)
