@@ -25,7 +25,9 @@ namespace cobalt {
 constexpr int kStatsThreads = 1024;
 constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 
-template <int KT>
+// kPacked: 16-bit counters, two per word.  The launcher selects it only when one CLUSTER sees at
+// most 65535 tokens, so that neither a tile nor the sum of a cluster's tiles can overflow a half.
+template <int KT, bool kPacked>
 __global__ void __launch_bounds__(kStatsThreads)
 coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E,
                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
@@ -40,21 +42,21 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     int32_t id[KMAX];
     if (t < T) load_token_ids<KT>(topk_ids, t, K, id);
-    const int n_vec = (static_cast<int>(tri_entries(E)) + 3) / 4;
+    const int n_vec = (static_cast<int>(tri_entries(E)) + (kPacked ? 7 : 3)) / (kPacked ? 8 : 4);
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     while (t < T) {
         const uint32_t bad = check_token_ids<KT>(id, K, E);
         if (bad) flag_error(err_word, bad);
-        else add_token_to_triangle<KT>(tri, id, K);
+        else add_token_to_triangle<KT, kPacked>(tri, id, K);
         t += stride;
         if (t < T) load_token_ids<KT>(topk_ids, t, K, id);
     }
 
     cluster.sync();            // every tile of the cluster is complete
     wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
-    merge_triangle_over_cluster(tri, E, coact, load);
+    merge_triangle_over_cluster<kPacked>(tri, E, coact, load);
     cluster.sync();            // no CTA may exit while a peer still reads its tile
 }
 
@@ -188,12 +190,18 @@ static int launch_spread(const int32_t* ids, int64_t T, int K, int E, uint32_t* 
     return COBALT_OK;
 }
 
-template <int KT>
-static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                       uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream)
+static size_t tile_bytes(int E, bool packed)
 {
-    auto kernel = coact_tile_kernel<KT>;
-    const size_t smem = round_up(tri_entries(E) * sizeof(uint32_t), 16);
+    return round_up((packed ? (tri_entries(E) + 1) / 2 : tri_entries(E)) * sizeof(uint32_t), 16);
+}
+
+template <int KT, bool kPacked>
+static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
+                       uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
+{
+    *launched = false;
+    auto kernel = coact_tile_kernel<KT, kPacked>;
+    const size_t smem = tile_bytes(E, kPacked);
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
 
@@ -217,7 +225,7 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
 
     // candidates: cluster sizes 16 (non-portable), 8, 4, 2, 1 -> CTAs that can be co-resident
     static std::mutex cache_lock;
-    static std::map<std::tuple<int, int, int, int>, std::pair<int, int>> cache;   // (dev, E, want, KT)
+    static std::map<std::tuple<int, int, int, int>, std::pair<int, int>> cache;   // (dev, E, want, KT); per kPacked
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
     const auto key = std::make_tuple(dev, E, static_cast<int>(want) + 4096 * g_tune.stats_cluster, KT);
@@ -265,13 +273,36 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
             cache[key] = std::make_pair(best_cs, best_cta);
         }
     }
-    if (best_cs == 0) return COBALT_ERR_UNSUPPORTED;
+    if (best_cs == 0) return kPacked ? COBALT_OK : COBALT_ERR_UNSUPPORTED;
+    if (kPacked) {
+        // tokens one cluster can see: its CTAs x the grid-stride trips of one CTA x the block size
+        const int64_t trips = (T + static_cast<int64_t>(best_cta) * kStatsThreads - 1) / (static_cast<int64_t>(best_cta) * kStatsThreads);
+        if (trips * kStatsThreads * best_cs > 65535) return COBALT_OK;   // caller takes the 32-bit tile
+    }
     attr[0].val.clusterDim.x = best_cs;
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
     set_programmatic_launch(&attr[1], after_zeroing);
     cfg.numAttrs = 2;
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, coact, load, err_word));
+    *launched = true;
     return COBALT_OK;
+}
+
+// The 16-bit tile when it is allowed and wanted, else the 32-bit tile when it fits.
+template <int KT>
+static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
+                        uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
+{
+    *launched = false;
+    const bool fits32 = tile_bytes(E, false) <= kStatsMaxTileBytes;
+    const bool fits16 = tile_bytes(E, true) <= kStatsMaxTileBytes;
+    const bool want16 = g_tune.stats_packed > 0 || (g_tune.stats_packed < 0 && !fits32);
+    if (fits16 && want16) {
+        const int rc = launch_tile<KT, true>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
+        if (rc != COBALT_OK || *launched) return rc;
+    }
+    if (!fits32) return COBALT_OK;
+    return launch_tile<KT, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
 }
 
 }  // namespace cobalt
@@ -314,39 +345,40 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     rc = sm_count(&n_sm);
     if (rc != COBALT_OK) return rc;
 
-    if (tri_entries(E) * sizeof(uint32_t) > kStatsMaxTileBytes) {
-        bool launched = false;
-        switch (K) {
-            case 2: rc = launch_spread<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 4: rc = launch_spread<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 6: rc = launch_spread<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 8: rc = launch_spread<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            default: rc = launch_spread<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
-        }
-        if (rc != COBALT_OK || launched) return rc;
-        // last resort (clusters unavailable): every pair straight to global memory
-        int64_t want = (T + 255) / 256;
-        const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
-        cudaLaunchConfig_t cfg = {};
-        cudaLaunchAttribute attr[1];
-        cfg.gridDim = dim3(grid);
-        cfg.blockDim = dim3(256);
-        cfg.stream = s;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        set_programmatic_launch(&attr[0], after_zeroing);
-        COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, coact_global_kernel, topk_ids, T, static_cast<int>(K),
-                                           static_cast<int>(E), coact, load, err_word));
-        return COBALT_OK;
-    }
+    bool launched = false;
     switch (K) {
-        case 1: return launch_tile<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
-        case 2: return launch_tile<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
-        case 4: return launch_tile<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
-        case 6: return launch_tile<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
-        case 8: return launch_tile<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
-        default: return launch_tile<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s);
+        case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
     }
+    if (rc != COBALT_OK || launched) return rc;
+    if (tile_bytes(E, false) <= kStatsMaxTileBytes) return COBALT_ERR_UNSUPPORTED;   // clusters unavailable
+
+    switch (K) {
+        case 2: rc = launch_spread<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 4: rc = launch_spread<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 6: rc = launch_spread<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        case 8: rc = launch_spread<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+        default: rc = launch_spread<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
+    }
+    if (rc != COBALT_OK || launched) return rc;
+    // last resort: every pair straight to global memory
+    int64_t want = (T + 255) / 256;
+    const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    set_programmatic_launch(&attr[0], after_zeroing);
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, coact_global_kernel, topk_ids, T, static_cast<int>(K),
+                                       static_cast<int>(E), coact, load, err_word));
+    return COBALT_OK;
 }
 
 }  // extern "C"

@@ -214,7 +214,9 @@ __device__ __forceinline__ void assign_token(const TableView& tv, const int32_t 
 }
 
 // Adds the K(K+1)/2 unordered pairs of one token (diagonal included) to a lower-triangle tile.
-template <int KT>
+// kPacked: two 16-bit counters per word (entry idx in the low or high half of word idx / 2); the
+// caller guarantees that no counter of the tile, nor its sum over the cluster, reaches 65536.
+template <int KT, bool kPacked = false>
 __device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32_t (&id)[TokenShape<KT>::KMAX], int K)
 {
     constexpr int KMAX = TokenShape<KT>::KMAX;
@@ -224,7 +226,9 @@ __device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32
         for (int b = a; b < KMAX; ++b) {
             if (b < K) {
                 const int hi = max(id[a], id[b]), lo = min(id[a], id[b]);
-                atomicAdd(&tri[hi * (hi + 1) / 2 + lo], 1u);
+                const int idx = hi * (hi + 1) / 2 + lo;
+                if (kPacked) atomicAdd(&tri[idx >> 1], (idx & 1) ? 0x10000u : 1u);
+                else atomicAdd(&tri[idx], 1u);
             }
         }
     }
@@ -245,13 +249,16 @@ __device__ __forceinline__ int tri_row(int idx)
 // all tiles of the cluster with 16-byte distributed-shared-memory loads and merges the sums into
 // coact (both (hi, lo) and (lo, hi)) and load (the diagonal) with global integer reductions.
 // The caller must hold a second cluster barrier before any CTA exits.
+template <bool kPacked = false>
 __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E, uint32_t* __restrict__ coact,
                                                             uint32_t* __restrict__ load)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    constexpr int kPerWord = kPacked ? 2 : 1;            // triangle entries per 32-bit word
     const int n_tri = static_cast<int>(tri_entries(E));
-    const int n_vec = (n_tri + 3) / 4;
+    const int n_words = (n_tri + kPerWord - 1) / kPerWord;
+    const int n_vec = (n_words + 3) / 4;
     const int csize = static_cast<int>(cluster.num_blocks());
     const int crank = static_cast<int>(cluster.block_rank());
     const int per = (n_vec + csize - 1) / csize;
@@ -260,17 +267,19 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
         uint4 s = make_uint4(0, 0, 0, 0);
         for (int r = 0; r < csize; ++r) {
             const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
-            s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+            s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;    // packed halves cannot carry (see above)
         }
-        const uint32_t part[4] = {s.x, s.y, s.z, s.w};
-        int hi = tri_row(4 * v);
-        int lo = 4 * v - hi * (hi + 1) / 2;
+        const uint32_t word[4] = {s.x, s.y, s.z, s.w};
+        const int first = 4 * kPerWord * v;                      // first triangle entry of this vector
+        int hi = tri_row(first);
+        int lo = first - hi * (hi + 1) / 2;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (4 * v + c < n_tri && part[c]) {
-                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], part[c]);
-                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], part[c]);
-                else atomicAdd(&load[hi], part[c]);
+        for (int c = 0; c < 4 * kPerWord; ++c) {
+            const uint32_t val = kPacked ? ((word[c >> 1] >> (16 * (c & 1))) & 0xFFFFu) : word[c];
+            if (first + c < n_tri && val) {
+                atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], val);
+                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
+                else atomicAdd(&load[hi], val);
             }
             if (++lo > hi) { ++hi; lo = 0; }
         }

@@ -166,10 +166,13 @@ def test_large_expert_count_takes_global_path(cb):
     check_index_stages(cb, w, step, 9)
 
 
-@pytest.mark.parametrize("E,K,T", [(320, 8, 20000), (384, 8, 131072), (451, 7, 9999), (512, 6, 30000),
+@pytest.mark.parametrize("E,K,T", [(320, 8, 20000), (384, 8, 131072), (451, 7, 9999), (452, 8, 70001),
+                                   (453, 8, 70001), (320, 8, 757777), (512, 6, 30000),
                                    (1024, 8, 50000), (1024, 16, 3000)])
 def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
-    """E > 316: the co-activation triangle no longer fits one CTA and is spread over the cluster."""
+    """E > 316: the 32-bit triangle no longer fits one CTA.  Up to E = 452 a tile of 16-bit counters
+    does, as long as a cluster sees at most 65535 tokens (T = 757777 does not qualify); beyond that
+    the triangle is spread over the CTAs of a cluster."""
     model = W.configs.ClusterModel(E, K, 8, 0.7, np.full(8, 1 / 8), np.ones(E))
     ids = W.sample_topk_ids(model, T, seed=E + K)
     ids_d = torch.from_numpy(ids).cuda()
@@ -182,6 +185,29 @@ def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
     assert cb.read_and_clear_device_error() == 0
     ref_coact, ref_load = O.coact_stats(ids, E)
     assert (u32(coact) == 2 * ref_coact).all() and (u32(load) == 2 * ref_load).all()
+
+
+@pytest.mark.parametrize("E,K,T", [(256, 8, 131072), (64, 6, 40000), (16, 2, 5000), (8, 8, 1500), (256, 8, 700000)])
+def test_statistics_with_sixteen_bit_tiles_forced(cb, E, K, T):
+    """The 16-bit tile, chosen by default only where the 32-bit one does not fit, gives the same counts
+    at every size; T = 700000 exceeds what it may count and must take the 32-bit tile by itself."""
+    import ctypes
+    tune = cb.binding._lib.cobalt_internal_tune
+    tune.argtypes = [ctypes.c_char_p, ctypes.c_int]
+    model = W.configs.ClusterModel(E, K, 4, 0.7, np.full(4, 1 / 4), np.ones(E))
+    ids = W.sample_topk_ids(model, T, seed=3 * E + K)
+    ids_d = torch.from_numpy(ids).cuda()
+    coact = torch.full((E, E), 7, dtype=torch.int32, device="cuda")
+    load = torch.full((E,), 7, dtype=torch.int32, device="cuda")
+    assert tune(b"stats_packed", 1) == 0
+    try:
+        cb.coact_stats(ids_d, E, coact, load)
+        torch.cuda.synchronize()
+    finally:
+        assert tune(b"stats_packed", -1) == 0
+    assert cb.read_and_clear_device_error() == 0
+    ref_coact, ref_load = O.coact_stats(ids, E)
+    assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
 
 
 def test_empty_batch(cb):
