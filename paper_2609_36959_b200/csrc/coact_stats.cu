@@ -224,22 +224,23 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     attr[0].val.clusterDim.z = 1;
 
     // candidates: cluster sizes 16 (non-portable), 8, 4, 2, 1 -> CTAs that can be co-resident
+    struct Candidates { int n = 0, cs[5], cta[5]; };
     static std::mutex cache_lock;
-    static std::map<std::tuple<int, int, int, int>, std::pair<int, int>> cache;   // (dev, E, want, KT); per kPacked
+    static std::map<std::tuple<int, int, int, int>, Candidates> cache;   // (dev, E, want, cluster knob); per <KT, kPacked>
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
-    const auto key = std::make_tuple(dev, E, static_cast<int>(want) + 4096 * g_tune.stats_cluster, KT);
-    int best_cs = 0, best_cta = 0;
+    const auto key = std::make_tuple(dev, E, static_cast<int>(want), g_tune.stats_cluster);
+    Candidates cand;
+    bool cached = false;
     {
         std::lock_guard<std::mutex> guard(cache_lock);
         auto it = cache.find(key);
         if (it != cache.end()) {
-            best_cs = it->second.first;
-            best_cta = it->second.second;
+            cand = it->second;
+            cached = true;
         }
     }
-    if (best_cs == 0) {
-        int cand_cs[5], cand_cta[5], n_cand = 0, most = 0;
+    if (!cached) {
         for (int cs = 16; cs >= 1; cs >>= 1) {
             if (cs > want) continue;
             if (g_tune.stats_cluster > 0 && cs != g_tune.stats_cluster) continue;
@@ -253,32 +254,35 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
             int n_cta = static_cast<int>(want) / cs * cs;
             if (n_cta > max_clusters * cs) n_cta = max_clusters * cs;
             if (n_cta < cs) continue;
-            cand_cs[n_cand] = cs;
-            cand_cta[n_cand] = n_cta;
-            ++n_cand;
-            if (n_cta > most) most = n_cta;
+            cand.cs[cand.n] = cs;
+            cand.cta[cand.n] = n_cta;
+            ++cand.n;
         }
-        // the largest cluster that keeps at least 3/4 of the best CTA count: the merge (distributed
-        // shared memory reads and global reductions, ~10 us of a 23 us kernel at E = 256) shrinks with
-        // the number of clusters, the per-token work (~4 us) grows only mildly with fewer CTAs
-        for (int i = 0; i < n_cand; ++i) {
-            if (cand_cta[i] * 4 >= most * 3) {
-                best_cs = cand_cs[i];
-                best_cta = cand_cta[i];
-                break;
-            }
-        }
-        if (best_cs != 0) {
-            std::lock_guard<std::mutex> guard(cache_lock);
-            cache[key] = std::make_pair(best_cs, best_cta);
+        std::lock_guard<std::mutex> guard(cache_lock);
+        cache[key] = cand;
+    }
+    // 16-bit tiles: a cluster may see at most 65535 tokens (its CTAs x the grid-stride trips of one
+    // CTA x the block size), which rules out the larger clusters when T is large
+    bool legal[5];
+    int most = 0;
+    for (int i = 0; i < cand.n; ++i) {
+        const int64_t per_trip = static_cast<int64_t>(cand.cta[i]) * kStatsThreads;
+        const int64_t trips = (T + per_trip - 1) / per_trip;
+        legal[i] = !kPacked || trips * kStatsThreads * cand.cs[i] <= 65535;
+        if (legal[i] && cand.cta[i] > most) most = cand.cta[i];
+    }
+    // the largest cluster that keeps at least 3/4 of the best CTA count: the merge (distributed
+    // shared memory reads and global reductions, ~10 us of a 23 us kernel at E = 256) shrinks with
+    // the number of clusters, the per-token work (~4 us) grows only mildly with fewer CTAs
+    int best_cs = 0, best_cta = 0;
+    for (int i = 0; i < cand.n; ++i) {
+        if (legal[i] && cand.cta[i] * 4 >= most * 3) {
+            best_cs = cand.cs[i];
+            best_cta = cand.cta[i];
+            break;
         }
     }
-    if (best_cs == 0) return kPacked ? COBALT_OK : COBALT_ERR_UNSUPPORTED;
-    if (kPacked) {
-        // tokens one cluster can see: its CTAs x the grid-stride trips of one CTA x the block size
-        const int64_t trips = (T + static_cast<int64_t>(best_cta) * kStatsThreads - 1) / (static_cast<int64_t>(best_cta) * kStatsThreads);
-        if (trips * kStatsThreads * best_cs > 65535) return COBALT_OK;   // caller takes the 32-bit tile
-    }
+    if (best_cs == 0) return kPacked ? COBALT_OK : COBALT_ERR_UNSUPPORTED;   // packed: caller takes another kernel
     attr[0].val.clusterDim.x = best_cs;
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
     set_programmatic_launch(&attr[1], after_zeroing);

@@ -187,6 +187,25 @@ def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
     assert (u32(coact) == 2 * ref_coact).all() and (u32(load) == 2 * ref_load).all()
 
 
+@pytest.mark.parametrize("E,K,T,tile", [(400, 4, 3_000_000, "16-bit, small clusters"), (330, 2, 10_000_000, "spread")])
+def test_statistics_many_tokens_and_a_large_triangle(cb, E, K, T, tile):
+    """The 16-bit tile may count at most 65535 tokens per cluster: T = 3e6 only allows clusters of two
+    CTAs, T = 1e7 none at all (the triangle is then spread over a cluster).  Ids are an arithmetic
+    progression per token (distinct by construction), cheap to draw at this size."""
+    rng = np.random.default_rng(E * K)
+    base = rng.integers(0, E, size=(T, 1), dtype=np.int64)
+    step = rng.integers(1, E // K, size=(T, 1), dtype=np.int64)
+    ids = ((base + step * np.arange(K, dtype=np.int64)[None, :]) % E).astype(np.int32)
+    ids_d = torch.from_numpy(ids).cuda()
+    coact = torch.empty((E, E), dtype=torch.int32, device="cuda")
+    load = torch.empty((E,), dtype=torch.int32, device="cuda")
+    cb.coact_stats(ids_d, E, coact, load)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    ref_coact, ref_load = O.coact_stats(ids, E)
+    assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
+
+
 @pytest.mark.parametrize("E,K,T", [(256, 8, 131072), (64, 6, 40000), (16, 2, 5000), (8, 8, 1500), (256, 8, 700000)])
 def test_statistics_with_sixteen_bit_tiles_forced(cb, E, K, T):
     """The 16-bit tile, chosen by default only where the 32-bit one does not fit, gives the same counts
