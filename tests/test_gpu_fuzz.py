@@ -2,6 +2,8 @@
 layout, backward), each compared with the oracle.  Shapes are drawn from the supported envelope
 with odd sizes on purpose: non-power-of-two E and D, K from 1 to 16, 1 to 8 nodes, empty slots,
 ragged T."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -13,29 +15,33 @@ from gpu_util import assert_combine_close, bf16_tensor_from_bits, bits_from_bf16
 pytestmark = pytest.mark.gpu
 
 
-def _draw_shape(rng):
+# COBALT_FUZZ_CASES=n runs n cases instead of 24; cases from 24 on draw from a wider envelope
+N_CASES = int(os.environ.get("COBALT_FUZZ_CASES", "24"))
+
+
+def _draw_shape(rng, wide=False):
     N = int(rng.choice([1, 2, 3, 4, 5, 8]))
     Q = int(rng.integers(1, 5))
     G = N * Q
     K = int(rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 12, 16]))
-    E = int(rng.integers(max(K, 2), 200))
+    E = int(rng.integers(max(K, 2), 1025 if wide else 200))
     per = -(-E // G)
     S = per + int(rng.integers(0, 3))
     if E < G:
         S = 1
     while G * S > 4096:
         S -= 1
-    T = int(rng.choice([1, 2, 31, 32, 33, 255, 256, 257, 1000, 2047, 2049, 5000, 9999]))
+    T = int(rng.choice([1, 2, 31, 32, 33, 255, 256, 257, 1000, 2047, 2049, 5000, 9999] + ([20000, 40001] if wide else [])))
     H = 8 * int(rng.integers(1, 40))
     empty = int(rng.integers(0, 3)) if E >= G else 0
     return T, E, K, H, N, Q, S, empty
 
 
-@pytest.mark.parametrize("case", range(24))
+@pytest.mark.parametrize("case", range(N_CASES))
 def test_random_shape(case):
     import paper_2609_36959_b200 as cb
     rng = np.random.default_rng(1000 + case)
-    T, E, K, H, N, Q, S, empty = _draw_shape(rng)
+    T, E, K, H, N, Q, S, empty = _draw_shape(rng, wide=case >= 24)
     w = W.make_custom(T, E, K, H, N, Q, S, seed=500 + case, C=int(rng.integers(1, 6)), p_in=0.6, n_empty=empty)
     seed = int(rng.integers(0, 2**63))
     layout, step = make_step(w, alias_expert_out=False)
