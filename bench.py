@@ -284,6 +284,18 @@ def extra_measurements(args, w, step, cb, torch):
         out["fused_route_index_us"] = None
         out["fused_error"] = str(exc)[:200]
 
+    # the four-stage step with the statistics on a side stream beside the other stages
+    try:
+        n = max(5, min(args.steps, 30))
+        for _ in range(3):
+            step.route(w.seed, overlap_stats=True)
+        out["stats_overlapped_step_ms"] = timed(lambda: step.route(w.seed, overlap_stats=True), n)
+        out["stats_overlapped_step_pairs_per_s"] = w.P / (out["stats_overlapped_step_ms"] * 1e-3)
+        out["sequential_step_ms_same_loop"] = timed(lambda: step.route(w.seed), n)
+    except Exception as exc:
+        out["stats_overlapped_step_ms"] = None
+        out["stats_overlap_error"] = str(exc)[:200]
+
     # the next two blocks allocate one more buffer of the send buffer's size: only with room to spare
     send_bytes = step.send.numel() * 2
 

@@ -64,14 +64,29 @@ class RouteStep:
     def combine(self, flags: int = 0) -> None:
         cb.combine(self.expert_out, self.row_of_pair, self.gate_w, self.y, flags=flags)
 
-    def route(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None) -> None:
-        """stats -> assign -> permute -> [experts(send, expert_out)] -> combine on the current stream."""
-        self.stats()
+    def route(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None,
+              overlap_stats: bool = False) -> None:
+        """stats -> assign -> permute -> [experts(send, expert_out)] -> combine on the current stream.
+
+        Nothing in the step consumes the statistics (they feed the planner of later steps), so with
+        `overlap_stats` they run on a side stream beside the other stages and are joined at the end.
+        """
+        main = torch.cuda.current_stream()
+        if overlap_stats:
+            if not hasattr(self, "_side"):
+                self._side = torch.cuda.Stream()
+            self._side.wait_stream(main)
+            with torch.cuda.stream(self._side):
+                self.stats()
+        else:
+            self.stats()
         self.assign(seed)
         self.permute()
         if experts is not None:
             experts(self.send, self.expert_out)
         self.combine()
+        if overlap_stats:
+            main.wait_stream(self._side)
 
     def route_fused(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None) -> None:
         """The same step with stages 1, 2 and the permutation index fused into one pass over the ids

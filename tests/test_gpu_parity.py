@@ -307,6 +307,24 @@ def test_fused_route_index_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     run_fused_and_compare(cb, w, step, 31337)
 
 
+def test_step_with_statistics_on_a_side_stream(cb):
+    """overlap_stats runs stage 1 beside the others; repeated steps give the results of the oracle."""
+    w = W.make_config("3", T=7001)
+    layout, step = make_step(w)
+    for _ in range(4):
+        step.coact.fill_(5)
+        step.route(w.seed, overlap_stats=True)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    coact, load = O.coact_stats(w.topk_ids, w.E)
+    assert (u32(step.coact) == coact).all() and (u32(step.load) == load).all()
+    r = oracle_assign(w, w.seed)
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    p = O.permute(r["assigned_slot"], w.D, w.hidden_rows())
+    assert (step.row_of_pair.cpu().numpy() == p["row_of_pair"]).all()
+    assert (bits_from_bf16_tensor(step.send) == p["send"]).all()
+
+
 def test_fused_route_step_equals_separate_stages(cb):
     w = W.make_config("3", T=12345)
     layout, step = make_step(w)
