@@ -11,6 +11,7 @@
 // of a cluster (coact_spread_kernel).
 #include <cooperative_groups.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -29,7 +30,7 @@ constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 // most 65535 tokens, so that neither a tile nor the sum of a cluster's tiles can overflow a half.
 template <int KT, bool kPacked>
 __global__ void __launch_bounds__(kStatsThreads)
-coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E,
+coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int tokens_per_trip,
                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(16) uint32_t tri[];   // lower triangle, padded to whole uint4
@@ -38,8 +39,11 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     cg::cluster_group cluster = cg::this_cluster();
 
     // the first token's ids are requested before the tile is cleared so that the two overlap
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    // a CTA takes tokens_per_trip (<= blockDim.x) consecutive tokens per trip: small batches are
+    // spread over more CTAs than they have blocks of 1024 tokens, which shortens every phase
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * tokens_per_trip;
+    int64_t t = static_cast<int>(threadIdx.x) < tokens_per_trip
+                    ? static_cast<int64_t>(blockIdx.x) * tokens_per_trip + threadIdx.x : T;
     int32_t id[KMAX];
     if (t < T) load_token_ids<KT>(topk_ids, t, K, id);
     const int n_vec = (static_cast<int>(tri_entries(E)) + (kPacked ? 7 : 3)) / (kPacked ? 8 : 4);
@@ -208,6 +212,9 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // about one token per thread, never more CTAs than can be co-resident (a second wave of
     // clusters would double the run time), clusters as large as the device schedules well
     int64_t want = (T + kStatsThreads - 1) / kStatsThreads;
+    // batches below 16 blocks still get up to one full cluster (64 tokens per CTA at least): the
+    // shared-memory adds and the merge are then split 16 ways at no extra global reductions
+    if (want < 16) want = std::min<int64_t>(16, (T + 63) / 64);
     if (want < 1) want = 1;
     if (want > n_sm) want = n_sm;
     if (g_tune.stats_max_ctas > 0 && want > g_tune.stats_max_ctas) want = g_tune.stats_max_ctas;
@@ -265,10 +272,14 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // CTA x the block size), which rules out the larger clusters when T is large
     bool legal[5];
     int most = 0;
+    auto tokens_per_trip = [T](int n_cta) {
+        return static_cast<int>(std::min<int64_t>(kStatsThreads, round_up((T + n_cta - 1) / n_cta, 32)));
+    };
     for (int i = 0; i < cand.n; ++i) {
-        const int64_t per_trip = static_cast<int64_t>(cand.cta[i]) * kStatsThreads;
+        const int tpt = tokens_per_trip(cand.cta[i]);
+        const int64_t per_trip = static_cast<int64_t>(cand.cta[i]) * tpt;
         const int64_t trips = (T + per_trip - 1) / per_trip;
-        legal[i] = !kPacked || trips * kStatsThreads * cand.cs[i] <= 65535;
+        legal[i] = !kPacked || trips * tpt * cand.cs[i] <= 65535;
         if (legal[i] && cand.cta[i] > most) most = cand.cta[i];
     }
     // the largest cluster that keeps at least 3/4 of the best CTA count: the merge (distributed
@@ -287,7 +298,7 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
     set_programmatic_launch(&attr[1], after_zeroing);
     cfg.numAttrs = 2;
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, coact, load, err_word));
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, tokens_per_trip(best_cta), coact, load, err_word));
     *launched = true;
     return COBALT_OK;
 }

@@ -247,7 +247,11 @@ __device__ __forceinline__ int tri_row(int idx)
 
 // After a cluster barrier: every CTA owns a contiguous slice of the flat triangle, sums it over
 // all tiles of the cluster with 16-byte distributed-shared-memory loads and merges the sums into
-// coact (both (hi, lo) and (lo, hi)) and load (the diagonal) with global integer reductions.
+// coact and load (the diagonal) with global integer reductions.  Entry (hi, lo) goes out straight
+// from the registers, lanes running along lo.  Its mirror (lo, hi) would put the 32 lanes of such a
+// reduction on 32 different rows of coact, so the sums are also written back into this CTA's own
+// tile (no peer reads that slice) and the mirrors are issued in a second walk whose lanes run along
+// hi, i.e. along a row of coact.
 // The caller must hold a second cluster barrier before any CTA exits.
 template <bool kPacked = false>
 __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E, uint32_t* __restrict__ coact,
@@ -262,13 +266,17 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
     const int csize = static_cast<int>(cluster.num_blocks());
     const int crank = static_cast<int>(cluster.block_rank());
     const int per = (n_vec + csize - 1) / csize;
-    const int v0 = crank * per, v1 = min(n_vec, v0 + per);
+    const int v0 = min(n_vec, crank * per), v1 = min(n_vec, v0 + per);
     for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
         uint4 s = make_uint4(0, 0, 0, 0);
-        for (int r = 0; r < csize; ++r) {
+#pragma unroll 4
+        for (int i = 0; i < csize; ++i) {
+            // every CTA starts at its own tile, so the CTAs of a cluster do not all read one peer at once
+            const int r = (crank + i) % csize;
             const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
             s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;    // packed halves cannot carry (see above)
         }
+        reinterpret_cast<uint4*>(tri)[v] = s;
         const uint32_t word[4] = {s.x, s.y, s.z, s.w};
         const int first = 4 * kPerWord * v;                      // first triangle entry of this vector
         int hi = tri_row(first);
@@ -278,10 +286,25 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
             const uint32_t val = kPacked ? ((word[c >> 1] >> (16 * (c & 1))) & 0xFFFFu) : word[c];
             if (first + c < n_tri && val) {
                 atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], val);
-                if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
-                else atomicAdd(&load[hi], val);
+                if (lo == hi) atomicAdd(&load[hi], val);
             }
             if (++lo > hi) { ++hi; lo = 0; }
+        }
+    }
+    __syncthreads();
+    // mirrors of the slice [f0, f1): it covers (parts of) rows a..b of the triangle
+    const int f0 = 4 * kPerWord * v0, f1 = min(n_tri, 4 * kPerWord * v1);
+    if (f0 >= f1) return;
+    const int a = tri_row(f0), b = tri_row(f1 - 1);
+    const int n_rows = b - a + 1;
+    const int n_walk = n_rows * b;                       // lo in [0, b), hi in [a, b]
+    for (int j = threadIdx.x; j < n_walk; j += blockDim.x) {
+        const int lo = j / n_rows;
+        const int hi = a + (j - lo * n_rows);
+        const int flat = hi * (hi + 1) / 2 + lo;
+        if (lo < hi && flat >= f0 && flat < f1) {
+            const uint32_t val = kPacked ? ((tri[flat >> 1] >> (16 * (flat & 1))) & 0xFFFFu) : tri[flat];
+            if (val) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
         }
     }
 }
