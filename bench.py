@@ -260,6 +260,35 @@ def extra_measurements(args, w, step, cb, torch):
         out["index_stages_graph_replay_warm_us"] = None
         out["graph_replay_error"] = str(exc)[:200]
 
+    # What the timing method itself costs: a pair of events around nothing, around one kernel that
+    # only clears 257 KB (coact_stats with an empty batch), and around the statistics call at this
+    # batch size, each behind a 256 MB fill so that the launches are queued before the GPU gets to them
+    try:
+        fill = torch.empty(256 << 20, dtype=torch.uint8, device=step.x.device)
+        none = torch.empty((0, w.K), dtype=torch.int32, device=step.x.device)
+
+        def cold_us(fn, n=30):
+            best = []
+            for _ in range(n + 3):
+                fill.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                torch.cuda.synchronize()
+                best.append(e0.elapsed_time(e1) * 1e3)
+            return float(np.median(best[3:]))
+
+        out["timing_floor_us"] = {
+            "event_pair_alone": cold_us(lambda: None),
+            "one_clearing_kernel": cold_us(lambda: cb.coact_stats(none, w.E, step.coact, step.load)),
+            "coact_stats": cold_us(step.stats),
+        }
+        del fill
+    except Exception as exc:
+        out["timing_floor_us"] = None
+        out["timing_floor_error"] = str(exc)[:200]
+
     # the same step with stages 1, 2 and the permutation index fused into one pass over the ids
     try:
         n = max(5, min(args.steps, 30))
