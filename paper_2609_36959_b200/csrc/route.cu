@@ -49,7 +49,7 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
                    uint32_t* __restrict__ coact, uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot,
                    uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
                    uint32_t* __restrict__ chunk_ws, int n_chunks, int tri_words, int tab_words,
-                   int tokens_per_round, uint32_t* __restrict__ err_word)
+                   int chunks_per_cta, uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t* tri = smem;
@@ -62,18 +62,17 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
     cg::cluster_group cluster = cg::this_cluster();
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the scan kernel may be scheduled early
-    // a CTA takes tokens_per_round (1 to 4 chunks of 256) consecutive tokens per round: small batches
-    // are spread over more CTAs than they have blocks of 1024 tokens
-    const int64_t grid_tokens_per_round = static_cast<int64_t>(gridDim.x) * tokens_per_round;
-    const int n_rounds = static_cast<int>((T + grid_tokens_per_round - 1) / grid_tokens_per_round);
-    const bool has_token = static_cast<int>(threadIdx.x) < tokens_per_round;
-    const int chunks_per_round = tokens_per_round / kRouteChunkTokens;
+    // a CTA owns chunks_per_cta consecutive chunks of 256 tokens (the batch cut evenly over the grid)
+    // and takes them in rounds of up to four, one token per thread
+    const int chunk_lo = min(n_chunks, static_cast<int>(blockIdx.x) * chunks_per_cta);
+    const int chunk_hi = min(n_chunks, chunk_lo + chunks_per_cta);
+    const int n_rounds = (chunk_hi - chunk_lo + kRouteChunksPerRound - 1) / kRouteChunksPerRound;
     // the first round's loads go out before the shared-memory set-up so that the two overlap
     int32_t id[KMAX], out[KMAX];
     int32_t s_t = src_uniform;
     {
-        const int64_t t0 = static_cast<int64_t>(blockIdx.x) * tokens_per_round + threadIdx.x;
-        if (n_rounds > 0 && has_token && t0 < T) {
+        const int64_t t0 = static_cast<int64_t>(chunk_lo) * kRouteChunkTokens + threadIdx.x;
+        if (static_cast<int>(threadIdx.x) < (chunk_hi - chunk_lo) * kRouteChunkTokens && t0 < T) {
             load_token_ids<KT>(topk_ids, t0, K, id);
             if (src_rank) s_t = __ldg(src_rank + t0);
         }
@@ -86,9 +85,10 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
 
     uint32_t cost_sum = 0, naive_sum = 0;
     for (int round = 0; round < n_rounds; ++round) {
-        const int64_t base = (static_cast<int64_t>(round) * gridDim.x + blockIdx.x) * tokens_per_round;
-        const int64_t t = base + threadIdx.x;
-        if (has_token && t < T) {
+        const int first_chunk = chunk_lo + round * kRouteChunksPerRound;
+        const int chunks_this_round = min(kRouteChunksPerRound, chunk_hi - first_chunk);
+        const int64_t t = static_cast<int64_t>(first_chunk) * kRouteChunkTokens + threadIdx.x;
+        if (static_cast<int>(threadIdx.x) < chunks_this_round * kRouteChunkTokens && t < T) {
             if (round > 0) {
                 load_token_ids<KT>(topk_ids, t, K, id);
                 if (src_rank) s_t = __ldg(src_rank + t);
@@ -118,11 +118,9 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
         }
         __syncthreads();
         // hand this round's chunk histograms to the scan (every chunk row is written, zeros included)
-        const int64_t first_chunk = base / kRouteChunkTokens;
-        for (int i = threadIdx.x; i < chunks_per_round * D; i += blockDim.x) {
+        for (int i = threadIdx.x; i < chunks_this_round * D; i += blockDim.x) {
             const int g = i / D, d = i - g * D;
-            const int64_t chunk = first_chunk + g;
-            if (chunk < n_chunks) chunk_ws[static_cast<size_t>(d) * n_chunks + chunk] = chist[i];
+            chunk_ws[static_cast<size_t>(d) * n_chunks + first_chunk + g] = chist[i];
             chist[i] = 0;
         }
         __syncthreads();
@@ -152,15 +150,6 @@ struct RouteLaunch {
     int ctas;
 };
 
-// Tokens a CTA takes per round: whole 1024-token blocks, except that batches under 16 such blocks
-// are cut into 256- or 512-token pieces so that they still fill one cluster.
-static int route_tokens_per_round(int64_t T)
-{
-    if (T <= 16 * kRouteChunkTokens) return kRouteChunkTokens;
-    if (T <= 32 * kRouteChunkTokens) return 2 * kRouteChunkTokens;
-    return kRouteThreads;
-}
-
 template <int KT>
 static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n_sm, RouteLaunch* out)
 {
@@ -169,8 +158,7 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
     static std::map<std::tuple<int, int, int, int64_t>, RouteLaunch> cache;
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
-    const int tpr = route_tokens_per_round(T);
-    int64_t want = (T + tpr - 1) / tpr;
+    int64_t want = (T + kRouteChunkTokens - 1) / kRouteChunkTokens;   // one chunk per CTA while CTAs last
     if (want < 1) want = 1;
     if (want > n_sm) want = n_sm;
     const auto key = std::make_tuple(dev, lv.E, lv.D, want * 1024 + lv.words % 1024);
@@ -278,7 +266,7 @@ static int launch_route(const RouteArgs& a)
                                        static_cast<uint32_t>(a.seed >> 32), a.coact, a.load, a.assigned_slot,
                                        a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.chunk_ws,
                                        a.n_chunks, static_cast<int>(sm.tri_words), static_cast<int>(sm.tab_words),
-                                       route_tokens_per_round(a.T), a.err_word));
+                                       (a.n_chunks + how.ctas - 1) / how.ctas, a.err_word));
     return COBALT_OK;
 }
 
