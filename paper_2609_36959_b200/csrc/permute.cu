@@ -35,6 +35,33 @@ ChunkPlan plan_chunks(int64_t P)
     return c;
 }
 
+// The same plan for batches with fewer chunks than the device has SMs: the chunk is shrunk (down to
+// half, in steps of one CTA's threads) so that more SMs share the work.  Measured at P = 32768:
+// 15.3 -> 13.3 us.  With more chunks than SMs the smaller chunks only lengthen the scan.
+// The result does not depend on the chunking.
+constexpr int kBalancedMinChunk = kMinChunk / 2;
+
+static ChunkPlan plan_chunks_balanced(int64_t P, int n_sm)
+{
+    ChunkPlan c = plan_chunks(P);
+    if (c.chunk != kMinChunk || c.n_chunks >= n_sm || P < 1) return c;
+    int64_t chunk = static_cast<int64_t>(round_up((P + n_sm - 1) / n_sm, kPermThreads));
+    if (chunk < kBalancedMinChunk) chunk = kBalancedMinChunk;
+    if (chunk > kMinChunk) chunk = kMinChunk;
+    c.chunk = static_cast<int>(chunk);
+    c.n_chunks = static_cast<int>((P + chunk - 1) / chunk);
+    return c;
+}
+
+// Most chunks plan_chunks_balanced can return for P pairs on any device.
+static int max_balanced_chunks(int64_t P)
+{
+    const ChunkPlan c = plan_chunks(P);
+    if (c.chunk != kMinChunk) return c.n_chunks;
+    const int64_t n = (P + kBalancedMinChunk - 1) / kBalancedMinChunk;
+    return static_cast<int>(n < 1 ? 1 : n);
+}
+
 // ---- K1 -----------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kPermThreads)
 perm_hist_kernel(const int32_t* __restrict__ slot, int64_t P, int D, int chunk, int n_chunks,
@@ -723,8 +750,7 @@ extern "C" {
 size_t cobalt_permute_workspace_bytes(int64_t T, int32_t K, int32_t D)
 {
     if (check_index_args(T, K, D) != COBALT_OK) return 0;
-    const ChunkPlan c = plan_chunks(T * K);
-    return round_up(static_cast<size_t>(D) * c.n_chunks * sizeof(uint32_t), 256);
+    return round_up(static_cast<size_t>(D) * max_balanced_chunks(T * K) * sizeof(uint32_t), 256);
 }
 
 int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
@@ -744,7 +770,10 @@ int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t P = T * K;
-    const ChunkPlan c = plan_chunks(P);
+    int n_sm = 0;
+    rc = sm_count(&n_sm);
+    if (rc != COBALT_OK) return rc;
+    const ChunkPlan c = plan_chunks_balanced(P, n_sm);
     uint32_t* ws = static_cast<uint32_t*>(workspace);
     uint32_t* err_word = nullptr;
     rc = device_error_word(&err_word);
