@@ -538,9 +538,13 @@ def run_cobalt(args):
             step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        # the steps are queued back to back without joining the copy-out stream in between, so a
+        # step's inputs start moving in while the previous step's last results move out; the
+        # closing event is recorded after the last copy out has been joined
         e0.record()
-        for _ in range(n_e2e):
-            step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
+        for i in range(n_e2e):
+            step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h,
+                            join=(i == n_e2e - 1))
         e1.record()
         barrier()
         e2e_ms = max_over_ranks(e0.elapsed_time(e1), "cuda") / n_e2e

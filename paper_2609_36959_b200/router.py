@@ -102,7 +102,7 @@ class RouteStep:
     # -- the same step from pinned host memory ----------------------------------------------
     def route_host(self, seed: int, ids_h: torch.Tensor, w_h: torch.Tensor, src_h: torch.Tensor,
                    x_h: torch.Tensor, y_h: torch.Tensor, coact_h: torch.Tensor, load_h: torch.Tensor,
-                   slot_load_h: torch.Tensor, totals_h: torch.Tensor, chunks: int = 16) -> None:
+                   slot_load_h: torch.Tensor, totals_h: torch.Tensor, chunks: int = 16, join: bool = True) -> None:
         """One step with inputs and results in pinned host memory.
 
         The gating output is small and goes first, so statistics, assignment and the permutation
@@ -111,13 +111,22 @@ class RouteStep:
         being no expert computation between dispatch and combine here) combined on the compute
         stream, and its result copied out on a third stream, so both copy directions and the
         kernels overlap.  The C entry points take plain pointers, so a block is just an offset.
+
+        With `join` the current stream waits for the last copy out, so the host buffers are valid once
+        it has been synchronised.  Without it the call returns with copies still queued and
+        `wait_host_results()` (or a device synchronise) must come before the host buffers are read;
+        the next call may then start copying its inputs in while this one's last results are still
+        on their way out, which keeps both copy directions busy across steps.
         """
         main = torch.cuda.current_stream()
         if not hasattr(self, "_h2d"):
             self._h2d, self._d2h = torch.cuda.Stream(), torch.cuda.Stream()
         h2d, d2h = self._h2d, self._d2h
-        h2d.wait_stream(main)          # the previous step may still be reading x / writing y
+        h2d.wait_stream(main)          # the previous step may still be reading x and the gating output
         d2h.wait_stream(main)
+        # results of the previous call that may still be on their way out must not be overwritten
+        prev_small = getattr(self, "_small_copied", None)
+        prev_y = getattr(self, "_y_copied", [])
         T, K = self.T, self.K
         chunks = max(1, min(chunks, T)) if T > 0 else 1
         # block starts on multiples of 4 tokens keep every offset pointer 16-byte aligned for any K
@@ -139,6 +148,11 @@ class RouteStep:
                 ev.record(h2d)
                 ready.append(ev)
         main.wait_event(gating_ready)
+        if prev_small is not None:
+            main.wait_event(prev_small)
+        if len(prev_y) != chunks:      # another block structure: wait for everything that is queued
+            main.wait_stream(d2h)
+            prev_y = []
         self.stats()
         self.assign(seed)
         cb.permute_index(self.assigned_slot, self.D, self.dest_counts, self.dest_offsets, self.row_of_pair,
@@ -151,6 +165,9 @@ class RouteStep:
             load_h.copy_(self.load, non_blocking=True)
             slot_load_h.copy_(self.slot_load, non_blocking=True)
             totals_h.copy_(self.totals, non_blocking=True)
+            self._small_copied = torch.cuda.Event()
+            self._small_copied.record(d2h)
+        y_copied = [None] * chunks
         for c in range(chunks):
             t0, t1 = bounds[c], bounds[c + 1]
             if t1 == t0:
@@ -159,13 +176,27 @@ class RouteStep:
             rop = self.row_of_pair[t0 * K:t1 * K]
             # rows index the whole send buffer, so the full buffers are passed with a token offset
             cb.permute_rows_block(self.x, rop, K, self.send, t0, t1)
+            if prev_y and prev_y[c] is not None:
+                main.wait_event(prev_y[c])
             cb.combine_block(self.expert_out, rop, self.gate_w, self.y, t0, t1)
             done = torch.cuda.Event()
             done.record(main)
             with torch.cuda.stream(d2h):
                 d2h.wait_event(done)
                 y_h[t0:t1].copy_(self.y[t0:t1], non_blocking=True)
-        main.wait_stream(d2h)
+                y_copied[c] = torch.cuda.Event()
+                y_copied[c].record(d2h)
+        self._y_copied = y_copied
+        self._host_done = torch.cuda.Event()
+        self._host_done.record(d2h)
+        if join:
+            main.wait_stream(d2h)
+
+    def wait_host_results(self) -> None:
+        """Block the host until the results of the last route_host call are in the host buffers."""
+        done = getattr(self, "_host_done", None)
+        if done is not None:
+            done.synchronize()
 
     def h2d_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.topk_ids, self.gate_w, self.src_rank, self.x))

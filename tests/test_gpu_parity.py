@@ -510,6 +510,54 @@ def test_host_driven_step_matches_the_resident_step(cb, name, T, chunks):
     assert torch.equal(step.row_of_pair, ref["row_of_pair"])
 
 
+def test_host_driven_steps_queued_without_joining(cb):
+    """Three different batches through route_host(join=False), queued back to back into separate host
+    buffers: a step starts while the one before still copies results out, and nothing is overwritten
+    before it has been copied.  Each batch must equal its own resident step."""
+    T, chunks = 20003, 8
+    w = W.make_config("3", T=T)
+    x_bits = w.hidden_rows()
+    layout, step = make_step(w)
+    seeds = [11, 22, 33]
+    host, refs = [], []
+    for i, seed in enumerate(seeds):
+        # batch i: tokens rotated by 1000 i, and its first 500 (i + 1) tokens all routed like token 0
+        ids = np.roll(w.topk_ids, 1000 * i, axis=0).copy()
+        ids[:500 * (i + 1)] = ids[0]
+        gate = np.roll(w.gate_w, 1000 * i, axis=0).copy()
+        src = np.roll(w.src_rank, 77 * i).copy()
+        x = np.roll(x_bits, 1000 * i, axis=0).copy()
+        step.topk_ids.copy_(torch.from_numpy(ids))
+        step.gate_w.copy_(torch.from_numpy(gate))
+        step.src_rank.copy_(torch.from_numpy(src))
+        step.x.copy_(bf16_tensor_from_bits(x, "cpu"))
+        step.route(seed)
+        torch.cuda.synchronize()
+        refs.append({k: getattr(step, k).cpu() for k in ("y", "coact", "load", "slot_load", "totals")})
+        host.append({
+            "ids": torch.from_numpy(ids).pin_memory(), "w": torch.from_numpy(gate).pin_memory(),
+            "src": torch.from_numpy(src).pin_memory(), "x": bf16_tensor_from_bits(x, "cpu").pin_memory(),
+            "y": torch.zeros((T, w.H), dtype=torch.bfloat16).pin_memory(),
+            "coact": torch.zeros((w.E, w.E), dtype=torch.int32).pin_memory(),
+            "load": torch.zeros((w.E,), dtype=torch.int32).pin_memory(),
+            "sl": torch.zeros((w.D,), dtype=torch.int32).pin_memory(),
+            "tot": torch.zeros((2,), dtype=torch.int64).pin_memory()})
+    assert not torch.equal(refs[0]["coact"], refs[1]["coact"]) and not torch.equal(refs[1]["y"], refs[2]["y"])
+    for buf in (step.x, step.y, step.send, step.topk_ids, step.coact):
+        buf.zero_()
+    torch.cuda.synchronize()
+    for h, seed in zip(host, seeds):
+        step.route_host(seed, h["ids"], h["w"], h["src"], h["x"], h["y"], h["coact"], h["load"], h["sl"],
+                        h["tot"], chunks=chunks, join=False)
+    step.wait_host_results()
+    for h, ref in zip(host, refs):
+        assert torch.equal(h["y"].view(torch.int16), ref["y"].view(torch.int16))
+        assert torch.equal(h["coact"], ref["coact"]) and torch.equal(h["load"], ref["load"])
+        assert torch.equal(h["sl"], ref["slot_load"]) and torch.equal(h["tot"], ref["totals"])
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+
+
 # ---------------------------------------------------------------------------------------------
 # bad data and bad arguments: flagged, never faulting
 # ---------------------------------------------------------------------------------------------
