@@ -260,6 +260,20 @@ def extra_measurements(args, w, step, cb, torch):
         out["index_stages_graph_replay_warm_us"] = None
         out["graph_replay_error"] = str(exc)[:200]
 
+    # each index stage warm: 50 calls back to back between one pair of events, inputs L2-resident,
+    # launches queued ahead of the GPU (what a stage costs when the gating kernel has just written the ids)
+    try:
+        out["index_stages_warm_us"] = {
+            "coact_stats": timed(step.stats, 50) * 1e3,
+            "assign": timed(lambda: step.assign(w.seed), 50) * 1e3,
+            "permute_index": timed(lambda: cb.permute_index(step.assigned_slot, w.D, step.dest_counts,
+                                                            step.dest_offsets, step.row_of_pair, step.pair_of_row,
+                                                            step.workspace), 50) * 1e3,
+        }
+    except Exception as exc:
+        out["index_stages_warm_us"] = None
+        out["index_stages_warm_error"] = str(exc)[:200]
+
     # What the timing method itself costs: a pair of events around nothing, around one kernel that
     # only clears 257 KB (coact_stats with an empty batch), and around the statistics call at this
     # batch size, each behind a 256 MB fill so that the launches are queued before the GPU gets to them
@@ -515,7 +529,8 @@ def run_cobalt(args):
     clocks = sampler.stop(t_epoch0, t_epoch0 + t_wall) if rank == 0 else None
 
     total_ms = ev[0][0].elapsed_time(ev[-1][5])
-    stage_ms = {n: sum(e[i].elapsed_time(e[i + 1]) for e in ev) / args.steps for i, n in enumerate(names)}
+    per_step = {n: [e[i].elapsed_time(e[i + 1]) for e in ev] for i, n in enumerate(names)}
+    stage_ms = {n: sum(v) / args.steps for n, v in per_step.items()}
     err_bits = cb.read_and_clear_device_error()
 
     ms_per_step = max_over_ranks(total_ms, "cuda") / args.steps
@@ -557,7 +572,8 @@ def run_cobalt(args):
         stages = {}
         for n in names:
             gbs = sb[n] / (stage_ms[n] * 1e-3) / 1e9
-            stages[n] = {"ms": stage_ms[n], "bytes": sb[n], "gbs": gbs, "frac": gbs / peak,
+            stages[n] = {"ms": stage_ms[n], "ms_median": statistics.median(per_step[n]), "ms_min": min(per_step[n]),
+                         "bytes": sb[n], "gbs": gbs, "frac": gbs / peak,
                          "frac_of_nominal_8TBs": gbs / 8000.0,
                          "frac_of_same_run_copy": (gbs / extras["same_run_copy_gbs"]
                                                    if extras.get("same_run_copy_gbs") else None),
