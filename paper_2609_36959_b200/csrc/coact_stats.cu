@@ -7,8 +7,9 @@
 // all CTAs of the cluster through distributed shared memory and merges the result into global
 // memory with integer reductions, mirroring (hi, lo) to (lo, hi) and writing the diagonal to
 // `load` as well.  Only integer adds are used, so the result is independent of scheduling.
-// Expert counts whose triangle does not fit in one CTA's shared memory spread it over the CTAs
-// of a cluster (coact_spread_kernel).
+// Expert counts whose triangle does not fit in one CTA's shared memory take 16-bit counters, two per
+// word (E <= 452, while a cluster sees at most 65535 tokens), else spread the triangle over the
+// CTAs of a cluster (coact_spread_kernel), else add straight to global memory.
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -38,9 +39,9 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     const int K = (KT > 0) ? KT : K_rt;
     cg::cluster_group cluster = cg::this_cluster();
 
-    // the first token's ids are requested before the tile is cleared so that the two overlap
-    // a CTA takes tokens_per_cta consecutive tokens (the batch cut evenly over the grid, so that no
-    // cluster is left with a second pass over a remainder while the others wait at the barrier)
+    // A CTA takes tokens_per_cta consecutive tokens (the batch cut evenly over the grid, so that no
+    // cluster is left with a second pass over a remainder while the others wait at the barrier).
+    // The first token's ids are requested before the tile is cleared so that the two overlap.
     const int64_t t_end = min(T, (static_cast<int64_t>(blockIdx.x) + 1) * tokens_per_cta);
     int64_t t = static_cast<int64_t>(blockIdx.x) * tokens_per_cta + threadIdx.x;
     int32_t id[KMAX];
