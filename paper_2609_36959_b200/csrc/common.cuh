@@ -34,7 +34,7 @@ struct Tuning {
     int rows_per_sm = 0;            // cap on CTAs per SM (0 = as many as shared memory allows)
     int rows_vec_per_sm = 0;        // vector row mover: CTAs per SM (0 = one CTA per token)
     int rows_hint = 0;              // 1 = evict-first L2 hints on the bulk copies
-    int stats_max_ctas = 0;         // statistics kernel: cap on CTAs (0 = one per 1024 tokens, at most the SM count)
+    int stats_max_ctas = 0;         // statistics kernel: cap on CTAs (0 = as many as can be co-resident)
     int stats_cluster = 0;          // statistics kernel: force this cluster size (0 = pick)
     int stats_tokens_per_cta = 0;   // statistics kernel: tokens per CTA the grid is sized for (0 = 256)
     int stats_packed = -1;          // statistics kernel: 16-bit tile (-1 = only where the 32-bit tile does not fit, 0 = never, 1 = whenever legal)
