@@ -8,8 +8,9 @@
 // memory with integer reductions, mirroring (hi, lo) to (lo, hi) and writing the diagonal to
 // `load` as well.  Only integer adds are used, so the result is independent of scheduling.
 // Expert counts whose triangle does not fit in one CTA's shared memory take 16-bit counters, two per
-// word (E <= 452, while a cluster sees at most 65535 tokens), else spread the triangle over the
-// CTAs of a cluster (coact_spread_kernel), else add straight to global memory.
+// word (E <= 452, while a cluster sees at most 65535 tokens); beyond that the triangle is split
+// over 2 to 8 CTAs that are fed the same tokens; few tokens over a large matrix go straight to
+// global memory.
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -29,10 +30,14 @@ constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 
 // kPacked: 16-bit counters, two per word.  The launcher selects it only when one CLUSTER sees at
 // most 65535 tokens, so that neither a tile nor the sum of a cluster's tiles can overflow a half.
-template <int KT, bool kPacked>
+// kSplit (E > 452): the triangle is cut into `parts` runs of part_entries flat entries; `parts`
+// consecutive CTAs form a group that is fed the same tokens, each CTA adding only the pairs that
+// fall into its own run.  All adds stay in the CTA's own shared memory.
+template <int KT, bool kPacked, bool kSplit>
 __global__ void __launch_bounds__(kStatsThreads)
-coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int tokens_per_cta,
-                  uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
+coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int tokens_per_cta, int parts,
+                  int part_entries, uint32_t* __restrict__ coact, uint32_t* __restrict__ load,
+                  uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(16) uint32_t tri[];   // lower triangle, padded to whole uint4
     constexpr int KMAX = TokenShape<KT>::KMAX;
@@ -42,29 +47,32 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
     // A CTA takes tokens_per_cta consecutive tokens (the batch cut evenly over the grid, so that no
     // cluster is left with a second pass over a remainder while the others wait at the barrier).
     // The first token's ids are requested before the tile is cleared so that the two overlap.
-    const int64_t t_end = min(T, (static_cast<int64_t>(blockIdx.x) + 1) * tokens_per_cta);
-    int64_t t = static_cast<int64_t>(blockIdx.x) * tokens_per_cta + threadIdx.x;
+    const int64_t group = kSplit ? blockIdx.x / parts : blockIdx.x;     // CTAs of a group share their tokens
+    const int first = kSplit ? static_cast<int>(blockIdx.x % parts) * part_entries : 0;
+    const int count = kSplit ? min(part_entries, static_cast<int>(tri_entries(E)) - first) : static_cast<int>(tri_entries(E));
+    const int64_t t_end = min(T, (group + 1) * tokens_per_cta);
+    int64_t t = group * tokens_per_cta + threadIdx.x;
     int32_t id[KMAX];
     if (t < t_end) load_token_ids<KT>(topk_ids, t, K, id);
-    const int n_vec = (static_cast<int>(tri_entries(E)) + (kPacked ? 7 : 3)) / (kPacked ? 8 : 4);
+    const int n_vec = ((kSplit ? part_entries : count) + (kPacked ? 7 : 3)) / (kPacked ? 8 : 4);
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     while (t < t_end) {
         const uint32_t bad = check_token_ids<KT>(id, K, E);
         if (bad) flag_error(err_word, bad);
-        else add_token_to_triangle<KT, kPacked>(tri, id, K);
+        else add_token_to_triangle<KT, kPacked, kSplit>(tri, id, K, first, count);
         t += blockDim.x;
         if (t < t_end) load_token_ids<KT>(topk_ids, t, K, id);
     }
 
     cluster.sync();            // every tile of the cluster is complete
     wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
-    merge_triangle_over_cluster<kPacked>(tri, E, coact, load);
+    merge_triangle_over_cluster<kPacked>(tri, E, coact, load, kSplit ? parts : 1, part_entries);
     cluster.sync();            // no CTA may exit while a peer still reads its tile
 }
 
-// Fallback for expert counts whose triangle does not fit in shared memory.
+// Every pair straight to global memory: few pairs over a large matrix, and the last resort.
 __global__ void __launch_bounds__(256)
 coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int E,
                     uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
@@ -86,126 +94,35 @@ coact_global_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K, int 
     }
 }
 
-// Expert counts whose triangle exceeds one CTA's shared memory: the triangle of a CLUSTER is
-// spread over its CTAs (flat index idx lives in CTA idx mod C at word idx / C, so that the hot
-// low-numbered entries do not pile onto one CTA) and every CTA adds its own tokens' pairs with
-// shared-memory atomics that may land in a peer's shared memory.  After a cluster barrier each CTA
-// merges the words it owns into global memory.  E = 1024 needs 2.1 MB per cluster: 16 CTAs x 131 KB.
-template <int KT>
-__global__ void __launch_bounds__(kStatsThreads)
-coact_spread_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int log2_c, int words_per_cta,
-                    uint32_t* __restrict__ coact, uint32_t* __restrict__ load, uint32_t* __restrict__ err_word)
-{
-    extern __shared__ __align__(16) uint32_t part[];   // this CTA's share of the cluster's triangle
-    constexpr int KMAX = TokenShape<KT>::KMAX;
-    const int K = (KT > 0) ? KT : K_rt;
-    cg::cluster_group cluster = cg::this_cluster();
-    const uint32_t c_mask = (1u << log2_c) - 1u;
-
-    for (int i = threadIdx.x; i < words_per_cta; i += blockDim.x) part[i] = 0;
-    cluster.sync();            // every share is cleared before any peer adds to it
-
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    for (int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; t < T; t += stride) {
-        int32_t id[KMAX];
-        load_token_ids<KT>(topk_ids, t, K, id);
-        const uint32_t bad = check_token_ids<KT>(id, K, E);
-        if (bad) {
-            flag_error(err_word, bad);
-            continue;
-        }
-#pragma unroll
-        for (int a = 0; a < KMAX; ++a) {
-#pragma unroll
-            for (int b = a; b < KMAX; ++b) {
-                if (b < K) {
-                    const uint32_t hi = max(id[a], id[b]), lo = min(id[a], id[b]);
-                    const uint32_t idx = hi * (hi + 1) / 2 + lo;
-                    atomicAdd(cluster.map_shared_rank(part, idx & c_mask) + (idx >> log2_c), 1u);
-                }
-            }
-        }
-    }
-    cluster.sync();            // all adds of the cluster have landed
-    wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
-    const uint32_t n_tri = static_cast<uint32_t>(tri_entries(E));
-    const uint32_t crank = cluster.block_rank();
-    for (int l = threadIdx.x; l < words_per_cta; l += blockDim.x) {
-        const uint32_t v = part[l];
-        const uint32_t idx = (static_cast<uint32_t>(l) << log2_c) | crank;
-        if (v && idx < n_tri) {
-            const int hi = tri_row(static_cast<int>(idx));
-            const int lo = static_cast<int>(idx) - hi * (hi + 1) / 2;
-            atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], v);
-            if (lo != hi) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], v);
-            else atomicAdd(&load[hi], v);
-        }
-    }
-}
-
-template <int KT>
-static int launch_spread(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                         uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
-{
-    *launched = false;
-    auto kernel = coact_spread_kernel<KT>;
-    const size_t n_tri = tri_entries(E);
-    int log2_c = 1;
-    while (log2_c < 4 && round_up((n_tri + (1u << log2_c) - 1) >> log2_c, 4) * sizeof(uint32_t) > kStatsMaxTileBytes / 2)
-        ++log2_c;                                    // shares of <= 100 KB when possible (two CTAs per SM)
-    while (log2_c <= 4 && round_up((n_tri + (1u << log2_c) - 1) >> log2_c, 4) * sizeof(uint32_t) > kStatsMaxTileBytes)
-        ++log2_c;
-    if (log2_c > 3) return COBALT_OK;   // 16 shares measured slower than plain global atomics: caller falls back
-    const int c = 1 << log2_c;
-    const int words = static_cast<int>(round_up((n_tri + c - 1) / c, 4));
-    const size_t smem = static_cast<size_t>(words) * sizeof(uint32_t);
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return COBALT_OK;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[2];
-    cfg.blockDim = dim3(kStatsThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = c;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3(c);
-    int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
-        (void)cudaGetLastError();
-        return COBALT_OK;
-    }
-    int64_t want = (T + kStatsThreads - 1) / kStatsThreads;      // about one token per thread
-    int64_t clusters = (want + c - 1) / c;
-    if (clusters > max_clusters) clusters = max_clusters;
-    if (clusters * c > 2ll * n_sm) clusters = 2ll * n_sm / c;
-    if (clusters < 1) clusters = 1;
-    cfg.gridDim = dim3(static_cast<unsigned>(clusters * c));
-    set_programmatic_launch(&attr[1], after_zeroing);
-    cfg.numAttrs = 2;
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, log2_c, words, coact, load, err_word));
-    *launched = true;
-    return COBALT_OK;
-}
-
 static size_t tile_bytes(int E, bool packed)
 {
     return round_up((packed ? (tri_entries(E) + 1) / 2 : tri_entries(E)) * sizeof(uint32_t), 16);
 }
 
-template <int KT, bool kPacked>
+// Split tiles (16-bit counters): the fewest parts, a power of two up to 8, whose runs fit one CTA.
+static int split_parts(int E, int* part_entries)
+{
+    for (int parts = 2; parts <= 8; parts *= 2) {
+        const size_t per = round_up((tri_entries(E) + parts - 1) / parts, 8);     // whole 16-byte vectors
+        if (per * 2 <= kStatsMaxTileBytes) {
+            *part_entries = static_cast<int>(per);
+            return parts;
+        }
+    }
+    return 0;
+}
+
+template <int KT, bool kPacked, bool kSplit>
 static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
                        uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
 {
+    static_assert(kPacked || !kSplit, "split tiles use 16-bit counters");
     *launched = false;
-    auto kernel = coact_tile_kernel<KT, kPacked>;
-    const size_t smem = tile_bytes(E, kPacked);
+    auto kernel = coact_tile_kernel<KT, kPacked, kSplit>;
+    int part_entries = 0;
+    const int parts = kSplit ? split_parts(E, &part_entries) : 1;
+    if (parts == 0) return COBALT_OK;
+    const size_t smem = kSplit ? static_cast<size_t>(part_entries) * 2 : tile_bytes(E, kPacked);
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
 
@@ -219,8 +136,10 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // shared-memory adds and the merge are then split 16 ways at no extra global reductions
     if (want < 16) want = std::min<int64_t>(16, (T + 63) / 64);
     if (want < 1) want = 1;
+    want *= parts;                      // `parts` CTAs per group of tokens
     if (want > n_sm) want = n_sm;
     if (g_tune.stats_max_ctas > 0 && want > g_tune.stats_max_ctas) want = g_tune.stats_max_ctas;
+    if (want < parts) want = parts;
 
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
@@ -252,7 +171,7 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     }
     if (!cached) {
         for (int cs = 16; cs >= 1; cs >>= 1) {
-            if (cs > want) continue;
+            if (cs > want || cs % parts != 0) continue;
             if (g_tune.stats_cluster > 0 && cs != g_tune.stats_cluster) continue;
             attr[0].val.clusterDim.x = cs;
             cfg.gridDim = dim3(cs);
@@ -275,9 +194,12 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // rules out the larger clusters when T is large
     bool legal[5];
     int most = 0;
-    auto tokens_per_cta = [T](int n_cta) { return static_cast<int64_t>(round_up((T + n_cta - 1) / n_cta, 32)); };
+    auto tokens_per_cta = [T, parts](int n_cta) {      // tokens of one group of `parts` CTAs
+        const int groups = n_cta / parts;
+        return static_cast<int64_t>(round_up((T + groups - 1) / groups, 32));
+    };
     for (int i = 0; i < cand.n; ++i) {
-        legal[i] = !kPacked || tokens_per_cta(cand.cta[i]) * cand.cs[i] <= 65535;
+        legal[i] = !kPacked || tokens_per_cta(cand.cta[i]) * (cand.cs[i] / parts) <= 65535;
         if (legal[i] && cand.cta[i] > most) most = cand.cta[i];
     }
     // the largest cluster that keeps at least 3/4 of the best CTA count: the merge (distributed
@@ -296,13 +218,14 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
     set_programmatic_launch(&attr[1], after_zeroing);
     cfg.numAttrs = 2;
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, static_cast<int>(tokens_per_cta(best_cta)), coact, load,
-                                       err_word));
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, static_cast<int>(tokens_per_cta(best_cta)), parts,
+                                       part_entries, coact, load, err_word));
     *launched = true;
     return COBALT_OK;
 }
 
-// The 16-bit tile when it is allowed and wanted, else the 32-bit tile when it fits.
+// The 16-bit tile when it is allowed and wanted, else the 32-bit tile when it fits, else split
+// 16-bit tiles.
 template <int KT>
 static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
                         uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
@@ -312,11 +235,13 @@ static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* c
     const bool fits16 = tile_bytes(E, true) <= kStatsMaxTileBytes;
     const bool want16 = g_tune.stats_packed > 0 || (g_tune.stats_packed < 0 && !fits32);
     if (fits16 && want16) {
-        const int rc = launch_tile<KT, true>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
+        const int rc = launch_tile<KT, true, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream,
+                                                    launched);
         if (rc != COBALT_OK || *launched) return rc;
     }
-    if (!fits32) return COBALT_OK;
-    return launch_tile<KT, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
+    if (fits32)
+        return launch_tile<KT, false, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
+    return launch_tile<KT, true, true>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
 }
 
 }  // namespace cobalt
@@ -359,27 +284,24 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     rc = sm_count(&n_sm);
     if (rc != COBALT_OK) return rc;
 
+    // Few pairs over a large matrix (the split tiles' merge costs about 20 us + 22 us (E/1024)^2 whatever
+    // the batch, a global atomic about 1/45 ns): every pair straight to global memory.
+    const bool large = tile_bytes(E, true) > kStatsMaxTileBytes;
+    const int64_t adds = T * static_cast<int64_t>(K) * K;
+    const bool sparse = large && adds < (2 << 20) && (E > 896 || adds < (300 << 10));
     bool launched = false;
-    switch (K) {
-        case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
+    if (!sparse) {
+        switch (K) {
+            case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
+            default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
+        }
+        if (rc != COBALT_OK || launched) return rc;
     }
-    if (rc != COBALT_OK || launched) return rc;
-    if (tile_bytes(E, false) <= kStatsMaxTileBytes) return COBALT_ERR_UNSUPPORTED;   // clusters unavailable
-
-    switch (K) {
-        case 2: rc = launch_spread<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 4: rc = launch_spread<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 6: rc = launch_spread<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        case 8: rc = launch_spread<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-        default: rc = launch_spread<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
-    }
-    if (rc != COBALT_OK || launched) return rc;
-    // last resort: every pair straight to global memory
+    // also the last resort when no cluster shape can be scheduled
     int64_t want = (T + 255) / 256;
     const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
     cudaLaunchConfig_t cfg = {};

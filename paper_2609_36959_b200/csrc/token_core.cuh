@@ -216,8 +216,11 @@ __device__ __forceinline__ void assign_token(const TableView& tv, const int32_t 
 // Adds the K(K+1)/2 unordered pairs of one token (diagonal included) to a lower-triangle tile.
 // kPacked: two 16-bit counters per word (entry idx in the low or high half of word idx / 2); the
 // caller guarantees that no counter of the tile, nor its sum over the cluster, reaches 65536.
-template <int KT, bool kPacked = false>
-__device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32_t (&id)[TokenShape<KT>::KMAX], int K)
+// kSplit: the tile holds only the entries [first, first + count) of the flat triangle; pairs outside
+// are skipped (another CTA, fed the same tokens, holds them).
+template <int KT, bool kPacked = false, bool kSplit = false>
+__device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32_t (&id)[TokenShape<KT>::KMAX], int K,
+                                                      int first = 0, int count = 0)
 {
     constexpr int KMAX = TokenShape<KT>::KMAX;
 #pragma unroll
@@ -226,7 +229,11 @@ __device__ __forceinline__ void add_token_to_triangle(uint32_t* tri, const int32
         for (int b = a; b < KMAX; ++b) {
             if (b < K) {
                 const int hi = max(id[a], id[b]), lo = min(id[a], id[b]);
-                const int idx = hi * (hi + 1) / 2 + lo;
+                int idx = hi * (hi + 1) / 2 + lo;
+                if (kSplit) {
+                    idx -= first;
+                    if (static_cast<unsigned>(idx) >= static_cast<unsigned>(count)) continue;
+                }
                 if (kPacked) atomicAdd(&tri[idx >> 1], (idx & 1) ? 0x10000u : 1u);
                 else atomicAdd(&tri[idx], 1u);
             }
@@ -253,18 +260,25 @@ __device__ __forceinline__ int tri_row(int idx)
 // tile (no peer reads that slice) and the mirrors are issued in a second walk whose lanes run along
 // hi, i.e. along a row of coact.
 // The caller must hold a second cluster barrier before any CTA exits.
+// parts > 1: the tiles are split (see add_token_to_triangle); CTA rank r of the cluster holds part
+// r mod parts, `part_entries` entries (a multiple of the entries of a 16-byte vector) starting at
+// flat entry part * part_entries, and is merged with the cluster's other CTAs of the same part.
 template <bool kPacked = false>
 __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E, uint32_t* __restrict__ coact,
-                                                            uint32_t* __restrict__ load)
+                                                            uint32_t* __restrict__ load, int parts = 1,
+                                                            int part_entries = 0)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     constexpr int kPerWord = kPacked ? 2 : 1;            // triangle entries per 32-bit word
     const int n_tri = static_cast<int>(tri_entries(E));
-    const int n_words = (n_tri + kPerWord - 1) / kPerWord;
+    const int part = static_cast<int>(cluster.block_rank()) % parts;
+    const int entry0 = part * part_entries;              // flat entry held by word 0 of this tile
+    const int n_here = parts > 1 ? max(0, min(part_entries, n_tri - entry0)) : n_tri;
+    const int n_words = (n_here + kPerWord - 1) / kPerWord;
     const int n_vec = (n_words + 3) / 4;
-    const int csize = static_cast<int>(cluster.num_blocks());
-    const int crank = static_cast<int>(cluster.block_rank());
+    const int csize = static_cast<int>(cluster.num_blocks()) / parts;     // CTAs holding this part
+    const int crank = static_cast<int>(cluster.block_rank()) / parts;     // this CTA's index among them
     const int per = (n_vec + csize - 1) / csize;
     const int v0 = min(n_vec, crank * per), v1 = min(n_vec, v0 + per);
     for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
@@ -272,13 +286,13 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
 #pragma unroll 4
         for (int i = 0; i < csize; ++i) {
             // every CTA starts at its own tile, so the CTAs of a cluster do not all read one peer at once
-            const int r = (crank + i) % csize;
+            const int r = ((crank + i) % csize) * parts + part;
             const uint4 q = reinterpret_cast<const uint4*>(cluster.map_shared_rank(tri, r))[v];
             s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;    // packed halves cannot carry (see above)
         }
         reinterpret_cast<uint4*>(tri)[v] = s;
         const uint32_t word[4] = {s.x, s.y, s.z, s.w};
-        const int first = 4 * kPerWord * v;                      // first triangle entry of this vector
+        const int first = entry0 + 4 * kPerWord * v;             // first triangle entry of this vector
         int hi = tri_row(first);
         int lo = first - hi * (hi + 1) / 2;
 #pragma unroll
@@ -293,7 +307,7 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
     }
     __syncthreads();
     // mirrors of the slice [f0, f1): it covers (parts of) rows a..b of the triangle
-    const int f0 = 4 * kPerWord * v0, f1 = min(n_tri, 4 * kPerWord * v1);
+    const int f0 = entry0 + 4 * kPerWord * v0, f1 = min(entry0 + n_here, entry0 + 4 * kPerWord * v1);
     if (f0 >= f1) return;
     const int a = tri_row(f0), b = tri_row(f1 - 1);
     const int n_rows = b - a + 1;
@@ -303,7 +317,8 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
         const int hi = a + (j - lo * n_rows);
         const int flat = hi * (hi + 1) / 2 + lo;
         if (lo < hi && flat >= f0 && flat < f1) {
-            const uint32_t val = kPacked ? ((tri[flat >> 1] >> (16 * (flat & 1))) & 0xFFFFu) : tri[flat];
+            const int at = flat - entry0;
+            const uint32_t val = kPacked ? ((tri[at >> 1] >> (16 * (at & 1))) & 0xFFFFu) : tri[at];
             if (val) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
         }
     }

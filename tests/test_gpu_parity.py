@@ -159,20 +159,22 @@ def test_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     assert_combine_close(bits_from_bf16_tensor(step.y), O.combine(out, p["row_of_pair"], w.gate_w))
 
 
-def test_large_expert_count_takes_global_path(cb):
-    """E = 700: the co-activation triangle exceeds shared memory."""
+def test_large_expert_count(cb):
+    """E = 700: the co-activation triangle exceeds one CTA's shared memory and the fused pass falls back
+    to the separate calls."""
     w = W.make_custom(6000, 700, 8, 8, 4, 8, 24, seed=3, C=7, p_in=0.7)
     layout, step = make_step(w, with_x=False)
     check_index_stages(cb, w, step, 9)
 
 
 @pytest.mark.parametrize("E,K,T", [(320, 8, 20000), (384, 8, 131072), (451, 7, 9999), (452, 8, 70001),
-                                   (453, 8, 70001), (320, 8, 757777), (512, 6, 30000),
-                                   (1024, 8, 50000), (1024, 16, 3000)])
-def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
+                                   (453, 8, 70001), (320, 8, 757777), (512, 6, 30000), (600, 4, 5000),
+                                   (641, 10, 40000), (1024, 8, 50000), (1024, 16, 3000), (1024, 16, 20000)])
+def test_statistics_with_a_triangle_larger_than_one_tile(cb, E, K, T):
     """E > 316: the 32-bit triangle no longer fits one CTA.  Up to E = 452 a tile of 16-bit counters
-    does, as long as a cluster sees at most 65535 tokens (T = 757777 does not qualify); beyond that
-    the triangle is spread over the CTAs of a cluster."""
+    does, as long as a cluster sees at most 65535 tokens (clusters shrink for T = 757777); beyond that
+    the triangle is split over 2, 4 or 8 CTAs fed the same tokens, and few tokens over a large matrix
+    (E = 600 with T = 5000, E = 1024 with T = 3000) are added straight to global memory."""
     model = W.configs.ClusterModel(E, K, 8, 0.7, np.full(8, 1 / 8), np.ones(E))
     ids = W.sample_topk_ids(model, T, seed=E + K)
     ids_d = torch.from_numpy(ids).cuda()
@@ -187,11 +189,13 @@ def test_statistics_with_the_triangle_spread_over_a_cluster(cb, E, K, T):
     assert (u32(coact) == 2 * ref_coact).all() and (u32(load) == 2 * ref_load).all()
 
 
-@pytest.mark.parametrize("E,K,T,tile", [(400, 4, 3_000_000, "16-bit, small clusters"), (330, 2, 10_000_000, "spread")])
+@pytest.mark.parametrize("E,K,T,tile", [(400, 4, 3_000_000, "16-bit, small clusters"),
+                                        (500, 2, 4_000_000, "split over pairs of CTAs, clusters of two"),
+                                        (330, 2, 10_000_000, "global")])
 def test_statistics_many_tokens_and_a_large_triangle(cb, E, K, T, tile):
-    """The 16-bit tile may count at most 65535 tokens per cluster: T = 3e6 only allows clusters of two
-    CTAs, T = 1e7 none at all (the triangle is then spread over a cluster).  Ids are an arithmetic
-    progression per token (distinct by construction), cheap to draw at this size."""
+    """The 16-bit tiles may count at most 65535 tokens per cluster: T = 3e6 and 4e6 only allow clusters
+    of two CTAs, T = 1e7 none at all (every pair then goes straight to global memory).  Ids are an
+    arithmetic progression per token (distinct by construction), cheap to draw at this size."""
     rng = np.random.default_rng(E * K)
     base = rng.integers(0, E, size=(T, 1), dtype=np.int64)
     step = rng.integers(1, E // K, size=(T, 1), dtype=np.int64)
