@@ -11,6 +11,7 @@
 // kernels of the permutation follow.  Results are bit-identical to the separate calls.
 #include <cooperative_groups.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -33,16 +34,18 @@ struct RouteSmem {
     size_t bytes() const { return (tri_words + tab_words + hist_words) * sizeof(uint32_t); }
 };
 
-static RouteSmem route_smem(const LayoutView& lv)
+static RouteSmem route_smem(const LayoutView& lv, bool packed)
 {
     RouteSmem r;
-    r.tri_words = (tri_entries(lv.E) + 3) / 4 * 4;
+    r.tri_words = ((packed ? (tri_entries(lv.E) + 1) / 2 : tri_entries(lv.E)) + 3) / 4 * 4;
     r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
     r.hist_words = static_cast<size_t>(kRouteChunksPerRound) * lv.D;
     return r;
 }
 
-template <int KT>
+// kPacked: 16-bit counters in the triangle (see the statistics kernel); the launcher allows it only
+// while one cluster sees at most 65535 tokens.
+template <int KT, bool kPacked>
 __global__ void __launch_bounds__(kRouteThreads)
 route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ src_rank,
                    int32_t src_uniform, int64_t T, int32_t K_rt, uint32_t seed_lo, uint32_t seed_hi,
@@ -98,7 +101,7 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
             if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
             if (bad) flag_error(err_word, bad);
             // the statistics only need valid ids, as in the stand-alone statistics call
-            if (!bad_ids) add_token_to_triangle<KT>(tri, id, K);
+            if (!bad_ids) add_token_to_triangle<KT, kPacked>(tri, id, K);
             uint32_t cost = 0, naive_cost = 0;
             if (bad) {
 #pragma unroll
@@ -139,7 +142,7 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
     }
     cluster.sync();            // every triangle of the cluster is complete (also orders cta_totals)
     wait_for_prior_kernel();   // coact / load / totals may still be being cleared by the kernel before this one
-    merge_triangle_over_cluster(tri, lv.E, coact, load);
+    merge_triangle_over_cluster<kPacked>(tri, lv.E, coact, load);
     if (totals && threadIdx.x < 2 && cta_totals[threadIdx.x])
         atomicAdd(&totals[threadIdx.x], cta_totals[threadIdx.x]);
     cluster.sync();            // no CTA may exit while a peer still reads its triangle
@@ -150,10 +153,10 @@ struct RouteLaunch {
     int ctas;
 };
 
-template <int KT>
+template <int KT, bool kPacked>
 static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n_sm, RouteLaunch* out)
 {
-    auto kernel = route_fused_kernel<KT>;
+    auto kernel = route_fused_kernel<KT, kPacked>;
     static std::mutex cache_lock;
     static std::map<std::tuple<int, int, int, int64_t>, RouteLaunch> cache;
     int dev = 0;
@@ -232,20 +235,28 @@ struct RouteArgs {
     uint32_t* chunk_ws;
     int n_chunks;
     uint32_t* err_word;
-    bool after_zeroing;
+    ZeroList zero;
     int n_sm;
     cudaStream_t stream;
 };
 
-template <int KT>
-static int launch_route(const RouteArgs& a)
+// *launched stays false (and nothing has been enqueued) when 16-bit counters would be needed but one
+// cluster would see more than 65535 tokens: the caller then takes the separate calls.
+template <int KT, bool kPacked>
+static int launch_route(const RouteArgs& a, bool* launched)
 {
+    *launched = false;
     const LayoutView& lv = *a.lv;
-    const RouteSmem sm = route_smem(lv);
+    const RouteSmem sm = route_smem(lv, kPacked);
     RouteLaunch how;
-    int rc = pick_route_launch<KT>(lv, a.T, sm.bytes(), a.n_sm, &how);
+    int rc = pick_route_launch<KT, kPacked>(lv, a.T, sm.bytes(), a.n_sm, &how);
     if (rc != COBALT_OK) return rc;
-    auto kernel = route_fused_kernel<KT>;
+    const int chunks_per_cta = (a.n_chunks + how.ctas - 1) / how.ctas;
+    if (kPacked && static_cast<int64_t>(chunks_per_cta) * kRouteChunkTokens * how.cluster > 65535) return COBALT_OK;
+    bool after_zeroing = false;
+    rc = launch_zero_list(a.zero, a.stream, &after_zeroing);
+    if (rc != COBALT_OK) return rc;
+    auto kernel = route_fused_kernel<KT, kPacked>;
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sm.bytes())));
     COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
     cudaLaunchConfig_t cfg = {};
@@ -260,14 +271,21 @@ static int launch_route(const RouteArgs& a)
     attr[0].val.clusterDim.x = how.cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    set_programmatic_launch(&attr[1], a.after_zeroing);
+    set_programmatic_launch(&attr[1], after_zeroing);
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T, a.K,
                                        static_cast<uint32_t>(a.seed & 0xFFFFFFFFu),
                                        static_cast<uint32_t>(a.seed >> 32), a.coact, a.load, a.assigned_slot,
                                        a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.chunk_ws,
                                        a.n_chunks, static_cast<int>(sm.tri_words), static_cast<int>(sm.tab_words),
-                                       (a.n_chunks + how.ctas - 1) / how.ctas, a.err_word));
+                                       chunks_per_cta, a.err_word));
+    *launched = true;
     return COBALT_OK;
+}
+
+template <int KT>
+static int launch_route_any(const RouteArgs& a, bool packed, bool* launched)
+{
+    return packed ? launch_route<KT, true>(a, launched) : launch_route<KT, false>(a, launched);
 }
 
 static ChunkPlan route_chunks(int64_t T, int32_t K)
@@ -280,7 +298,13 @@ static ChunkPlan route_chunks(int64_t T, int32_t K)
     return c;
 }
 
-static bool fused_fits(const LayoutView& lv) { return route_smem(lv).bytes() <= kRouteMaxSmem; }
+// 0: the triangle does not fit beside the tables, 1: it fits with 32-bit counters, 2: with 16-bit ones
+static int fused_mode(const LayoutView& lv)
+{
+    if (route_smem(lv, false).bytes() <= kRouteMaxSmem) return 1;
+    if (route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
+    return 0;
+}
 
 }  // namespace cobalt
 
@@ -292,9 +316,12 @@ size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t
 {
     if (!layout || T < 0 || K < 1 || K > COBALT_MAX_TOPK || T * static_cast<int64_t>(K) >= (1ll << 31)) return 0;
     const LayoutView& lv = layout->view;
-    if (!fused_fits(lv) || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
+    const int mode = fused_mode(lv);
+    if (mode == 0 || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
     const ChunkPlan c = route_chunks(T, K);
-    return round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
+    const size_t fused = round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
+    // 16-bit counters may turn out not to be allowed for this T: room for the separate calls as well
+    return mode == 2 ? std::max(fused, cobalt_permute_workspace_bytes(T, K, lv.D)) : fused;
 }
 
 int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
@@ -321,7 +348,35 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != layout->device) return COBALT_ERR_INVALID_ARG;
 
-    if (!fused_fits(lv) || T == 0) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int mode = fused_mode(lv);
+    bool launched = false;
+    const ChunkPlan c = route_chunks(T, K);
+    if (mode != 0 && T > 0) {
+        RouteArgs a;
+        a.zero = ZeroList{{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
+        if (!(flags & COBALT_STATS_ACCUMULATE)) {
+            a.zero.ptr[0] = coact; a.zero.n[0] = lv.E * lv.E;
+            a.zero.ptr[1] = load;  a.zero.n[1] = lv.E;
+        }
+        a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K; a.seed = seed;
+        a.coact = coact; a.load = load; a.assigned_slot = assigned_slot; a.remote_nodes = remote_nodes; a.totals = totals;
+        a.chunk_ws = static_cast<uint32_t*>(workspace); a.n_chunks = c.n_chunks; a.stream = s;
+        int rc = device_error_word(&a.err_word);
+        if (rc != COBALT_OK) return rc;
+        rc = sm_count(&a.n_sm);
+        if (rc != COBALT_OK) return rc;
+        switch (K) {
+            case 1: rc = launch_route_any<1>(a, mode == 2, &launched); break;
+            case 2: rc = launch_route_any<2>(a, mode == 2, &launched); break;
+            case 4: rc = launch_route_any<4>(a, mode == 2, &launched); break;
+            case 6: rc = launch_route_any<6>(a, mode == 2, &launched); break;
+            case 8: rc = launch_route_any<8>(a, mode == 2, &launched); break;
+            default: rc = launch_route_any<0>(a, mode == 2, &launched);
+        }
+        if (rc != COBALT_OK) return rc;
+    }
+    if (!launched) {
         // the co-activation triangle does not fit beside the tables (or there is nothing to route):
         // same results from the separate calls
         int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags, nullptr, 0, stream);
@@ -332,37 +387,8 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         return cobalt_permute_index(assigned_slot, T, K, lv.D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
                                     workspace, workspace_bytes, stream);
     }
-
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    RouteArgs a;
-    a.after_zeroing = false;
-    ZeroList z = {{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
-    if (!(flags & COBALT_STATS_ACCUMULATE)) {
-        z.ptr[0] = coact; z.n[0] = lv.E * lv.E;
-        z.ptr[1] = load;  z.n[1] = lv.E;
-    }
-    int rc = launch_zero_list(z, s, &a.after_zeroing);
-    if (rc != COBALT_OK) return rc;
-
-    const ChunkPlan c = route_chunks(T, K);
-    a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K; a.seed = seed;
-    a.coact = coact; a.load = load; a.assigned_slot = assigned_slot; a.remote_nodes = remote_nodes; a.totals = totals;
-    a.chunk_ws = static_cast<uint32_t*>(workspace); a.n_chunks = c.n_chunks; a.stream = s;
-    rc = device_error_word(&a.err_word);
-    if (rc != COBALT_OK) return rc;
-    rc = sm_count(&a.n_sm);
-    if (rc != COBALT_OK) return rc;
-    switch (K) {
-        case 1: rc = launch_route<1>(a); break;
-        case 2: rc = launch_route<2>(a); break;
-        case 4: rc = launch_route<4>(a); break;
-        case 6: rc = launch_route<6>(a); break;
-        case 8: rc = launch_route<8>(a); break;
-        default: rc = launch_route<0>(a);
-    }
-    if (rc != COBALT_OK) return rc;
-    return launch_scan_and_rank(assigned_slot, T * K, lv.D, c, a.chunk_ws, dest_counts, dest_offsets, row_of_pair,
-                                pair_of_row, 0, s);
+    return launch_scan_and_rank(assigned_slot, T * K, lv.D, c, static_cast<uint32_t*>(workspace), dest_counts, dest_offsets,
+                                row_of_pair, pair_of_row, 0, s);
 }
 
 }  // extern "C"

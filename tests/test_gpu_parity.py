@@ -304,7 +304,11 @@ def test_fused_route_index_on_configs(cb, name):
     (1, 4, 1, 8, 1, 2, 2, 0), (7, 9, 2, 8, 3, 2, 2, 1), (255, 13, 3, 8, 4, 2, 3, 2), (257, 13, 3, 8, 4, 2, 3, 2),
     (1000, 20, 5, 8, 8, 1, 5, 0), (2049, 40, 8, 8, 2, 4, 6, 0), (4099, 100, 16, 8, 4, 8, 5, 7),
     (5000, 257, 7, 8, 4, 4, 20, 0), (6000, 700, 8, 8, 4, 8, 24, 0), (200000, 6, 2, 8, 4, 2, 1, 0),
-    (1100000, 40, 4, 8, 4, 2, 6, 0)])
+    (1100000, 40, 4, 8, 4, 2, 6, 0),
+    # E = 320..440: the fused pass keeps the triangle in 16-bit counters; with 600000 tokens a cluster
+    # would see more than 65535 of them and the separate calls take over
+    (20000, 384, 8, 8, 4, 8, 13, 0), (131072, 320, 8, 8, 4, 8, 11, 3), (9000, 440, 6, 8, 2, 4, 56, 0),
+    (600000, 330, 2, 8, 4, 2, 42, 0)])
 def test_fused_route_index_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     w = W.make_custom(T, E, K, H, N, Q, S, seed=2000 + T + E, C=3, p_in=0.6, n_empty=empty)
     layout, step = make_step(w, with_x=False)
