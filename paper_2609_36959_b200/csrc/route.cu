@@ -320,8 +320,9 @@ size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t
     if (mode == 0 || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
     const ChunkPlan c = route_chunks(T, K);
     const size_t fused = round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
-    // 16-bit counters may turn out not to be allowed for this T: room for the separate calls as well
-    return mode == 2 ? std::max(fused, cobalt_permute_workspace_bytes(T, K, lv.D)) : fused;
+    // the call may still take the separate calls (K without a compiled variant, 16-bit counters not
+    // allowed for this T): room for them as well
+    return std::max(fused, cobalt_permute_workspace_bytes(T, K, lv.D));
 }
 
 int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
@@ -352,7 +353,11 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     const int mode = fused_mode(lv);
     bool launched = false;
     const ChunkPlan c = route_chunks(T, K);
-    if (mode != 0 && T > 0) {
+    // The kernel is compiled for K = 1, 2, 4, 6, 8 with the K ids of a token in registers; its variant
+    // for any other K (loops to 16, spills) measured slower than the separate calls (K = 10: 85 us
+    // against 58 us at T = 65536, E = 256), so those take the separate calls.
+    const bool k_compiled = K == 1 || K == 2 || K == 4 || K == 6 || K == 8;
+    if (mode != 0 && T > 0 && k_compiled) {
         RouteArgs a;
         a.zero = ZeroList{{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
         if (!(flags & COBALT_STATS_ACCUMULATE)) {
@@ -372,7 +377,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
             case 4: rc = launch_route_any<4>(a, mode == 2, &launched); break;
             case 6: rc = launch_route_any<6>(a, mode == 2, &launched); break;
             case 8: rc = launch_route_any<8>(a, mode == 2, &launched); break;
-            default: rc = launch_route_any<0>(a, mode == 2, &launched);
+            default: rc = COBALT_ERR_UNSUPPORTED;
         }
         if (rc != COBALT_OK) return rc;
     }
