@@ -123,8 +123,8 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     const int parts = kSplit ? split_parts(E, &part_entries) : 1;
     if (parts == 0) return COBALT_OK;
     const size_t smem = kSplit ? static_cast<size_t>(part_entries) * 2 : tile_bytes(E, kPacked);
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), smem, true);
+    if (rc_attr != COBALT_OK) return rc_attr;
 
     // never more CTAs than can be co-resident (a second wave of
     // clusters would double the run time), clusters as large as the device schedules well

@@ -25,6 +25,11 @@ int device_error_word(uint32_t** out);
 // Number of SMs of the current device (cached per device).
 int sm_count(int* out);
 
+// Lets `kernel` be launched with up to `bytes` of dynamic shared memory (and, if asked, with a
+// cluster size above 8) on the current device.  The runtime calls are made only the first time
+// and when a larger size is asked for; later calls cost a map lookup.
+int ensure_kernel_attributes(const void* kernel, size_t bytes, bool non_portable_cluster);
+
 // Unsupported tuning knobs for parameter sweeps (set through cobalt_internal_tune; the defaults
 // are what the library ships with).
 struct Tuning {

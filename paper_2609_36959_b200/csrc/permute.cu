@@ -573,8 +573,8 @@ int launch_row_gather_scatter(const void* src, const int32_t* src_row, const int
     if (grid > 0x7FFFFFFFll) return COBALT_ERR_UNSUPPORTED;
     if (grid == 0) return COBALT_OK;
     const size_t smem = round_up(seg_bytes, 128);
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(row_gather_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem)));
+    const int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(row_gather_scatter_kernel), smem, false);
+    if (rc_attr != COBALT_OK) return rc_attr;
     row_gather_scatter_kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
         static_cast<const uint8_t*>(src), src_row, dst_row, n, src_rows, dst_rows, row_bytes, n_seg, seg_bytes,
         static_cast<uint8_t*>(dst), err_word);
@@ -642,8 +642,8 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     if (n_items > 0x7FFFFFFFll) return COBALT_ERR_UNSUPPORTED;
     if (impl == COBALT_IMPL_BULK) {
         const size_t smem1 = stage_bytes;
-        COBALT_CUDA_TRY(cudaFuncSetAttribute(perm_rows_bulk_oneshot_kernel,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem1)));
+        const int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(perm_rows_bulk_oneshot_kernel), smem1, false);
+        if (rc_attr != COBALT_OK) return rc_attr;
         perm_rows_bulk_oneshot_kernel<<<static_cast<unsigned>(n_items), 32, smem1, stream>>>(
             static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
             static_cast<uint8_t*>(send), err_word);

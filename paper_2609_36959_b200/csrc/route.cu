@@ -173,8 +173,8 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
             return COBALT_OK;
         }
     }
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), smem, true);
+    if (rc_attr != COBALT_OK) return rc_attr;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     cfg.blockDim = dim3(kRouteThreads);
@@ -257,8 +257,8 @@ static int launch_route(const RouteArgs& a, bool* launched)
     rc = launch_zero_list(a.zero, a.stream, &after_zeroing);
     if (rc != COBALT_OK) return rc;
     auto kernel = route_fused_kernel<KT, kPacked>;
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sm.bytes())));
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), sm.bytes(), true);
+    if (rc != COBALT_OK) return rc;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     cfg.blockDim = dim3(kRouteThreads);

@@ -2,6 +2,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <map>
+#include <mutex>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -24,9 +27,39 @@ __device__ uint32_t g_device_error_word = 0;
 
 int device_error_word(uint32_t** out)
 {
+    static uint32_t* cached[64] = {nullptr};      // the symbol's address on each device
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && cached[dev]) {
+        *out = cached[dev];
+        return COBALT_OK;
+    }
     void* p = nullptr;
     COBALT_CUDA_TRY(cudaGetSymbolAddress(&p, g_device_error_word));
+    if (dev >= 0 && dev < 64) cached[dev] = static_cast<uint32_t*>(p);
     *out = static_cast<uint32_t*>(p);
+    return COBALT_OK;
+}
+
+int ensure_kernel_attributes(const void* kernel, size_t bytes, bool non_portable_cluster)
+{
+    static std::mutex lock;
+    static std::map<std::pair<const void*, int>, size_t> granted;   // (kernel, device) -> bytes + 1 once set up
+    int dev = 0;
+    COBALT_CUDA_TRY(cudaGetDevice(&dev));
+    const auto key = std::make_pair(kernel, dev);
+    {
+        std::lock_guard<std::mutex> guard(lock);
+        auto it = granted.find(key);
+        if (it != granted.end() && it->second > bytes) return COBALT_OK;
+    }
+    if (bytes > 48 * 1024)
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)));
+    if (non_portable_cluster)
+        COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+    std::lock_guard<std::mutex> guard(lock);
+    size_t& have = granted[key];
+    if (have < bytes + 1) have = bytes + 1;
     return COBALT_OK;
 }
 
