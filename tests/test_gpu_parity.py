@@ -137,6 +137,8 @@ EDGE = [
     (3000, 17, 4, 16392, 2, 2, 5, 0),     # a row larger than one pipeline stage
     (70000, 6, 2, 8, 4, 2, 1, 0),
     (1100000, 40, 4, 8, 4, 2, 6, 0),      # more than 2048 chunks of 2048 pairs: the chunk size doubles
+    (3000, 1024, 16, 8, 8, 8, 64, 0),     # the largest supported layout: N = 8, K = 16, E = 1024, D = 4096
+    (2500, 1000, 13, 16, 8, 8, 64, 96),   # nearly so, with empty slots and an odd K
 ]
 
 
@@ -308,7 +310,7 @@ def test_fused_route_index_on_configs(cb, name):
     # E = 320..440: the fused pass keeps the triangle in 16-bit counters; with 600000 tokens a cluster
     # would see more than 65535 of them and the separate calls take over
     (20000, 384, 8, 8, 4, 8, 13, 0), (131072, 320, 8, 8, 4, 8, 11, 3), (9000, 440, 6, 8, 2, 4, 56, 0),
-    (600000, 330, 2, 8, 4, 2, 42, 0)])
+    (600000, 330, 2, 8, 4, 2, 42, 0), (3000, 1024, 16, 8, 8, 8, 64, 0)])
 def test_fused_route_index_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     w = W.make_custom(T, E, K, H, N, Q, S, seed=2000 + T + E, C=3, p_in=0.6, n_empty=empty)
     layout, step = make_step(w, with_x=False)
