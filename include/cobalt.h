@@ -158,7 +158,9 @@ int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids,
  *   pair_of_row     = inverse of row_of_pair (NULL to skip)           int32 [P]
  *   send[row_of_pair[p]] = x[p / K]    bit copy of H 16-bit elements  bf16 [P, H]
  * x is bf16 [T, H].  cobalt_permute = cobalt_permute_index followed by cobalt_permute_rows;
- * the two halves are exported so that the maps can be reused (e.g. for another tensor). */
+ * the two halves are exported so that the maps can be reused (e.g. for another tensor).
+ * The rows are moved as bits, so cobalt_permute_rows serves any element type whose row is a
+ * multiple of 16 bytes: pass H = row bytes / 2 (an 8-bit tensor of 7168 columns is H = 3584). */
 size_t cobalt_permute_workspace_bytes(int64_t T, int32_t K, int32_t D);
 int cobalt_permute_index(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D,
                          uint32_t* dest_counts, uint32_t* dest_offsets, int32_t* row_of_pair,
