@@ -148,6 +148,215 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
     cluster.sync();            // no CTA may exit while a peer still reads its triangle
 }
 
+// ---- batches of at most 16 chunks: everything in ONE kernel, one cluster --------------------------
+// Every CTA owns one chunk of 256 tokens.  The per-chunk destination histograms are exchanged through
+// distributed shared memory instead of a workspace in global memory, so the scan across chunks and
+// the stable rank run in the same kernel (two cluster barriers, no further launches), and with a
+// single cluster the statistics can be stored instead of added, so nothing is cleared beforehand.
+constexpr int kSmallMaxChunks = 16;
+constexpr int kSmallMaxDests = 992;        // one destination per thread in the scan over d; the last warp sums the totals
+constexpr int kSmallWarps = kRouteThreads / 32;
+
+struct SmallSmem {
+    size_t tri_words, tab_words, dest_words, slot_words, rank_words;
+    size_t bytes() const { return (tri_words + tab_words + 2 * dest_words + slot_words + rank_words) * sizeof(uint32_t); }
+};
+
+static SmallSmem small_smem(const LayoutView& lv, int K)
+{
+    SmallSmem r;
+    r.tri_words = (tri_entries(lv.E) + 3) / 4 * 4;
+    r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
+    r.dest_words = static_cast<size_t>(lv.D + 3) / 4 * 4;                   // chist, and the totals per destination
+    r.slot_words = static_cast<size_t>(kRouteChunkTokens) * K;              // this chunk's slots, in pair order
+    r.rank_words = static_cast<size_t>(1 + kSmallWarps) * r.dest_words;     // base[d] and the per-warp counters
+    return r;
+}
+
+template <int KT, bool kAccumulate>
+__global__ void __launch_bounds__(kRouteThreads)
+route_small_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ src_rank,
+                   int32_t src_uniform, int64_t T, uint32_t seed_lo, uint32_t seed_hi, uint32_t* __restrict__ coact,
+                   uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot, uint8_t* __restrict__ remote_nodes,
+                   unsigned long long* __restrict__ totals, uint32_t* __restrict__ dest_counts,
+                   uint32_t* __restrict__ dest_offsets, int32_t* __restrict__ row_of_pair,
+                   int32_t* __restrict__ pair_of_row, int tri_words, int tab_words, int dest_words, int key_bits,
+                   uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* tri = smem;
+    uint32_t* tab = tri + tri_words;
+    uint32_t* chist = tab + tab_words;             // [D] this chunk's pairs per destination
+    uint32_t* tot = chist + dest_words;            // [D] all chunks' pairs per destination
+    int32_t* slots = reinterpret_cast<int32_t*>(tot + dest_words);      // [256 * K]
+    uint32_t* base = reinterpret_cast<uint32_t*>(slots) + kRouteChunkTokens * KT;   // [D]
+    uint32_t* wcnt = base + dest_words;            // [kSmallWarps][dest_words]
+    __shared__ unsigned long long cta_totals[2];
+    __shared__ uint32_t warp_sums[kSmallWarps];
+    constexpr int K = KT;
+    const int D = lv.D;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int chunk = static_cast<int>(cluster.block_rank());
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // threads 0..255 run Algorithm 1 for the chunk's tokens, threads 256..511 add the same tokens to
+    // the triangle: two short instruction chains side by side instead of one long one
+    const int64_t t = static_cast<int64_t>(chunk) * kRouteChunkTokens + (tid & (kRouteChunkTokens - 1));
+    const bool has_token = tid < kRouteChunkTokens && t < T;
+    const bool counts_token = tid >= kRouteChunkTokens && tid < 2 * kRouteChunkTokens && t < T;
+    int32_t id[K], out[K];
+    int32_t s_t = src_uniform;
+    if (has_token || counts_token) {
+        load_token_ids<KT>(topk_ids, t, K, id);
+        if (has_token && src_rank) s_t = __ldg(src_rank + t);
+    }
+    for (int i = tid; i < tri_words / 4; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < dest_words; i += blockDim.x) chist[i] = 0;
+    for (int i = tid; i < kSmallWarps * dest_words; i += blockDim.x) wcnt[i] = 0;
+    if (tid < 2) cta_totals[tid] = 0;
+    const TableView tv = stage_tables(lv, tab);
+    __syncthreads();
+
+    uint32_t cost = 0, naive_cost = 0;
+    if (has_token) {
+        const uint32_t bad_ids = check_token_ids<KT>(id, K, lv.E);
+        uint32_t bad = bad_ids;
+        if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
+        if (bad) flag_error(err_word, bad);
+        if (bad) {
+#pragma unroll
+            for (int a = 0; a < K; ++a) out[a] = -1;
+        } else {
+            assign_token<KT, kAssignSlot>(tv, id, K, s_t, static_cast<uint32_t>(t), seed_lo, seed_hi, out, cost, naive_cost);
+#pragma unroll
+            for (int a = 0; a < K; ++a) atomicAdd(&chist[out[a]], 1u);
+        }
+        store_token_slots<KT>(assigned_slot + t * K, out, K);
+#pragma unroll
+        for (int a = 0; a < K; ++a) slots[tid * K + a] = out[a];
+        if (remote_nodes) remote_nodes[t] = static_cast<uint8_t>(cost);
+    } else if (counts_token) {
+        // the statistics only need valid ids, as in the stand-alone statistics call
+        if (!check_token_ids<KT>(id, K, lv.E)) add_token_to_triangle<KT>(tri, id, K);
+    }
+    if (totals && tid < kRouteChunkTokens) {      // the first eight warps hold the tokens
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            cost += __shfl_xor_sync(0xFFFFFFFFu, cost, off);
+            naive_cost += __shfl_xor_sync(0xFFFFFFFFu, naive_cost, off);
+        }
+        if (lane == 0) {
+            if (cost) atomicAdd(&cta_totals[0], static_cast<unsigned long long>(cost));
+            if (naive_cost) atomicAdd(&cta_totals[1], static_cast<unsigned long long>(naive_cost));
+        }
+    }
+    cluster.sync();            // every triangle, chunk histogram and cost sum of the cluster is complete
+
+    merge_triangle_over_cluster<false, !kAccumulate>(tri, lv.E, coact, load);
+    // scan across chunks, one destination per thread: pairs of lower chunks, and of all chunks
+    // (the cluster always has kSmallMaxChunks CTAs: all remote loads are issued before the first is used)
+    uint32_t mine_total = 0;
+    if (tid < D) {
+        uint32_t c[kSmallMaxChunks];
+#pragma unroll
+        for (int r = 0; r < kSmallMaxChunks; ++r) c[r] = cluster.map_shared_rank(chist, r)[tid];
+        uint32_t before = 0;
+#pragma unroll
+        for (int r = 0; r < kSmallMaxChunks; ++r) {
+            if (r < chunk) before += c[r];
+            mine_total += c[r];
+        }
+        base[tid] = before;
+        tot[tid] = mine_total;
+    } else if (totals && chunk == 0 && tid >= kSmallMaxDests && tid < kSmallMaxDests + 2) {
+        const int which = tid - kSmallMaxDests;
+        unsigned long long part[kSmallMaxChunks];
+#pragma unroll
+        for (int r = 0; r < kSmallMaxChunks; ++r) part[r] = cluster.map_shared_rank(cta_totals, r)[which];
+        unsigned long long sum = 0;
+#pragma unroll
+        for (int r = 0; r < kSmallMaxChunks; ++r) sum += part[r];
+        totals[which] = sum;
+    }
+    cluster.sync();            // no CTA may exit, nor may shared memory change, while a peer still reads it
+    // exclusive scan of the totals over d (one destination per thread, D <= blockDim.x)
+    uint32_t incl = mine_total;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    uint32_t offset = incl - mine_total;
+    for (int w = 0; w < warp; ++w) offset += warp_sums[w];
+    if (tid < D) {
+        base[tid] += offset;                    // first row of this chunk inside destination d
+        if (chunk == 0) {
+            dest_counts[tid] = mine_total;
+            dest_offsets[tid] = offset;
+            if (tid == D - 1) dest_offsets[D] = offset + mine_total;
+        }
+    }
+    __syncthreads();
+
+    // stable rank of the chunk's pairs: each warp owns 8 K consecutive pairs (at most four 32-pair steps)
+    const int n_tok = static_cast<int>(min(static_cast<int64_t>(kRouteChunkTokens),
+                                           max(static_cast<int64_t>(0), T - static_cast<int64_t>(chunk) * kRouteChunkTokens)));
+    const int n_pairs = n_tok * K;
+    constexpr int kSub = kRouteChunkTokens * K / kSmallWarps;
+    constexpr int kSteps = (kSub + 31) / 32;
+    const int w0 = warp * kSub, w1 = min(n_pairs, w0 + kSub);
+    const int64_t p0 = static_cast<int64_t>(chunk) * kRouteChunkTokens * K;
+    uint32_t* mine = wcnt + warp * dest_words;
+    int32_t dreg[kSteps];
+    uint32_t preg[kSteps];
+#pragma unroll
+    for (int st = 0; st < kSteps; ++st) {
+        const int p = w0 + st * 32 + lane;
+        const int32_t d = (st * 32 + lane < kSub && p < w1) ? slots[p] : -1;
+        const uint32_t key = static_cast<uint32_t>(d < 0 ? D : d);
+        uint32_t peers = 0xFFFFFFFFu;
+        for (int b = 0; b < key_bits; ++b) {
+            const uint32_t bit = (key >> b) & 1u;
+            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, bit);
+            peers &= bit ? vote : ~vote;
+        }
+        dreg[st] = d;
+        preg[st] = peers;
+        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
+        __syncwarp();
+    }
+    __syncthreads();
+    if (tid < D) {                              // per destination: per-warp counts -> starting rows, in warp order
+        uint32_t run = base[tid];
+#pragma unroll 8
+        for (int w = 0; w < kSmallWarps; ++w) {
+            const uint32_t c = wcnt[w * dest_words + tid];
+            wcnt[w * dest_words + tid] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int st = 0; st < kSteps; ++st) {
+        const int p = w0 + st * 32 + lane;
+        const bool in_range = st * 32 + lane < kSub && p < w1;
+        const int32_t d = dreg[st];
+        const uint32_t peers = preg[st];
+        if (d >= 0) {
+            const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
+            row_of_pair[p0 + p] = static_cast<int32_t>(row);
+            if (pair_of_row) pair_of_row[row] = static_cast<int32_t>(p0 + p);
+        } else if (in_range) {
+            row_of_pair[p0 + p] = -1;
+        }
+        __syncwarp();
+        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);
+        __syncwarp();
+    }
+}
+
 struct RouteLaunch {
     int cluster;
     int ctas;
@@ -282,6 +491,80 @@ static int launch_route(const RouteArgs& a, bool* launched)
     return COBALT_OK;
 }
 
+struct SmallArgs {
+    uint32_t* dest_counts;
+    uint32_t* dest_offsets;
+    int32_t* row_of_pair;
+    int32_t* pair_of_row;
+    bool accumulate;
+};
+
+// *launched stays false (nothing enqueued) when the batch, the layout or the device does not qualify.
+template <int KT>
+static int launch_route_small(const RouteArgs& a, const SmallArgs& b, bool* launched)
+{
+    *launched = false;
+    const LayoutView& lv = *a.lv;
+    if (a.T < 1 || a.n_chunks > kSmallMaxChunks || lv.D > kSmallMaxDests) return COBALT_OK;
+    const SmallSmem sm = small_smem(lv, KT);
+    if (sm.bytes() > kRouteMaxSmem) return COBALT_OK;
+    // always a full cluster: CTAs without tokens still take their share of the clearing and the merge
+    const int cluster = kSmallMaxChunks;
+    using Kernel = void (*)(LayoutView, const int32_t*, const int32_t*, int32_t, int64_t, uint32_t, uint32_t, uint32_t*,
+                            uint32_t*, int32_t*, uint8_t*, unsigned long long*, uint32_t*, uint32_t*, int32_t*, int32_t*,
+                            int, int, int, int, uint32_t*);
+    Kernel kernel = b.accumulate ? route_small_kernel<KT, true> : route_small_kernel<KT, false>;
+    int rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), sm.bytes(), true);
+    if (rc != COBALT_OK) return rc;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(kRouteThreads);
+    cfg.gridDim = dim3(static_cast<unsigned>(cluster));
+    cfg.dynamicSmemBytes = sm.bytes();
+    cfg.stream = a.stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    {   // can the device hold one such cluster at all?  asked once per (device, kernel, cluster, bytes)
+        static std::mutex lock;
+        static std::map<std::tuple<int, const void*, int, size_t>, bool> fits;
+        int dev = 0;
+        COBALT_CUDA_TRY(cudaGetDevice(&dev));
+        const auto key = std::make_tuple(dev, reinterpret_cast<const void*>(kernel), cluster, sm.bytes());
+        bool known = false, ok = false;
+        {
+            std::lock_guard<std::mutex> guard(lock);
+            auto it = fits.find(key);
+            if (it != fits.end()) { known = true; ok = it->second; }
+        }
+        if (!known) {
+            int max_clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess) {
+                (void)cudaGetLastError();
+                max_clusters = 0;
+            }
+            ok = max_clusters >= 1;
+            std::lock_guard<std::mutex> guard(lock);
+            fits[key] = ok;
+        }
+        if (!ok) return COBALT_OK;
+    }
+    int key_bits = 1;
+    while ((1 << key_bits) <= lv.D) ++key_bits;          // keys 0..D
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T,
+                                       static_cast<uint32_t>(a.seed & 0xFFFFFFFFu), static_cast<uint32_t>(a.seed >> 32),
+                                       a.coact, a.load, a.assigned_slot, a.remote_nodes,
+                                       reinterpret_cast<unsigned long long*>(a.totals), b.dest_counts, b.dest_offsets,
+                                       b.row_of_pair, b.pair_of_row, static_cast<int>(sm.tri_words),
+                                       static_cast<int>(sm.tab_words), static_cast<int>(sm.dest_words), key_bits,
+                                       a.err_word));
+    *launched = true;
+    return COBALT_OK;
+}
+
 template <int KT>
 static int launch_route_any(const RouteArgs& a, bool packed, bool* launched)
 {
@@ -371,6 +654,18 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         if (rc != COBALT_OK) return rc;
         rc = sm_count(&a.n_sm);
         if (rc != COBALT_OK) return rc;
+        if (mode == 1 && g_tune.route_small != 0) {
+            const SmallArgs b = {dest_counts, dest_offsets, row_of_pair, pair_of_row, (flags & COBALT_STATS_ACCUMULATE) != 0};
+            bool small = false;
+            switch (K) {
+                case 1: rc = launch_route_small<1>(a, b, &small); break;
+                case 2: rc = launch_route_small<2>(a, b, &small); break;
+                case 4: rc = launch_route_small<4>(a, b, &small); break;
+                case 6: rc = launch_route_small<6>(a, b, &small); break;
+                default: rc = launch_route_small<8>(a, b, &small);
+            }
+            if (rc != COBALT_OK || small) return rc;     // the single kernel has done everything
+        }
         switch (K) {
             case 1: rc = launch_route_any<1>(a, mode == 2, &launched); break;
             case 2: rc = launch_route_any<2>(a, mode == 2, &launched); break;

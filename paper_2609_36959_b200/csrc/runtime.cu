@@ -187,6 +187,7 @@ int cobalt_internal_tune(const char* key, int value)
     else if (!strcmp(key, "stats_max_ctas")) g_tune.stats_max_ctas = value;
     else if (!strcmp(key, "stats_cluster")) g_tune.stats_cluster = value;
     else if (!strcmp(key, "stats_packed")) g_tune.stats_packed = value;
+    else if (!strcmp(key, "route_small")) g_tune.route_small = value;
     else if (!strcmp(key, "stats_tokens_per_cta")) g_tune.stats_tokens_per_cta = value;
     else if (!strcmp(key, "combine_per_sm")) g_tune.combine_per_sm = value;
     else return COBALT_ERR_INVALID_ARG;

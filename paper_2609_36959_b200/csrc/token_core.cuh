@@ -263,7 +263,9 @@ __device__ __forceinline__ int tri_row(int idx)
 // parts > 1: the tiles are split (see add_token_to_triangle); CTA rank r of the cluster holds part
 // r mod parts, `part_entries` entries (a multiple of the entries of a 16-byte vector) starting at
 // flat entry part * part_entries, and is merged with the cluster's other CTAs of the same part.
-template <bool kPacked = false>
+// kStore: the grid is this one cluster and the outputs are to be overwritten: every entry (zeros
+// included) is stored instead of added, so the outputs need no clearing beforehand.
+template <bool kPacked = false, bool kStore = false>
 __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E, uint32_t* __restrict__ coact,
                                                             uint32_t* __restrict__ load, int parts = 1,
                                                             int part_entries = 0)
@@ -298,7 +300,12 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
 #pragma unroll
         for (int c = 0; c < 4 * kPerWord; ++c) {
             const uint32_t val = kPacked ? ((word[c >> 1] >> (16 * (c & 1))) & 0xFFFFu) : word[c];
-            if (first + c < n_tri && val) {
+            if (kStore) {
+                if (first + c < n_tri) {
+                    coact[static_cast<size_t>(hi) * E + lo] = val;
+                    if (lo == hi) load[hi] = val;
+                }
+            } else if (first + c < n_tri && val) {
                 atomicAdd(&coact[static_cast<size_t>(hi) * E + lo], val);
                 if (lo == hi) atomicAdd(&load[hi], val);
             }
@@ -319,7 +326,8 @@ __device__ __forceinline__ void merge_triangle_over_cluster(uint32_t* tri, int E
         if (lo < hi && flat >= f0 && flat < f1) {
             const int at = flat - entry0;
             const uint32_t val = kPacked ? ((tri[at >> 1] >> (16 * (at & 1))) & 0xFFFFu) : tri[at];
-            if (val) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
+            if (kStore) coact[static_cast<size_t>(lo) * E + hi] = val;
+            else if (val) atomicAdd(&coact[static_cast<size_t>(lo) * E + hi], val);
         }
     }
 }

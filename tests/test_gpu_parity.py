@@ -335,6 +335,35 @@ def test_step_with_statistics_on_a_side_stream(cb):
     assert (bits_from_bf16_tensor(step.send) == p["send"]).all()
 
 
+@pytest.mark.parametrize("T,E,K,N,Q,S,empty", [(4096, 256, 8, 4, 8, 9, 0), (4095, 64, 6, 4, 8, 3, 2), (257, 16, 2, 2, 4, 3, 0),
+                                               (1, 8, 1, 1, 2, 4, 0), (3000, 100, 4, 8, 4, 4, 5), (2049, 24, 8, 3, 2, 5, 0)])
+def test_fused_pass_in_a_single_cluster(cb, T, E, K, N, Q, S, empty):
+    """Up to 16 chunks of 256 tokens the fused entry runs ONE kernel in one cluster (histograms
+    exchanged through distributed shared memory, statistics stored instead of added).  Same results
+    as the oracle, as the general kernels (switched to with the sweep knob), and with the
+    accumulate flag on top of what is already there."""
+    import ctypes
+    tune = cb.binding._lib.cobalt_internal_tune
+    tune.argtypes = [ctypes.c_char_p, ctypes.c_int]
+    w = W.make_custom(T, E, K, 8, N, Q, S, seed=900 + T, C=2, p_in=0.7, n_empty=empty)
+    layout, step = make_step(w, with_x=False)
+    run_fused_and_compare(cb, w, step, 321)
+    small = {k: getattr(step, k).clone() for k in ("coact", "load", "assigned_slot", "dest_counts", "dest_offsets",
+                                                     "row_of_pair", "pair_of_row", "remote_nodes", "totals")}
+    assert tune(b"route_small", 0) == 0
+    try:
+        run_fused_and_compare(cb, w, step, 321)
+    finally:
+        assert tune(b"route_small", 1) == 0
+    for k, v in small.items():
+        assert torch.equal(getattr(step, k), v), k
+    cb.route_index(layout, step.topk_ids, step.src_rank, 321, step.coact, step.load, step.assigned_slot,
+                   step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace, flags=cb.STATS_ACCUMULATE)
+    torch.cuda.synchronize()
+    assert torch.equal(step.coact, 2 * small["coact"]) and torch.equal(step.load, 2 * small["load"])
+    assert torch.equal(step.row_of_pair, small["row_of_pair"]) and torch.equal(step.dest_offsets, small["dest_offsets"])
+
+
 def test_fused_route_step_equals_separate_stages(cb):
     w = W.make_config("3", T=12345)
     layout, step = make_step(w)
