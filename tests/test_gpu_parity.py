@@ -631,6 +631,42 @@ def test_bad_data_sets_the_error_word(cb):
     assert cb.read_and_clear_device_error() == 0
 
 
+@pytest.mark.parametrize("T", [2000, 9000])
+def test_bad_data_through_the_fused_entry(cb, T):
+    """The one-pass kernels (single cluster at T = 2000, general at T = 9000) treat bad tokens exactly as
+    the separate calls do: same error bits, slots of -1, rows of -1, counts without them."""
+    w = W.make_config("3", T=T)
+    layout, step = make_step(w, with_x=False)
+    ids = w.topk_ids.copy()
+    ids[10, 0] = w.E + 5
+    ids[300, 1] = ids[300, 0]
+    ids[T - 1, 2] = -4
+    step.topk_ids.copy_(torch.from_numpy(ids))
+    step.src_rank[30] = w.G
+    step.src_rank[T - 2] = -1
+    step.stats()
+    step.assign(7)
+    cb.permute_index(step.assigned_slot, w.D, step.dest_counts, step.dest_offsets, step.row_of_pair,
+                     step.pair_of_row, step.workspace)
+    torch.cuda.synchronize()
+    bits = cb.read_and_clear_device_error()
+    names = ("coact", "load", "assigned_slot", "remote_nodes", "totals", "dest_counts", "dest_offsets", "row_of_pair")
+    ref = {k: getattr(step, k).clone() for k in names}
+    n_valid = int(step.dest_offsets[-1])
+    ref_por = step.pair_of_row[:n_valid].clone()
+    for k in names:
+        getattr(step, k).fill_(9)
+    cb.route_index(layout, step.topk_ids, step.src_rank, 7, step.coact, step.load, step.assigned_slot,
+                   step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
+                   remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == bits & ~cb.DEVERR_BAD_SLOT
+    assert n_valid == (T - 5) * w.K
+    for k in names:
+        assert torch.equal(getattr(step, k), ref[k]), k
+    assert torch.equal(step.pair_of_row[:n_valid], ref_por)
+
+
 def test_argument_checks(cb):
     w = W.make_config("1", T=256)
     layout, step = make_step(w)
