@@ -33,7 +33,9 @@ constexpr size_t kStatsMaxTileBytes = 200 * 1024;
 // kSplit (E > 452): the triangle is cut into `parts` runs of part_entries flat entries; `parts`
 // consecutive CTAs form a group that is fed the same tokens, each CTA adding only the pairs that
 // fall into its own run.  All adds stay in the CTA's own shared memory.
-template <int KT, bool kPacked, bool kSplit>
+// kStore: the grid is a single cluster and the outputs are overwritten: the merge stores every entry
+// instead of adding to cleared outputs, and no clearing kernel runs before this one.
+template <int KT, bool kPacked, bool kSplit, bool kStore>
 __global__ void __launch_bounds__(kStatsThreads)
 coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int E, int tokens_per_cta, int parts,
                   int part_entries, uint32_t* __restrict__ coact, uint32_t* __restrict__ load,
@@ -68,7 +70,7 @@ coact_tile_kernel(const int32_t* __restrict__ topk_ids, int64_t T, int K_rt, int
 
     cluster.sync();            // every tile of the cluster is complete
     wait_for_prior_kernel();   // the outputs may still be being cleared by the kernel before this one
-    merge_triangle_over_cluster<kPacked>(tri, E, coact, load, kSplit ? parts : 1, part_entries);
+    merge_triangle_over_cluster<kPacked, kStore>(tri, E, coact, load, kSplit ? parts : 1, part_entries);
     cluster.sync();            // no CTA may exit while a peer still reads its tile
 }
 
@@ -114,11 +116,11 @@ static int split_parts(int E, int* part_entries)
 
 template <int KT, bool kPacked, bool kSplit>
 static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                       uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
+                       uint32_t* err_word, int n_sm, bool clear, cudaStream_t stream, bool* launched)
 {
     static_assert(kPacked || !kSplit, "split tiles use 16-bit counters");
     *launched = false;
-    auto kernel = coact_tile_kernel<KT, kPacked, kSplit>;
+    auto kernel = coact_tile_kernel<KT, kPacked, kSplit, false>;
     int part_entries = 0;
     const int parts = kSplit ? split_parts(E, &part_entries) : 1;
     if (parts == 0) return COBALT_OK;
@@ -132,10 +134,9 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // 15.4 us on 64 CTAs, 19.2 us on 16)
     const int per_cta = g_tune.stats_tokens_per_cta > 0 ? g_tune.stats_tokens_per_cta : 256;
     int64_t want = (T + per_cta - 1) / per_cta;
-    // batches below 16 blocks still get up to one full cluster (64 tokens per CTA at least): the
-    // shared-memory adds and the merge are then split 16 ways at no extra global reductions
-    if (want < 16) want = std::min<int64_t>(16, (T + 63) / 64);
-    if (want < 1) want = 1;
+    // small batches still get one full cluster: CTAs without tokens take their share of the merge
+    // (T = 64 on one CTA: 31 us), at no extra global reductions
+    if (want < 16) want = 16;
     want *= parts;                      // `parts` CTAs per group of tokens
     if (want > n_sm) want = n_sm;
     if (g_tune.stats_max_ctas > 0 && want > g_tune.stats_max_ctas) want = g_tune.stats_max_ctas;
@@ -216,6 +217,18 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     if (best_cs == 0) return kPacked ? COBALT_OK : COBALT_ERR_UNSUPPORTED;   // packed: caller takes another kernel
     attr[0].val.clusterDim.x = best_cs;
     cfg.gridDim = dim3(static_cast<unsigned>(best_cta));
+    // one cluster in all: it can store its sums, and the outputs need no clearing first
+    const bool store = clear && !kSplit && best_cta == best_cs;
+    bool after_zeroing = false;
+    if (clear && !store) {
+        const int rc = launch_zero_words(coact, E * E, load, E, stream, &after_zeroing);
+        if (rc != COBALT_OK) return rc;
+    }
+    if (store) {
+        kernel = coact_tile_kernel<KT, kPacked, kSplit, !kSplit>;
+        const int rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), smem, true);
+        if (rc != COBALT_OK) return rc;
+    }
     set_programmatic_launch(&attr[1], after_zeroing);
     cfg.numAttrs = 2;
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, ids, T, K, E, static_cast<int>(tokens_per_cta(best_cta)), parts,
@@ -228,20 +241,20 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
 // 16-bit tiles.
 template <int KT>
 static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                        uint32_t* err_word, int n_sm, bool after_zeroing, cudaStream_t stream, bool* launched)
+                        uint32_t* err_word, int n_sm, bool clear, cudaStream_t stream, bool* launched)
 {
     *launched = false;
     const bool fits32 = tile_bytes(E, false) <= kStatsMaxTileBytes;
     const bool fits16 = tile_bytes(E, true) <= kStatsMaxTileBytes;
     const bool want16 = g_tune.stats_packed > 0 || (g_tune.stats_packed < 0 && !fits32);
     if (fits16 && want16) {
-        const int rc = launch_tile<KT, true, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream,
+        const int rc = launch_tile<KT, true, false>(ids, T, K, E, coact, load, err_word, n_sm, clear, stream,
                                                     launched);
         if (rc != COBALT_OK || *launched) return rc;
     }
     if (fits32)
-        return launch_tile<KT, false, false>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
-    return launch_tile<KT, true, true>(ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, stream, launched);
+        return launch_tile<KT, false, false>(ids, T, K, E, coact, load, err_word, n_sm, clear, stream, launched);
+    return launch_tile<KT, true, true>(ids, T, K, E, coact, load, err_word, n_sm, clear, stream, launched);
 }
 
 }  // namespace cobalt
@@ -270,12 +283,9 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int rc = COBALT_OK;
+    const bool clear = !(flags & COBALT_STATS_ACCUMULATE);
     bool after_zeroing = false;
-    if (!(flags & COBALT_STATS_ACCUMULATE)) {
-        rc = launch_zero_words(coact, E * E, load, E, s, &after_zeroing);
-        if (rc != COBALT_OK) return rc;
-    }
-    if (T == 0) return COBALT_OK;
+    if (T == 0) return clear ? launch_zero_words(coact, E * E, load, E, s, &after_zeroing) : COBALT_OK;
 
     uint32_t* err_word = nullptr;
     rc = device_error_word(&err_word);
@@ -292,16 +302,20 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     bool launched = false;
     if (!sparse) {
         switch (K) {
-            case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched); break;
-            default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, after_zeroing, s, &launched);
+            case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched);
         }
         if (rc != COBALT_OK || launched) return rc;
     }
     // also the last resort when no cluster shape can be scheduled
+    if (clear) {
+        rc = launch_zero_words(coact, E * E, load, E, s, &after_zeroing);
+        if (rc != COBALT_OK) return rc;
+    }
     int64_t want = (T + 255) / 256;
     const unsigned grid = static_cast<unsigned>(want > 8 * n_sm ? 8 * n_sm : want);
     cudaLaunchConfig_t cfg = {};
