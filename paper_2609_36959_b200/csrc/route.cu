@@ -371,7 +371,7 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
     int64_t want = (T + kRouteChunkTokens - 1) / kRouteChunkTokens;   // one chunk per CTA while CTAs last
-    if (want < 1) want = 1;
+    if (want < 16) want = 16;      // a full cluster at least: CTAs without tokens still share the merge
     if (want > n_sm) want = n_sm;
     const auto key = std::make_tuple(dev, lv.E, lv.D, want * 1024 + lv.words % 1024);
     {
