@@ -235,6 +235,26 @@ def test_statistics_with_sixteen_bit_tiles_forced(cb, E, K, T):
     assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
 
 
+@pytest.mark.parametrize("E,K,T", [(256, 8, 3000), (64, 6, 1), (300, 4, 4096), (400, 8, 2500)])
+def test_statistics_of_a_small_batch_overwrite_used_buffers(cb, E, K, T):
+    """A batch small enough for a single cluster stores its sums without a clearing kernel before
+    it: whatever the outputs held is gone, and the accumulate flag still adds."""
+    model = W.configs.ClusterModel(E, K, 4, 0.7, np.full(4, 1 / 4), np.ones(E))
+    ids = W.sample_topk_ids(model, T, seed=E + T)
+    ids_d = torch.from_numpy(ids).cuda()
+    coact = torch.full((E, E), 123456, dtype=torch.int32, device="cuda")
+    load = torch.full((E,), 654321, dtype=torch.int32, device="cuda")
+    cb.coact_stats(ids_d, E, coact, load)
+    torch.cuda.synchronize()
+    ref_coact, ref_load = O.coact_stats(ids, E)
+    assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
+    cb.coact_stats(ids_d, E, coact, load, flags=cb.STATS_ACCUMULATE)
+    cb.coact_stats(ids_d, E, coact, load, flags=cb.STATS_ACCUMULATE)
+    torch.cuda.synchronize()
+    assert (u32(coact) == 3 * ref_coact).all() and (u32(load) == 3 * ref_load).all()
+    assert cb.read_and_clear_device_error() == 0
+
+
 def test_empty_batch(cb):
     w = W.make_custom(0, 8, 2, 16, 2, 2, 3, seed=1)
     layout, step = make_step(w)
