@@ -548,7 +548,7 @@ def run_cobalt(args):
         load_h = torch.empty((w.E,), dtype=torch.int32).pin_memory()
         sl_h = torch.empty((w.D,), dtype=torch.int32).pin_memory()
         tot_h = torch.empty((2,), dtype=torch.int64).pin_memory()
-        n_e2e = max(3, min(args.steps, 10))
+        n_e2e = max(3, min(args.steps, 30))
         for _ in range(2):
             step.route_host(w.seed, ids_h, w_h, src_h, x_h, y_h, coact_h, load_h, sl_h, tot_h)
         barrier()
