@@ -33,6 +33,12 @@ UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
 KERNELS_PER_STEP = 9               # stats 2 (clear + tile), assign 2 (clear + assign), permute 4 (hist, scan, rank, rows), combine 1
 
+
+def kernels_per_step(T):
+    """Launches of one four-stage step: the statistics of a batch that fits a single cluster
+    (at most 16 CTAs of 256 tokens) store their sums and need no clearing kernel."""
+    return KERNELS_PER_STEP - (1 if 0 < T <= 4096 else 0)
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes per pair, measured on a reduced token count and scaled by the pairs of a launch)
 NCU_TRAFFIC_BYTES_PER_PAIR = {"permute_rows": 15683.4, "combine": 15972.4}   # profiles/perm_rows_and_combine_T16384.md
@@ -598,7 +604,7 @@ def run_cobalt(args):
                              "so every stage starts cold" if w.P * w.H * 2 > (1 << 28) else
                              "inputs smaller than L2: stages run warm",
                        "parallelism": "replicas only (no cross-GPU step on this path)"},
-            "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "e2e": e2e, "gpu_launches": kernels_per_step(w.T) * args.steps,
             "roofline": roofline, "stages": stages, "clocks": clocks,
             "traffic_model": {"V_cobalt": totals[0], "V_naive": totals[1],
                               "remote_nodes_per_token_cobalt": totals[0] / max(w.T, 1),
