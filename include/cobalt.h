@@ -187,7 +187,7 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
  * The top-k ids are read once and the co-activation triangle, the layout tables and the chunk
  * histograms of the permutation share one cluster-launched kernel; the scan and stable-rank
  * kernels follow.  (Section 3.2 Stage 1, Section 3.3 Algorithm 1, Fig. 1 "Dispatch".)
- * The one-pass kernel exists for K = 1, 2, 4, 6, 8 and for layouts whose triangle fits beside the
+ * The one-pass kernel exists for K = 1, 2, 4, 6, 8, 10, 12, 16 and for layouts whose triangle fits beside the
  * tables (up to about 440 experts); every other case runs the three separate calls internally,
  * with the same results.  The workspace query covers both.
  * flags: COBALT_STATS_ACCUMULATE only.  remote_nodes, totals, pair_of_row may be NULL.

@@ -174,6 +174,9 @@ static int dispatch_assign(const AssignArgs& a)
         case 4: return launch_assign<4, MODE>(a);
         case 6: return launch_assign<6, MODE>(a);
         case 8: return launch_assign<8, MODE>(a);
+        case 10: return launch_assign<10, MODE>(a);
+        case 12: return launch_assign<12, MODE>(a);
+        case 16: return launch_assign<16, MODE>(a);
         default: return launch_assign<0, MODE>(a);
     }
 }

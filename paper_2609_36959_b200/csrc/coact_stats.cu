@@ -307,6 +307,9 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
             case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
             case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
             case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 10: rc = launch_tiles<10>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 12: rc = launch_tiles<12>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
+            case 16: rc = launch_tiles<16>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
             default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched);
         }
         if (rc != COBALT_OK || launched) return rc;

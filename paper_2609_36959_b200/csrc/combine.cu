@@ -217,6 +217,9 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
         COBALT_COMBINE_CASE(4);
         COBALT_COMBINE_CASE(6);
         COBALT_COMBINE_CASE(8);
+        COBALT_COMBINE_CASE(10);
+        COBALT_COMBINE_CASE(12);
+        COBALT_COMBINE_CASE(16);
         default:
             if (gate_w)
                 combine_kernel<0, false><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
@@ -281,6 +284,9 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
         COBALT_CBWD_CASE(4);
         COBALT_CBWD_CASE(6);
         COBALT_CBWD_CASE(8);
+        COBALT_CBWD_CASE(10);
+        COBALT_CBWD_CASE(12);
+        COBALT_CBWD_CASE(16);
         default:
             combine_backward_kernel<0><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go,
                                                                         grad_gate_w, err_word);

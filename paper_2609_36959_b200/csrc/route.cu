@@ -636,10 +636,10 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     const int mode = fused_mode(lv);
     bool launched = false;
     const ChunkPlan c = route_chunks(T, K);
-    // The kernel is compiled for K = 1, 2, 4, 6, 8 with the K ids of a token in registers; its variant
+    // The kernel is compiled for K = 1, 2, 4, 6, 8, 10, 12, 16 with the K ids of a token in registers; its variant
     // for any other K (loops to 16, spills) measured slower than the separate calls (K = 10: 85 us
     // against 58 us at T = 65536, E = 256), so those take the separate calls.
-    const bool k_compiled = K == 1 || K == 2 || K == 4 || K == 6 || K == 8;
+    const bool k_compiled = K == 1 || K == 2 || K == 4 || K == 6 || K == 8 || K == 10 || K == 12 || K == 16;
     if (mode != 0 && T > 0 && k_compiled) {
         RouteArgs a;
         a.zero = ZeroList{{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
@@ -654,7 +654,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         if (rc != COBALT_OK) return rc;
         rc = sm_count(&a.n_sm);
         if (rc != COBALT_OK) return rc;
-        if (mode == 1 && g_tune.route_small != 0) {
+        if (mode == 1 && g_tune.route_small != 0 && K <= 8) {
             const SmallArgs b = {dest_counts, dest_offsets, row_of_pair, pair_of_row, (flags & COBALT_STATS_ACCUMULATE) != 0};
             bool small = false;
             switch (K) {
@@ -672,6 +672,9 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
             case 4: rc = launch_route_any<4>(a, mode == 2, &launched); break;
             case 6: rc = launch_route_any<6>(a, mode == 2, &launched); break;
             case 8: rc = launch_route_any<8>(a, mode == 2, &launched); break;
+            case 10: rc = launch_route_any<10>(a, mode == 2, &launched); break;
+            case 12: rc = launch_route_any<12>(a, mode == 2, &launched); break;
+            case 16: rc = launch_route_any<16>(a, mode == 2, &launched); break;
             default: rc = COBALT_ERR_UNSUPPORTED;
         }
         if (rc != COBALT_OK) return rc;
