@@ -345,6 +345,18 @@ def extra_measurements(args, w, step, cb, torch):
         out["stats_overlapped_step_ms"] = None
         out["stats_overlap_error"] = str(exc)[:200]
 
+    # the four-stage step replayed from a CUDA graph (seed read from a device word at run time)
+    try:
+        n = max(5, min(args.steps, 30))
+        step.capture()
+        out["graph_step_ms"] = timed(lambda: step.replay(w.seed), n)
+        out["graph_step_pairs_per_s"] = w.P / (out["graph_step_ms"] * 1e-3)
+        step.capture(fused=True)
+        out["graph_fused_step_ms"] = timed(lambda: step.replay(w.seed), n)
+    except Exception as exc:
+        out["graph_step_ms"] = None
+        out["graph_step_error"] = str(exc)[:200]
+
     # the next two blocks allocate one more buffer of the send buffer's size: only with room to spare
     send_bytes = step.send.numel() * 2
 

@@ -69,6 +69,9 @@ extern "C" {
 #define COBALT_STATS_ACCUMULATE 0x1u         /* add to coact/load instead of overwriting them */
 #define COBALT_ASSIGN_NAIVE 0x1u             /* primary-replica rule instead of Algorithm 1 */
 #define COBALT_ASSIGN_ROUND_ROBIN 0x2u       /* deal each (expert, node) group's tasks to its replicas in turn */
+#define COBALT_SEED_ON_DEVICE 0x4u           /* cobalt_assign, cobalt_route_index: the `seed` argument is the device
+                                                address (8-byte aligned) of a uint64 that the kernel reads when it
+                                                runs, so that a captured CUDA graph can be replayed with a new seed */
 #define COBALT_IMPL_MASK 0xF00u              /* kernel variant override, 0 = library default */
 #define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
 #define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies, one work item per CTA (default) */
@@ -190,7 +193,7 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
  * The one-pass kernel exists for K = 1, 2, 4, 6, 8, 10, 12, 16 and for layouts whose triangle fits beside the
  * tables (up to about 440 experts); every other case runs the three separate calls internally,
  * with the same results.  The workspace query covers both.
- * flags: COBALT_STATS_ACCUMULATE only.  remote_nodes, totals, pair_of_row may be NULL.
+ * flags: COBALT_STATS_ACCUMULATE, COBALT_SEED_ON_DEVICE.  remote_nodes, totals, pair_of_row may be NULL.
  * Follow with cobalt_permute_rows to fill the send buffer. */
 size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);
 int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,

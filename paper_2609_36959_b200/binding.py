@@ -33,6 +33,7 @@ DEVERR_WAIT_TIMEOUT = 0x10
 STATS_ACCUMULATE = 0x1
 ASSIGN_NAIVE = 0x1
 ASSIGN_ROUND_ROBIN = 0x2
+SEED_ON_DEVICE = 0x4
 EMA_INITIALISE = 0x1
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200
@@ -150,6 +151,17 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+def _seed_arg(seed, flags: int):
+    """A Python int is passed by value; a one-element int64 CUDA tensor is passed by address and read
+    by the kernel when it runs (COBALT_SEED_ON_DEVICE), which lets a captured graph be replayed with
+    another seed."""
+    if isinstance(seed, torch.Tensor):
+        if seed.numel() != 1:
+            raise TypeError("a seed tensor must have one element")
+        return _ptr(seed, torch.int64, "seed"), flags | SEED_ON_DEVICE
+    return seed & (2**64 - 1), flags
+
+
 def _host_i32(a) -> "C.Array":
     vals = [int(v) for v in a]
     return (C.c_int32 * len(vals))(*vals)
@@ -223,7 +235,8 @@ def assign(layout: Layout, topk_ids: torch.Tensor, src_rank, seed: int, assigned
            slot_load: Optional[torch.Tensor] = None, remote_nodes: Optional[torch.Tensor] = None,
            totals: Optional[torch.Tensor] = None, flags: int = 0,
            workspace: Optional[torch.Tensor] = None) -> None:
-    """src_rank: int32 tensor [T], or a Python int used for every token."""
+    """src_rank: int32 tensor [T], or a Python int used for every token.  seed: a Python int, or a
+    one-element int64 CUDA tensor read when the kernel runs."""
     T, K = topk_ids.shape
     if assigned_slot.numel() != T * K:
         raise CobaltError(ERR_INVALID_ARG, "assign (assigned_slot size)")
@@ -240,8 +253,9 @@ def assign(layout: Layout, topk_ids: torch.Tensor, src_rank, seed: int, assigned
             raise CobaltError(ERR_INVALID_ARG, "assign (src_rank size)")
         src_ptr, src_uniform = _ptr(src_rank, torch.int32, "src_rank"), 0
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    seed, flags = _seed_arg(seed, flags)
     _check(_lib.cobalt_assign(layout.handle, _ptr(topk_ids, torch.int32, "topk_ids"), src_ptr, src_uniform,
-                              T, K, seed & (2**64 - 1), _ptr(assigned_slot, torch.int32, "assigned_slot"),
+                              T, K, seed, _ptr(assigned_slot, torch.int32, "assigned_slot"),
                               _ptr(slot_load, torch.int32, "slot_load"),
                               _ptr(remote_nodes, torch.uint8, "remote_nodes"),
                               _ptr(totals, torch.int64, "totals"), flags, _ptr(workspace), ws_bytes,
@@ -273,8 +287,9 @@ def route_index(layout: Layout, topk_ids: torch.Tensor, src_rank, seed: int, coa
         if src_rank.numel() != T:
             raise CobaltError(ERR_INVALID_ARG, "route_index (src_rank size)")
         src_ptr, src_uniform = _ptr(src_rank, torch.int32, "src_rank"), 0
+    seed, flags = _seed_arg(seed, flags)
     _check(_lib.cobalt_route_index(layout.handle, _ptr(topk_ids, torch.int32, "topk_ids"), src_ptr, src_uniform, T, K,
-                                   seed & (2**64 - 1), _ptr(coact, torch.int32, "coact"),
+                                   seed, _ptr(coact, torch.int32, "coact"),
                                    _ptr(load, torch.int32, "load"), _ptr(assigned_slot, torch.int32, "assigned_slot"),
                                    _ptr(remote_nodes, torch.uint8, "remote_nodes"), _ptr(totals, torch.int64, "totals"),
                                    _ptr(dest_counts, torch.int32, "dest_counts"),

@@ -25,9 +25,14 @@ assign_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t
               int32_t src_uniform, int64_t T, int32_t K_rt, uint32_t seed_lo, uint32_t seed_hi,
               int32_t* __restrict__ assigned_slot, uint32_t* __restrict__ slot_load,
               uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
-              uint32_t* __restrict__ err_word)
+              const unsigned long long* __restrict__ seed_on_device, uint32_t* __restrict__ err_word)
 {
     extern __shared__ __align__(16) uint32_t smem[];
+    if (seed_on_device) {                               // the seed of this run, not of the capture
+        const unsigned long long sd = __ldg(seed_on_device);
+        seed_lo = static_cast<uint32_t>(sd);
+        seed_hi = static_cast<uint32_t>(sd >> 32);
+    }
     uint32_t* tab = smem;                               // lv.words, padded to a multiple of 4
     uint32_t* hist = smem + (lv.words + 3) / 4 * 4;     // lv.D (only when slot_load != nullptr)
     __shared__ unsigned long long cta_totals[2];
@@ -126,6 +131,7 @@ struct AssignArgs {
     int64_t T;
     int32_t K;
     uint64_t seed;
+    const unsigned long long* seed_on_device;
     int32_t* assigned_slot;
     uint32_t* slot_load;
     uint8_t* remote_nodes;
@@ -161,7 +167,8 @@ static int launch_assign(const AssignArgs& a)
     COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T, a.K,
                                        static_cast<uint32_t>(a.seed & 0xFFFFFFFFu),
                                        static_cast<uint32_t>(a.seed >> 32), a.assigned_slot, a.slot_load,
-                                       a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.err_word));
+                                       a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals),
+                                       a.seed_on_device, a.err_word));
     return COBALT_OK;
 }
 
@@ -232,6 +239,8 @@ int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids, const 
     if (!aligned16(topk_ids) || !aligned16(assigned_slot) || !aligned16(src_rank) || !aligned16(slot_load) ||
         !aligned16(totals) || !aligned16(workspace))
         return COBALT_ERR_INVALID_ARG;
+    const bool seed_on_device = (flags & COBALT_SEED_ON_DEVICE) != 0;
+    if (seed_on_device && (seed == 0 || (seed & 7u) != 0)) return COBALT_ERR_INVALID_ARG;
     const bool naive = (flags & COBALT_ASSIGN_NAIVE) != 0;
     const bool round_robin = (flags & COBALT_ASSIGN_ROUND_ROBIN) != 0 && !naive;
     RoundRobinPlan rr = {};
@@ -252,7 +261,9 @@ int cobalt_assign(const cobalt_layout_t* layout, const int32_t* topk_ids, const 
     if (T == 0) return COBALT_OK;
 
     a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K;
-    a.seed = seed; a.assigned_slot = assigned_slot; a.slot_load = slot_load; a.remote_nodes = remote_nodes;
+    a.seed = seed_on_device ? 0 : seed;
+    a.seed_on_device = seed_on_device ? reinterpret_cast<const unsigned long long*>(static_cast<uintptr_t>(seed)) : nullptr;
+    a.assigned_slot = assigned_slot; a.slot_load = slot_load; a.remote_nodes = remote_nodes;
     a.totals = totals; a.stream = s;
     rc = device_error_word(&a.err_word);
     if (rc != COBALT_OK) return rc;

@@ -52,8 +52,14 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
                    uint32_t* __restrict__ coact, uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot,
                    uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
                    uint32_t* __restrict__ chunk_ws, int n_chunks, int tri_words, int tab_words,
-                   int chunks_per_cta, uint32_t* __restrict__ err_word)
+                   int chunks_per_cta, const unsigned long long* __restrict__ seed_on_device,
+                   uint32_t* __restrict__ err_word)
 {
+    if (seed_on_device) {                               // the seed of this run, not of the capture
+        const unsigned long long sd = __ldg(seed_on_device);
+        seed_lo = static_cast<uint32_t>(sd);
+        seed_hi = static_cast<uint32_t>(sd >> 32);
+    }
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t* tri = smem;
     uint32_t* tab = smem + tri_words;
@@ -181,8 +187,13 @@ route_small_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
                    unsigned long long* __restrict__ totals, uint32_t* __restrict__ dest_counts,
                    uint32_t* __restrict__ dest_offsets, int32_t* __restrict__ row_of_pair,
                    int32_t* __restrict__ pair_of_row, int tri_words, int tab_words, int dest_words, int key_bits,
-                   uint32_t* __restrict__ err_word)
+                   const unsigned long long* __restrict__ seed_on_device, uint32_t* __restrict__ err_word)
 {
+    if (seed_on_device) {                               // the seed of this run, not of the capture
+        const unsigned long long sd = __ldg(seed_on_device);
+        seed_lo = static_cast<uint32_t>(sd);
+        seed_hi = static_cast<uint32_t>(sd >> 32);
+    }
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t* tri = smem;
     uint32_t* tab = tri + tri_words;
@@ -436,6 +447,7 @@ struct RouteArgs {
     int64_t T;
     int32_t K;
     uint64_t seed;
+    const unsigned long long* seed_on_device;
     uint32_t* coact;
     uint32_t* load;
     int32_t* assigned_slot;
@@ -486,7 +498,7 @@ static int launch_route(const RouteArgs& a, bool* launched)
                                        static_cast<uint32_t>(a.seed >> 32), a.coact, a.load, a.assigned_slot,
                                        a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.chunk_ws,
                                        a.n_chunks, static_cast<int>(sm.tri_words), static_cast<int>(sm.tab_words),
-                                       chunks_per_cta, a.err_word));
+                                       chunks_per_cta, a.seed_on_device, a.err_word));
     *launched = true;
     return COBALT_OK;
 }
@@ -512,7 +524,7 @@ static int launch_route_small(const RouteArgs& a, const SmallArgs& b, bool* laun
     const int cluster = kSmallMaxChunks;
     using Kernel = void (*)(LayoutView, const int32_t*, const int32_t*, int32_t, int64_t, uint32_t, uint32_t, uint32_t*,
                             uint32_t*, int32_t*, uint8_t*, unsigned long long*, uint32_t*, uint32_t*, int32_t*, int32_t*,
-                            int, int, int, int, uint32_t*);
+                            int, int, int, int, const unsigned long long*, uint32_t*);
     Kernel kernel = b.accumulate ? route_small_kernel<KT, true> : route_small_kernel<KT, false>;
     int rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), sm.bytes(), true);
     if (rc != COBALT_OK) return rc;
@@ -560,7 +572,7 @@ static int launch_route_small(const RouteArgs& a, const SmallArgs& b, bool* laun
                                        reinterpret_cast<unsigned long long*>(a.totals), b.dest_counts, b.dest_offsets,
                                        b.row_of_pair, b.pair_of_row, static_cast<int>(sm.tri_words),
                                        static_cast<int>(sm.tab_words), static_cast<int>(sm.dest_words), key_bits,
-                                       a.err_word));
+                                       a.seed_on_device, a.err_word));
     *launched = true;
     return COBALT_OK;
 }
@@ -625,7 +637,9 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         !aligned16(assigned_slot) || !aligned16(totals) || !aligned16(dest_counts) || !aligned16(dest_offsets) ||
         !aligned16(row_of_pair) || !aligned16(pair_of_row) || !aligned16(workspace))
         return COBALT_ERR_INVALID_ARG;
-    if (flags & ~COBALT_STATS_ACCUMULATE) return COBALT_ERR_INVALID_ARG;
+    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_SEED_ON_DEVICE)) return COBALT_ERR_INVALID_ARG;
+    const bool seed_on_device = (flags & COBALT_SEED_ON_DEVICE) != 0;
+    if (seed_on_device && (seed == 0 || (seed & 7u) != 0)) return COBALT_ERR_INVALID_ARG;
     const size_t need = cobalt_route_index_workspace_bytes(layout, T, K);
     if (!workspace || workspace_bytes < need) return COBALT_ERR_WORKSPACE_TOO_SMALL;
     int dev = 0;
@@ -647,7 +661,9 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
             a.zero.ptr[0] = coact; a.zero.n[0] = lv.E * lv.E;
             a.zero.ptr[1] = load;  a.zero.n[1] = lv.E;
         }
-        a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K; a.seed = seed;
+        a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K;
+        a.seed = seed_on_device ? 0 : seed;
+        a.seed_on_device = seed_on_device ? reinterpret_cast<const unsigned long long*>(static_cast<uintptr_t>(seed)) : nullptr;
         a.coact = coact; a.load = load; a.assigned_slot = assigned_slot; a.remote_nodes = remote_nodes; a.totals = totals;
         a.chunk_ws = static_cast<uint32_t*>(workspace); a.n_chunks = c.n_chunks; a.stream = s;
         int rc = device_error_word(&a.err_word);
@@ -682,10 +698,10 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     if (!launched) {
         // the co-activation triangle does not fit beside the tables (or there is nothing to route):
         // same results from the separate calls
-        int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags, nullptr, 0, stream);
+        int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags & COBALT_STATS_ACCUMULATE, nullptr, 0, stream);
         if (rc != COBALT_OK) return rc;
         rc = cobalt_assign(layout, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot, nullptr,
-                           remote_nodes, totals, 0, nullptr, 0, stream);
+                           remote_nodes, totals, flags & COBALT_SEED_ON_DEVICE, nullptr, 0, stream);
         if (rc != COBALT_OK) return rc;
         return cobalt_permute_index(assigned_slot, T, K, lv.D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
                                     workspace, workspace_bytes, stream);

@@ -88,6 +88,31 @@ class RouteStep:
         if overlap_stats:
             main.wait_stream(self._side)
 
+    # -- the resident step replayed from a CUDA graph ------------------------------------------
+    def capture(self, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None,
+                fused: bool = False) -> None:
+        """Capture one step (the four stages, or the fused pass and the two row stages) into a CUDA
+        graph.  The seed lives in a device word that the assignment kernels read when they run, so
+        `replay(seed)` draws afresh every step.  The graph holds the addresses of this object's
+        buffers: new inputs are copied into topk_ids / gate_w / src_rank / x before a replay."""
+        self._seed_dev = torch.zeros(1, dtype=torch.int64, device=self.device)
+        run = (lambda: self.route_fused(self._seed_dev, experts)) if fused else (lambda: self.route(self._seed_dev, experts))
+        side = torch.cuda.Stream(device=self.device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(2):                     # first calls look up device attributes; not capturable
+                run()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize(self.device)
+        self._graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self._graph):
+            run()
+
+    def replay(self, seed: int) -> None:
+        """One captured step with this seed, enqueued on the current stream."""
+        self._seed_dev.fill_(seed if seed < 2**63 else seed - 2**64)
+        self._graph.replay()
+
     def route_fused(self, seed: int, experts: Optional[Callable[[torch.Tensor, torch.Tensor], None]] = None) -> None:
         """The same step with stages 1, 2 and the permutation index fused into one pass over the ids
         (cobalt_route_index); slot_load is delivered as dest_counts."""

@@ -384,6 +384,33 @@ def test_fused_pass_in_a_single_cluster(cb, T, E, K, N, Q, S, empty):
     assert torch.equal(step.row_of_pair, small["row_of_pair"]) and torch.equal(step.dest_offsets, small["dest_offsets"])
 
 
+@pytest.mark.parametrize("name,T,fused", [("3", 9000, False), ("3", 9000, True), ("1", 3000, True), ("5", 20000, False)])
+def test_step_replayed_from_a_graph_with_a_seed_on_the_device(cb, name, T, fused):
+    """capture() records one step whose assignment kernels read the seed from a device word;
+    replay(seed) must give what route(seed) gives, for every seed, including one above 2^63."""
+    w = W.make_config(name, T=T)
+    layout, step = make_step(w)
+    names = ("coact", "load", "assigned_slot", "remote_nodes", "totals", "dest_counts", "dest_offsets",
+             "row_of_pair", "pair_of_row", "send", "y")
+    step.capture(fused=fused)
+    for seed in (5, 2**63 + 12345, w.seed):
+        step.route_fused(seed) if fused else step.route(seed)
+        torch.cuda.synchronize()
+        ref = {k: getattr(step, k).clone() for k in names}
+        for k in names:
+            getattr(step, k).zero_()
+        step.replay(seed)
+        torch.cuda.synchronize()
+        for k in names:
+            a, b = getattr(step, k), ref[k]
+            if a.dtype == torch.bfloat16:
+                a, b = a.view(torch.int16), b.view(torch.int16)
+            assert torch.equal(a, b), (k, seed)
+    r = oracle_assign(w, w.seed)
+    assert (step.assigned_slot.cpu().numpy() == r["assigned_slot"]).all()
+    assert cb.read_and_clear_device_error() == 0
+
+
 def test_fused_route_step_equals_separate_stages(cb):
     w = W.make_config("3", T=12345)
     layout, step = make_step(w)
