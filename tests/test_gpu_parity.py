@@ -733,5 +733,13 @@ def test_argument_checks(cb):
     with pytest.raises(cb.CobaltError) as e:
         cb.Layout(2, 2, 2, 4, [0, 0, 2, 0, 1, 2, 3, 0])
     assert e.value.status == cb.ERR_INVALID_ARG
+    for bad_address in (0, step.totals.data_ptr() + 4):                     # null, and not 8-byte aligned
+        with pytest.raises(cb.CobaltError) as e:
+            cb.assign(layout, step.topk_ids, step.src_rank, bad_address, step.assigned_slot, flags=cb.SEED_ON_DEVICE)
+        assert e.value.status == cb.ERR_INVALID_ARG
+        with pytest.raises(cb.CobaltError) as e:
+            cb.route_index(layout, step.topk_ids, step.src_rank, bad_address, step.coact, step.load, step.assigned_slot,
+                           step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace, flags=cb.SEED_ON_DEVICE)
+        assert e.value.status == cb.ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert cb.read_and_clear_device_error() == 0
