@@ -171,7 +171,9 @@ struct SmallSmem {
 static SmallSmem small_smem(const LayoutView& lv, int K)
 {
     SmallSmem r;
-    r.tri_words = (tri_entries(lv.E) + 3) / 4 * 4;
+    // 16-bit counters (a cluster sees at most 4096 tokens): the merge is bound by the bytes that cross
+    // distributed shared memory, and these are half as many
+    r.tri_words = ((tri_entries(lv.E) + 1) / 2 + 3) / 4 * 4;
     r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
     r.dest_words = static_cast<size_t>(lv.D + 3) / 4 * 4;                   // chist, and the totals per destination
     r.slot_words = static_cast<size_t>(kRouteChunkTokens) * K;              // this chunk's slots, in pair order
@@ -248,7 +250,7 @@ route_small_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
         if (remote_nodes) remote_nodes[t] = static_cast<uint8_t>(cost);
     } else if (counts_token) {
         // the statistics only need valid ids, as in the stand-alone statistics call
-        if (!check_token_ids<KT>(id, K, lv.E)) add_token_to_triangle<KT>(tri, id, K);
+        if (!check_token_ids<KT>(id, K, lv.E)) add_token_to_triangle<KT, true>(tri, id, K);
     }
     if (totals && tid < kRouteChunkTokens) {      // the first eight warps hold the tokens
 #pragma unroll
@@ -263,7 +265,7 @@ route_small_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
     }
     cluster.sync();            // every triangle, chunk histogram and cost sum of the cluster is complete
 
-    merge_triangle_over_cluster<false, !kAccumulate>(tri, lv.E, coact, load);
+    merge_triangle_over_cluster<true, !kAccumulate>(tri, lv.E, coact, load);
     // scan across chunks, one destination per thread: pairs of lower chunks, and of all chunks
     // (the cluster always has kSmallMaxChunks CTAs: all remote loads are issued before the first is used)
     uint32_t mine_total = 0;
@@ -670,7 +672,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         if (rc != COBALT_OK) return rc;
         rc = sm_count(&a.n_sm);
         if (rc != COBALT_OK) return rc;
-        if (mode == 1 && g_tune.route_small != 0 && K <= 8) {
+        if (g_tune.route_small != 0 && K <= 8) {
             const SmallArgs b = {dest_counts, dest_offsets, row_of_pair, pair_of_row, (flags & COBALT_STATS_ACCUMULATE) != 0};
             bool small = false;
             switch (K) {

@@ -356,7 +356,8 @@ def test_step_with_statistics_on_a_side_stream(cb):
 
 
 @pytest.mark.parametrize("T,E,K,N,Q,S,empty", [(4096, 256, 8, 4, 8, 9, 0), (4095, 64, 6, 4, 8, 3, 2), (257, 16, 2, 2, 4, 3, 0),
-                                               (1, 8, 1, 1, 2, 4, 0), (3000, 100, 4, 8, 4, 4, 5), (2049, 24, 8, 3, 2, 5, 0)])
+                                               (1, 8, 1, 1, 2, 4, 0), (3000, 100, 4, 8, 4, 4, 5), (2049, 24, 8, 3, 2, 5, 0),
+                                               (4000, 384, 8, 4, 8, 13, 0), (4096, 420, 6, 2, 4, 60, 7)])
 def test_fused_pass_in_a_single_cluster(cb, T, E, K, N, Q, S, empty):
     """Up to 16 chunks of 256 tokens the fused entry runs ONE kernel in one cluster (histograms
     exchanged through distributed shared memory, statistics stored instead of added).  Same results
