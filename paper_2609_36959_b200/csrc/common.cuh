@@ -42,7 +42,7 @@ struct Tuning {
     int stats_max_ctas = 0;         // statistics kernel: cap on CTAs (0 = as many as can be co-resident)
     int stats_cluster = 0;          // statistics kernel: force this cluster size (0 = pick)
     int stats_tokens_per_cta = 0;   // statistics kernel: tokens per CTA the grid is sized for (0 = 256)
-    int stats_packed = -1;          // statistics kernel: 16-bit tile (-1 = only where the 32-bit tile does not fit, 0 = never, 1 = whenever legal)
+    int stats_packed = -1;          // statistics kernel: 16-bit tile (-1 = where it pays or the 32-bit tile does not fit, 0 = never, 1 = whenever legal)
     int route_small = 1;            // fused index pass: 0 = never take the single-cluster kernel
     int combine_per_sm = 0;         // CTAs per SM of the combine kernel's grid (0 = one CTA per token)
 };

@@ -598,6 +598,10 @@ static ChunkPlan route_chunks(int64_t T, int32_t K)
 // 0: the triangle does not fit beside the tables, 1: it fits with 32-bit counters, 2: with 16-bit ones
 static int fused_mode(const LayoutView& lv)
 {
+    // from about 180 experts on the 16-bit triangle is taken even where the 32-bit one fits: the merge
+    // is bound by the bytes that cross distributed shared memory
+    const bool large_tile = tri_entries(lv.E) * sizeof(uint32_t) >= 64 * 1024;
+    if (large_tile && g_tune.stats_packed != 0 && route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
     if (route_smem(lv, false).bytes() <= kRouteMaxSmem) return 1;
     if (route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
     return 0;
@@ -684,17 +688,23 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
             }
             if (rc != COBALT_OK || small) return rc;     // the single kernel has done everything
         }
-        switch (K) {
-            case 1: rc = launch_route_any<1>(a, mode == 2, &launched); break;
-            case 2: rc = launch_route_any<2>(a, mode == 2, &launched); break;
-            case 4: rc = launch_route_any<4>(a, mode == 2, &launched); break;
-            case 6: rc = launch_route_any<6>(a, mode == 2, &launched); break;
-            case 8: rc = launch_route_any<8>(a, mode == 2, &launched); break;
-            case 10: rc = launch_route_any<10>(a, mode == 2, &launched); break;
-            case 12: rc = launch_route_any<12>(a, mode == 2, &launched); break;
-            case 16: rc = launch_route_any<16>(a, mode == 2, &launched); break;
-            default: rc = COBALT_ERR_UNSUPPORTED;
-        }
+        auto launch_general = [&](bool packed) {
+            switch (K) {
+                case 1: return launch_route_any<1>(a, packed, &launched);
+                case 2: return launch_route_any<2>(a, packed, &launched);
+                case 4: return launch_route_any<4>(a, packed, &launched);
+                case 6: return launch_route_any<6>(a, packed, &launched);
+                case 8: return launch_route_any<8>(a, packed, &launched);
+                case 10: return launch_route_any<10>(a, packed, &launched);
+                case 12: return launch_route_any<12>(a, packed, &launched);
+                case 16: return launch_route_any<16>(a, packed, &launched);
+                default: return static_cast<int>(COBALT_ERR_UNSUPPORTED);
+            }
+        };
+        rc = launch_general(mode == 2);
+        // 16-bit counters refused for this many tokens: the 32-bit triangle, if it fits
+        if (rc == COBALT_OK && !launched && mode == 2 && route_smem(lv, false).bytes() <= kRouteMaxSmem)
+            rc = launch_general(false);
         if (rc != COBALT_OK) return rc;
     }
     if (!launched) {
