@@ -8,7 +8,9 @@
 // K(K+1)/2 pairs to the triangle, runs Algorithm 1, stores the K slots and counts them in the
 // histogram of its permutation chunk (256 consecutive tokens = 8 warps).  The triangle is then
 // merged over the cluster exactly as in the stand-alone statistics kernel; the scan and rank
-// kernels of the permutation follow.  Results are bit-identical to the separate calls.
+// kernels of the permutation follow.  Batches of at most 16 chunks run in a second kernel that does
+// all of it, scan and rank included, in one cluster (route_small_kernel).  Results are bit-identical
+// to the separate calls.
 #include <cooperative_groups.h>
 
 #include <algorithm>
