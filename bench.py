@@ -57,6 +57,7 @@ def parse_args():
                     help="tokens of the workload the CPU oracle is timed on (default 32768; 8192 for --impl reference)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="only the timed step loop (for launch lists under a profiler)")
     return ap.parse_args()
 
 
@@ -556,7 +557,7 @@ def run_cobalt(args):
 
     extras = {}
     if rank == 0:
-        extras = extra_measurements(args, w, step, cb, torch)
+        extras = {} if args.no_extras else extra_measurements(args, w, step, cb, torch)
 
     # end to end from pinned host buffers: H2D of the inputs, four stages, D2H of the results
     e2e = None
