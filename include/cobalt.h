@@ -27,6 +27,11 @@
  *    without synchronising; outputs are valid once the stream reaches that point.
  *  - Return value: COBALT_OK or a negative COBALT_ERR_* code.  Nothing is enqueued when an
  *    argument check fails.  The library never throws, exits, traps or waits unboundedly.
+ *  - Threads: every entry point may be called from several host threads at once.  The library
+ *    keeps no mutable state besides per-device caches of device attributes (guarded), the layout
+ *    handles (immutable once created; destroy one only when no call uses it) and one error word
+ *    per device.  Calls that run on the GPU at the same time must not share a workspace or
+ *    output buffers; cobalt_last_cuda_error is per host thread.
  *  - Data preconditions: ids in [0, E) and distinct within a token (D_t is a set); source
  *    ranks in [0, G); assigned slots in [0, D).  A violation never causes an out-of-bounds
  *    access: the kernel sets a bit in the device error word, skips the offending token or
@@ -50,10 +55,12 @@ extern "C" {
 #define COBALT_ERR_UNSUPPORTED (-3)          /* outside the supported size envelope (see below) */
 #define COBALT_ERR_CUDA (-4)                 /* a CUDA runtime call failed; see cobalt_last_cuda_error */
 #define COBALT_ERR_SCRATCH_LIMIT (-5)        /* problem needs more than the library's built-in scratch */
+#define COBALT_ERR_HOST_ALLOC (-6)           /* a host-side allocation failed (layout handle, planner scratch) */
 
-/* Supported envelope: N <= 8 nodes, K <= 16, E <= 1024, D <= 4096, P = T*K < 2^31,
- * H a multiple of 8 (rows are whole 16-byte vectors). */
+/* Supported envelope: N <= 8 nodes, Q <= 255 ranks per node, K <= 16, E <= 1024, D <= 4096,
+ * P = T*K < 2^31, H a multiple of 8 (rows are whole 16-byte vectors). */
 #define COBALT_MAX_NODES 8
+#define COBALT_MAX_RANKS_PER_NODE 255
 #define COBALT_MAX_TOPK 16
 #define COBALT_MAX_EXPERTS 1024
 #define COBALT_MAX_DESTS 4096
@@ -72,10 +79,14 @@ extern "C" {
 #define COBALT_SEED_ON_DEVICE 0x4u           /* cobalt_assign, cobalt_route_index: the `seed` argument is the device
                                                 address (8-byte aligned) of a uint64 that the kernel reads when it
                                                 runs, so that a captured CUDA graph can be replayed with a new seed */
-#define COBALT_IMPL_MASK 0xF00u              /* kernel variant override, 0 = library default */
+#define COBALT_STATS_TILE16 0x10u            /* cobalt_coact_stats: 16-bit counters in the shared-memory tile wherever
+                                                they cannot overflow (default: only where that is faster or the
+                                                32-bit tile does not fit) */
+#define COBALT_STATS_TILE32 0x20u            /* cobalt_coact_stats, cobalt_route_index: 32-bit counters wherever the tile fits */
+#define COBALT_ROUTE_GENERAL_KERNELS 0x40u   /* cobalt_route_index: do not take the single-cluster kernel for small batches */
+#define COBALT_IMPL_MASK 0xF00u              /* row-kernel variant override, 0 = library default */
 #define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
 #define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies, one work item per CTA (default) */
-#define COBALT_IMPL_BULK_RING 0x300u         /* same copies from a persistent CTA with a shared-memory ring */
 
 typedef struct cobalt_layout cobalt_layout_t;   /* opaque, owned by the library */
 typedef void* cobalt_stream_t;                  /* a cudaStream_t */
@@ -92,7 +103,8 @@ int cobalt_last_cuda_error(void);
  * A layout is rejected with COBALT_ERR_INVALID_ARG when an expert has no replica (Eq. 2,
  * first constraint), an expert sits twice on one rank (Section 3.2, Stage 2), an id is outside
  * [-1, E), or a given primary slot does not hold its expert; with COBALT_ERR_UNSUPPORTED
- * outside the size envelope.  cobalt_layout_check runs only these host-side checks (no device
+ * outside the size envelope, with COBALT_ERR_HOST_ALLOC when host memory runs out.
+ * cobalt_layout_check runs only these host-side checks (no device
  * needed).  cobalt_layout_create also builds the device tables (one allocation, one copy, on
  * the current device; synchronous) and returns a handle to be released with
  * cobalt_layout_destroy (NULL is accepted). */
@@ -111,7 +123,9 @@ int32_t cobalt_layout_num_dests(const cobalt_layout_t* layout);
  * coact[i*E+j] = number of tokens selecting both i and j (whose EMA is c^_ij); symmetric,
  *                diagonal = load.
  * topk_ids: int32 [T, K] row-major.  coact: uint32 [E*E].  load: uint32 [E].
- * Outputs are overwritten unless COBALT_STATS_ACCUMULATE is set.  T = 0 is allowed. */
+ * Outputs are overwritten unless COBALT_STATS_ACCUMULATE is set.  T = 0 is allowed.
+ * flags: COBALT_STATS_ACCUMULATE, and at most one of COBALT_STATS_TILE16 / COBALT_STATS_TILE32
+ * (counter width of the privatised shared-memory tile; the results are the same). */
 size_t cobalt_coact_stats_workspace_bytes(int64_t T, int32_t K, int32_t E);
 int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
                        uint32_t* coact, uint32_t* load, uint32_t flags,
@@ -193,7 +207,8 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
  * The one-pass kernel exists for K = 1, 2, 4, 6, 8, 10, 12, 16 and for layouts whose triangle fits beside the
  * tables (up to about 440 experts); every other case runs the three separate calls internally,
  * with the same results.  The workspace query covers both.
- * flags: COBALT_STATS_ACCUMULATE, COBALT_SEED_ON_DEVICE.  remote_nodes, totals, pair_of_row may be NULL.
+ * flags: COBALT_STATS_ACCUMULATE, COBALT_SEED_ON_DEVICE, COBALT_STATS_TILE32, COBALT_ROUTE_GENERAL_KERNELS
+ * (the last two select kernel variants, not results).  remote_nodes, totals, pair_of_row may be NULL.
  * Follow with cobalt_permute_rows to fill the send buffer. */
 size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);
 int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
@@ -231,7 +246,8 @@ int cobalt_permute_index_static(const int32_t* assigned_slot, int64_t T, int32_t
 /* ---- stage 4: combine (Fig. 1, "Weighted sum"; Section 1) ----------------------------------
  * y[t][h] = bf16( sum_{k<K} gate_w[t*K+k] * float(expert_out[row_of_pair[t*K+k]][h]) ),
  * fp32 accumulation in ascending k, one round-to-nearest-even at the end.
- * expert_out: bf16 [P, H] in the row order of `send`.  gate_w: fp32 [P].  y: bf16 [T, H]. */
+ * expert_out: bf16 [P, H] in the row order of `send`.  gate_w: fp32 [P] (required: NULL is
+ * COBALT_ERR_INVALID_ARG).  y: bf16 [T, H]. */
 int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w,
                    int64_t T, int32_t K, int32_t H, void* y, uint32_t flags,
                    cobalt_stream_t stream);
@@ -271,7 +287,8 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
  *   slots of a rank fill in placement order.  A node where some replica finds no admissible rank
  *   keeps its placement.  Outputs: new_slot_expert_host [G*S]; moved_from_host [G*S] (old slot
  *   of every new slot, -1 for empty; may be NULL); *nodes_kept_host (may be NULL).  Replicas never
- *   leave their node, so no cross-node parameter movement is implied. */
+ *   leave their node, so no cross-node parameter movement is implied.  The load of every occupied
+ *   slot must be finite and >= 0 (COBALT_ERR_INVALID_ARG otherwise). */
 #define COBALT_EMA_INITIALISE 0x1u
 int cobalt_ema_update(const uint32_t* counts, float* ema, int64_t n, float decay, uint32_t flags,
                       cobalt_stream_t stream);

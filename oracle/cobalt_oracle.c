@@ -143,26 +143,78 @@ int oracle_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
 }
 
 /* ------------------------------------------------------------------------------------------
- * Algorithm 1, token by token, in the paper's line order.
+ * Communication-aware task assignment (Section 3.3, Algorithm 1), token by token.
  *
- * Readings:  RemoteMask (line 4): bit j of an (N-1)-bit mask stands for the j-th remote node
- * in ascending node id with the source node skipped.  Lines 5-8: b ascends from 0 and
- * replaces b* only on a strictly smaller BitCount, so among equal-size covers the numerically
- * smallest b wins.  RandomNode (line 10): uniform over the set bits of b* & m, i-th set bit
- * counted from bit 0, i = floor(hash(stream 0) * popcount / 2^32).  UniformChoice (line 15):
- * uniform over R_{e,n} in ascending slot order with hash stream 1; the source rank gets no
- * preference inside its node.  Hash key is (token, expert), not the position k.
+ * Step 1 (node per expert).  Experts with a replica on the source node N(s_t) run there.  The
+ * others form U_t; each has a mask m_{t,e} over the N-1 remote nodes that hold it, and the
+ * token must reach a set of remote nodes b that meets every mask.  The paper finds the set with
+ * the fewest nodes by trying every (N-1)-bit mask.  Readings: bit j of a mask stands for the j-th
+ * remote node in ascending node id with the source node skipped; among covers of the minimum
+ * size the numerically smallest mask wins (the paper scans masks in ascending order and only
+ * replaces its candidate on a strictly smaller node count).  An expert of U_t then picks a node
+ * uniformly among the nodes of b* that hold it: the i-th set bit of b* & m_{t,e} counted from
+ * bit 0, i = floor(hash(stream 0) * popcount / 2^32).
+ * Step 2 (replica inside the node).  Uniform over R_{e,n} in ascending slot order with hash
+ * stream 1; the source rank gets no preference inside its node.  The hash key is (token, expert),
+ * not the position k.
  *
  * Outputs: assigned_slot[t*K+k] (r_te as global slot id); optional slot_load[d] = w_er
- * (Section 3.1); optional remote_nodes[t] = BitCount(b*) (0 when U_t is empty) = the token's
- * term of Eq. 1; optional totals[0] = V of this assignment, totals[1] = V of the naive rule.
+ * (Section 3.1); optional remote_nodes[t] = number of nodes in b* (0 when U_t is empty) = the
+ * token's term of Eq. 1; optional totals[0] = V of this assignment, totals[1] = V of the naive rule.
  * flags bit0: use the naive primary-replica rule (every task goes to primary[e]) instead.
  * flags bit1: round-robin replica pick.  Step 1 is unchanged; in Step 2 the tasks of a group
  *   (expert e, node n) are dealt to R_{e,n} in turn: walking the pairs in ascending p = t*K + k,
- *   the j-th task of the group (j from 0) goes to R_{e,n}[j mod |R_{e,n}|].  This makes "equal
- *   workloads in expectation" (Section 3.3, Step 2) exact: replica loads inside a group differ
- *   by at most one.  Not in the paper; an optional mode of this repository.
+ *   the j-th task of the group (j from 0) goes to R_{e,n}[j mod |R_{e,n}|].  Where the paper's
+ *   uniform pick balances the replicas of a group only on average (Section 3.3, Step 2), this
+ *   makes their loads differ by at most one.  Not in the paper; an optional mode of this repository.
  * ---------------------------------------------------------------------------------------- */
+
+/* m_{t,e}: which remote nodes (all nodes but n_s, ascending, bit j = j-th of them) hold an expert
+ * whose node set is `held`; 0 if the source node itself holds it (the expert is not in U_t). */
+static uint32_t remote_mask(uint32_t held, int32_t n_s, int32_t N)
+{
+    if (held & (1u << n_s)) return 0u;
+    uint32_t m = 0;
+    int32_t j = 0;
+    for (int32_t n = 0; n < N; ++n) {
+        if (n == n_s) continue;
+        if (held & (1u << n)) m |= 1u << j;
+        ++j;
+    }
+    return m;
+}
+
+/* b*: the smallest set of remote nodes that meets every non-zero mask (a minimum set cover by
+ * exhaustive search, sizes in increasing order, masks of one size in ascending value).  The empty
+ * set covers an empty U_t; the set of all remote nodes covers anything, so the search ends. */
+static uint32_t smallest_cover(const uint32_t* m, int32_t K, int32_t n_remote)
+{
+    for (int32_t size = 0; size <= n_remote; ++size) {
+        for (uint32_t b = 0; b < (1u << n_remote); ++b) {
+            if (popcount32(b) != size) continue;
+            int covers = 1;
+            for (int32_t a = 0; a < K; ++a)
+                if (m[a] != 0 && (b & m[a]) == 0) covers = 0;
+            if (covers) return b;
+        }
+    }
+    return 0u;   /* not reached */
+}
+
+/* Position of the i-th set bit of c, counting set bits from bit 0 (i < popcount(c)). */
+static int32_t nth_set_bit(uint32_t c, uint32_t i)
+{
+    for (int32_t bit = 0; bit < 32; ++bit) {
+        if (!(c & (1u << bit))) continue;
+        if (i == 0) return bit;
+        --i;
+    }
+    return -1;
+}
+
+/* Node id of remote-mask bit j as seen from source node n_s. */
+static int32_t remote_node(int32_t j, int32_t n_s) { return j < n_s ? j : j + 1; }
+
 int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
                   const int32_t* slot_expert, const int32_t* primary_in,
                   const int32_t* topk_ids, const int32_t* src_rank, int64_t T, int32_t K,
@@ -215,55 +267,25 @@ int oracle_assign(int32_t N, int32_t Q, int32_t S, int32_t E,
             continue;
         }
 
-        /* remote node list: all nodes but n_s, ascending; bit j <-> rem[j] */
-        int32_t rem[32];
-        int32_t n_rem = 0;
-        for (int32_t n = 0; n < N; ++n)
-            if (n != n_s) rem[n_rem++] = n;
-
-        /* line 3: U_t; line 4: m_{t,e} for e in U_t (m = 0 marks "not in U_t") */
+        /* Step 1: masks of the experts that are not on the source node, the smallest cover b*, and
+         * a node for every expert */
         int any_remote = 0;
         for (int32_t a = 0; a < K; ++a) {
-            uint32_t held = nodes_mask[D_t[a]];
-            m[a] = 0;
-            if (!(held & (1u << n_s))) {
-                for (int32_t j = 0; j < n_rem; ++j)
-                    if (held & (1u << rem[j])) m[a] |= 1u << j;
-                any_remote = 1;
-            }
+            m[a] = remote_mask(nodes_mask[D_t[a]], n_s, N);
+            if (m[a] != 0) any_remote = 1;
         }
-
-        /* lines 5-8 */
-        uint32_t b_star = (n_rem > 0) ? ((1u << n_rem) - 1u) : 0u;
-        if (n_rem > 0) {
-            for (uint32_t b = 0; b + 1 < (1u << n_rem); ++b) {
-                int feasible = 1;
-                for (int32_t a = 0; a < K; ++a)
-                    if (m[a] != 0 && (b & m[a]) == 0) { feasible = 0; break; }
-                if (feasible && popcount32(b) < popcount32(b_star)) b_star = b;
-            }
-        }
-
-        /* lines 9-13 */
+        uint32_t b_star = smallest_cover(m, K, N - 1);
         for (int32_t a = 0; a < K; ++a) {
+            n_te[a] = n_s;
             if (m[a] != 0) {
                 uint32_t c = b_star & m[a];
                 uint32_t i = oracle_hash_index(oracle_hash(seed, (uint32_t)t, (uint32_t)D_t[a], 0u),
                                                (uint32_t)popcount32(c));
-                int32_t bit = 0;
-                for (;; ++bit) {
-                    if (c & (1u << bit)) {
-                        if (i == 0) break;
-                        --i;
-                    }
-                }
-                n_te[a] = rem[bit];
-            } else {
-                n_te[a] = n_s;
+                n_te[a] = remote_node(nth_set_bit(c, i), n_s);
             }
         }
 
-        /* lines 14-16 */
+        /* Step 2: a replica of the expert inside its node */
         for (int32_t a = 0; a < K; ++a) {
             int64_t en = (int64_t)D_t[a] * N + n_te[a];
             uint32_t i;

@@ -22,6 +22,7 @@ ERR_WORKSPACE_TOO_SMALL = -2
 ERR_UNSUPPORTED = -3
 ERR_CUDA = -4
 ERR_SCRATCH_LIMIT = -5
+ERR_HOST_ALLOC = -6
 STATIC_SCRATCH_WORDS = 1 << 20
 
 DEVERR_BAD_EXPERT_ID = 0x1
@@ -34,10 +35,12 @@ STATS_ACCUMULATE = 0x1
 ASSIGN_NAIVE = 0x1
 ASSIGN_ROUND_ROBIN = 0x2
 SEED_ON_DEVICE = 0x4
+STATS_TILE16 = 0x10
+STATS_TILE32 = 0x20
+ROUTE_GENERAL_KERNELS = 0x40
 EMA_INITIALISE = 0x1
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200
-IMPL_BULK_RING = 0x300
 
 # every symbol include/cobalt.h declares
 EXPORTS = (

@@ -132,14 +132,12 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // clusters would double the run time), clusters as large as the device schedules well
     // sized for 256 tokens per CTA until the co-resident clusters run out (measured: T = 16384 takes
     // 15.4 us on 64 CTAs, 19.2 us on 16)
-    const int per_cta = g_tune.stats_tokens_per_cta > 0 ? g_tune.stats_tokens_per_cta : 256;
-    int64_t want = (T + per_cta - 1) / per_cta;
+    int64_t want = (T + 255) / 256;
     // small batches still get one full cluster: CTAs without tokens take their share of the merge
     // (T = 64 on one CTA: 31 us), at no extra global reductions
     if (want < 16) want = 16;
     want *= parts;                      // `parts` CTAs per group of tokens
     if (want > n_sm) want = n_sm;
-    if (g_tune.stats_max_ctas > 0 && want > g_tune.stats_max_ctas) want = g_tune.stats_max_ctas;
     if (want < parts) want = parts;
 
     cudaLaunchConfig_t cfg = {};
@@ -156,10 +154,10 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     // candidates: cluster sizes 16 (non-portable), 8, 4, 2, 1 -> CTAs that can be co-resident
     struct Candidates { int n = 0, cs[5], cta[5]; };
     static std::mutex cache_lock;
-    static std::map<std::tuple<int, int, int, int>, Candidates> cache;   // (dev, E, want, cluster knob); per <KT, kPacked>
+    static std::map<std::tuple<int, int, int>, Candidates> cache;   // (dev, E, want); per <KT, kPacked>
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
-    const auto key = std::make_tuple(dev, E, static_cast<int>(want), g_tune.stats_cluster);
+    const auto key = std::make_tuple(dev, E, static_cast<int>(want));
     Candidates cand;
     bool cached = false;
     {
@@ -173,7 +171,6 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
     if (!cached) {
         for (int cs = 16; cs >= 1; cs >>= 1) {
             if (cs > want || cs % parts != 0) continue;
-            if (g_tune.stats_cluster > 0 && cs != g_tune.stats_cluster) continue;
             attr[0].val.clusterDim.x = cs;
             cfg.gridDim = dim3(cs);
             int max_clusters = 0;
@@ -241,7 +238,8 @@ static int launch_tile(const int32_t* ids, int64_t T, int K, int E, uint32_t* co
 // 16-bit tiles.
 template <int KT>
 static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* coact, uint32_t* load,
-                        uint32_t* err_word, int n_sm, bool clear, cudaStream_t stream, bool* launched)
+                        uint32_t* err_word, int n_sm, bool clear, uint32_t tile_flags, cudaStream_t stream,
+                        bool* launched)
 {
     *launched = false;
     const bool fits32 = tile_bytes(E, false) <= kStatsMaxTileBytes;
@@ -249,7 +247,8 @@ static int launch_tiles(const int32_t* ids, int64_t T, int K, int E, uint32_t* c
     // the merge is bound by the bytes that cross distributed shared memory: from about 180 experts on
     // the halved tile wins (E = 256: 19.5 -> 17.4 us), below that the unpacking costs more (E = 64)
     const bool large_tile = tile_bytes(E, false) >= 64 * 1024;
-    const bool want16 = g_tune.stats_packed > 0 || (g_tune.stats_packed < 0 && (!fits32 || large_tile));
+    const bool want16 = (tile_flags & COBALT_STATS_TILE16) != 0 ||
+                        (!(tile_flags & COBALT_STATS_TILE32) && (!fits32 || large_tile));
     if (fits16 && want16) {
         const int rc = launch_tile<KT, true, false>(ids, T, K, E, coact, load, err_word, n_sm, clear, stream,
                                                     launched);
@@ -284,6 +283,9 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     if (T > 0 && !topk_ids) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(topk_ids) || !aligned16(coact) || !aligned16(load)) return COBALT_ERR_INVALID_ARG;
 
+    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_STATS_TILE16 | COBALT_STATS_TILE32)) return COBALT_ERR_INVALID_ARG;
+    const uint32_t tile_flags = flags & (COBALT_STATS_TILE16 | COBALT_STATS_TILE32);
+    if (tile_flags == (COBALT_STATS_TILE16 | COBALT_STATS_TILE32)) return COBALT_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int rc = COBALT_OK;
     const bool clear = !(flags & COBALT_STATS_ACCUMULATE);
@@ -305,15 +307,15 @@ int cobalt_coact_stats(const int32_t* topk_ids, int64_t T, int32_t K, int32_t E,
     bool launched = false;
     if (!sparse) {
         switch (K) {
-            case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 10: rc = launch_tiles<10>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 12: rc = launch_tiles<12>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            case 16: rc = launch_tiles<16>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched); break;
-            default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, s, &launched);
+            case 1: rc = launch_tiles<1>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 2: rc = launch_tiles<2>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 4: rc = launch_tiles<4>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 6: rc = launch_tiles<6>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 8: rc = launch_tiles<8>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 10: rc = launch_tiles<10>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 12: rc = launch_tiles<12>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            case 16: rc = launch_tiles<16>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched); break;
+            default: rc = launch_tiles<0>(topk_ids, T, K, E, coact, load, err_word, n_sm, clear, tile_flags, s, &launched);
         }
         if (rc != COBALT_OK || launched) return rc;
     }

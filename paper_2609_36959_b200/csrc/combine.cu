@@ -164,22 +164,18 @@ combine_backward_kernel(const uint4* __restrict__ grad_y, const uint4* __restric
     }
 }
 
-}  // namespace cobalt
-
-using namespace cobalt;
-
-extern "C" {
-
-int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
-                         int32_t K, int32_t H, void* y, int64_t total_rows, uint32_t flags,
-                         cobalt_stream_t stream)
+// Argument checks and launch shared by the combine and by the backward of the dispatch gather.
+// gate_w == nullptr selects unit weights (the plain sum of the K rows); the public combine entries
+// reject it before they get here.
+static int launch_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
+                          int32_t K, int32_t H, void* y, int64_t total_rows, uint32_t flags,
+                          cobalt_stream_t stream)
 {
     if (T < 0 || K < 1 || H < 1 || total_rows < 0) return COBALT_ERR_INVALID_ARG;
     if (K > COBALT_MAX_TOPK || H % 8 != 0 || T * static_cast<int64_t>(K) >= (1ll << 31) ||
         total_rows >= (1ll << 31))
         return COBALT_ERR_UNSUPPORTED;
     if (T == 0) return COBALT_OK;
-    // gate_w == NULL means unit weights (the plain sum of the K rows), used by cobalt_permute_backward
     if (!expert_out || !row_of_pair || !y) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(expert_out) || !aligned16(y) || !aligned16(row_of_pair) || !aligned16(gate_w))
         return COBALT_ERR_INVALID_ARG;
@@ -189,17 +185,13 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
     uint32_t* err_word = nullptr;
     int rc = device_error_word(&err_word);
     if (rc != COBALT_OK) return rc;
-    int n_sm = 0;
-    rc = sm_count(&n_sm);
-    if (rc != COBALT_OK) return rc;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int n_vec = H / 8;
     const int64_t P = total_rows;      // bound on the row indices (rows of the whole expert_out buffer)
     // one CTA per token: the block scheduler overlaps the per-token index loads of one CTA with
     // the row streaming of the others (measured faster than a persistent grid-stride grid)
-    const int64_t max_grid = g_tune.combine_per_sm > 0 ? static_cast<int64_t>(g_tune.combine_per_sm) * n_sm : 0x7FFFFFFFll;
-    const unsigned grid = static_cast<unsigned>(T < max_grid ? T : max_grid);
+    const unsigned grid = static_cast<unsigned>(T < 0x7FFFFFFFll ? T : 0x7FFFFFFFll);
     const uint4* src = static_cast<const uint4*>(expert_out);
     uint4* dst = static_cast<uint4*>(y);
 #define COBALT_COMBINE_CASE(KT)                                                                         \
@@ -233,6 +225,20 @@ int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, con
     return COBALT_OK;
 }
 
+}  // namespace cobalt
+
+using namespace cobalt;
+
+extern "C" {
+
+int cobalt_combine_block(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
+                         int32_t K, int32_t H, void* y, int64_t total_rows, uint32_t flags,
+                         cobalt_stream_t stream)
+{
+    if (T > 0 && !gate_w) return COBALT_ERR_INVALID_ARG;
+    return launch_combine(expert_out, row_of_pair, gate_w, T, K, H, y, total_rows, flags, stream);
+}
+
 int cobalt_combine(const void* expert_out, const int32_t* row_of_pair, const float* gate_w, int64_t T,
                    int32_t K, int32_t H, void* y, uint32_t flags, cobalt_stream_t stream)
 {
@@ -246,8 +252,7 @@ int cobalt_permute_backward(const void* grad_send, const int32_t* row_of_pair, i
 {
     if (T < 0 || K < 1) return COBALT_ERR_INVALID_ARG;
     // the adjoint of the gather is the sum of the token's K rows: the combine with unit weights
-    return cobalt_combine_block(grad_send, row_of_pair, nullptr, T, K, H, grad_x, T * static_cast<int64_t>(K), flags,
-                                stream);
+    return launch_combine(grad_send, row_of_pair, nullptr, T, K, H, grad_x, T * static_cast<int64_t>(K), flags, stream);
 }
 
 int cobalt_combine_backward(const void* grad_y, const void* expert_out, const int32_t* row_of_pair,

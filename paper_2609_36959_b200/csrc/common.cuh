@@ -30,23 +30,9 @@ int sm_count(int* out);
 // and when a larger size is asked for; later calls cost a map lookup.
 int ensure_kernel_attributes(const void* kernel, size_t bytes, bool non_portable_cluster);
 
-// Unsupported tuning knobs for parameter sweeps (set through cobalt_internal_tune; the defaults
-// are what the library ships with).
-struct Tuning {
-    int rows_item_bytes = 32768;    // default row mover: largest work item (whole rows of consecutive tokens)
-    int rows_stages = 6;            // ring variant: ring slots (3, 4, 6, 8 or 12)
-    int rows_stage_bytes = 18432;   // ring variant: largest ring slot
-    int rows_per_sm = 0;            // cap on CTAs per SM (0 = as many as shared memory allows)
-    int rows_vec_per_sm = 0;        // vector row mover: CTAs per SM (0 = one CTA per token)
-    int rows_hint = 0;              // 1 = evict-first L2 hints on the bulk copies
-    int stats_max_ctas = 0;         // statistics kernel: cap on CTAs (0 = as many as can be co-resident)
-    int stats_cluster = 0;          // statistics kernel: force this cluster size (0 = pick)
-    int stats_tokens_per_cta = 0;   // statistics kernel: tokens per CTA the grid is sized for (0 = 256)
-    int stats_packed = -1;          // statistics kernel: 16-bit tile (-1 = where it pays or the 32-bit tile does not fit, 0 = never, 1 = whenever legal)
-    int route_small = 1;            // fused index pass: 0 = never take the single-cluster kernel
-    int combine_per_sm = 0;         // CTAs per SM of the combine kernel's grid (0 = one CTA per token)
-};
-extern Tuning g_tune;
+// Largest work item of the bulk row movers: whole rows of consecutive tokens, or one column segment
+// of a longer row (measured flat between 14 and 112 KB; 32 KB keeps up to seven CTAs on an SM).
+constexpr int kRowsItemBytes = 32768;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

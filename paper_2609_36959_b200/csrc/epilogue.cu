@@ -3,6 +3,8 @@
 // the per-step intra-node greedy rebalancing of replicas (host code: the paper runs it on the
 // CPU, overlapped with model computation; it touches a few hundred numbers).
 #include <algorithm>
+#include <cmath>
+#include <new>
 #include <vector>
 
 #include "common.cuh"
@@ -78,6 +80,12 @@ int cobalt_rebalance_intra_node(int32_t N, int32_t Q, int32_t S, int32_t E, cons
     int rc = cobalt_layout_check(N, Q, S, E, slot_expert_host, nullptr);
     if (rc != COBALT_OK) return rc;
     if (!slot_load_host || !new_slot_expert_host) return COBALT_ERR_INVALID_ARG;
+    // loads of occupied slots must be finite and non-negative: a NaN would leave the sort below
+    // without a strict weak order
+    for (int32_t d = 0; d < N * Q * S; ++d)
+        if (slot_expert_host[d] >= 0 && !(slot_load_host[d] >= 0.0f && std::isfinite(slot_load_host[d])))
+            return COBALT_ERR_INVALID_ARG;
+    try {
     struct Replica {
         int32_t slot, expert;
         float load;
@@ -135,6 +143,9 @@ int cobalt_rebalance_intra_node(int32_t N, int32_t Q, int32_t S, int32_t E, cons
         }
     }
     if (nodes_kept_host) *nodes_kept_host = kept;
+    } catch (const std::bad_alloc&) {
+        return COBALT_ERR_HOST_ALLOC;
+    }
     return COBALT_OK;
 }
 

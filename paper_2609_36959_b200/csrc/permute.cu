@@ -9,11 +9,10 @@
 //       the CTA scans the per-warp counts in warp order, and each warp walks its sub-range
 //       again, ranking equal destinations inside a 32-pair step by lane order
 //       (per-bit ballots + popcount of lower lanes).
-// Row part: K4 moves each token's row to its K rows of the send buffer.  Three variants:
+// Row part: K4 moves each token's row to its K rows of the send buffer.  Two variants:
 // (default) one work item per single-warp CTA: a bulk async copy global -> shared, then one
 // bulk async copy shared -> global per destination row, many small CTAs in flight per SM;
-// a persistent variant of the same with a shared-memory ring; and plain 16-byte streaming
-// loads/stores.
+// and plain 16-byte streaming loads/stores.
 #include "permute_index.cuh"
 
 namespace cobalt {
@@ -330,145 +329,9 @@ __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uin
                  : "memory");
 }
 
-__device__ __forceinline__ uint64_t policy_evict_first()
-{
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-
-__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar,
-                                               uint64_t pol)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
-            smem_addr(smem_dst)),
-        "l"(gsrc), "r"(bytes), "r"(smem_addr(bar)), "l"(pol)
-        : "memory");
-}
-
-__device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src, uint32_t bytes, uint64_t pol)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
-                 "r"(smem_addr(smem_src)), "r"(bytes), "l"(pol)
-                 : "memory");
-}
-
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 
-template <int N>
-__device__ __forceinline__ void bulk_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-// One warp per CTA; kStages ring slots, loads run kLag items ahead of the stores; kHint marks both
-// directions evict-first in L2 (every byte is touched exactly once).  Work item i: `rows_per_item` whole rows of consecutive tokens (n_seg == 1),
-// or one column segment of one token's row (n_seg > 1, rows_per_item == 1).
-template <int kStages, int kLag, bool kHint>
-__global__ void __launch_bounds__(32)
-perm_rows_bulk_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_pair, int64_t T,
-                      int K, int64_t P, uint32_t row_bytes, int rows_per_item, int n_seg,
-                      uint32_t seg_bytes, uint32_t stage_bytes, int64_t n_items,
-                      uint8_t* __restrict__ send, uint32_t* __restrict__ err_word)
-{
-    extern __shared__ __align__(128) uint8_t ring[];
-    __shared__ __align__(8) uint64_t full[kStages];
-    __shared__ int32_t rows_sm[kStages][32];
-
-    const int lane = threadIdx.x;
-    uint64_t pol = 0;
-    if (kHint) pol = policy_evict_first();
-    if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < kStages; ++s) mbar_init(&full[s], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncwarp();
-
-    const int64_t first = blockIdx.x;
-    const int64_t step = gridDim.x;
-    const int64_t n_mine = (n_items > first) ? (n_items - first + step - 1) / step : 0;
-
-    auto item_tokens = [&](int64_t item, int64_t& t0, int& n_rows, uint32_t& col, uint32_t& bytes) {
-        if (n_seg == 1) {
-            t0 = item * rows_per_item;
-            n_rows = (T - t0 < rows_per_item) ? static_cast<int>(T - t0) : rows_per_item;
-            col = 0;
-            bytes = row_bytes;
-        } else {
-            t0 = item / n_seg;
-            n_rows = 1;
-            col = static_cast<uint32_t>(item % n_seg) * seg_bytes;
-            bytes = min(seg_bytes, row_bytes - col);
-        }
-    };
-    auto lane_row = [&](int64_t item) -> int32_t {
-        int64_t t0; int n_rows; uint32_t col, bytes;
-        item_tokens(item, t0, n_rows, col, bytes);
-        if (lane < n_rows * K) return __ldg(row_of_pair + t0 * K + lane);
-        return -1;
-    };
-
-    bool ok = true;
-    int32_t pref = (n_mine > 0) ? lane_row(first) : -1;
-    for (int64_t j = 0; j < n_mine + kLag && ok; ++j) {
-        if (j < n_mine) {
-            // produce item j: its stage was last used by item j - kStages
-            const int s = static_cast<int>(j % kStages);
-            bulk_wait_read<kStages - kLag - 1>();
-            rows_sm[s][lane] = pref;
-            if (j + 1 < n_mine) pref = lane_row(first + (j + 1) * step);
-            __syncwarp();
-            if (lane == 0) {
-                int64_t t0; int n_rows; uint32_t col, bytes;
-                item_tokens(first + j * step, t0, n_rows, col, bytes);
-                const uint32_t total = (n_seg == 1) ? static_cast<uint32_t>(n_rows) * row_bytes : bytes;
-                mbar_expect_tx(&full[s], total);
-                if (kHint)
-                    bulk_load_hint(ring + static_cast<size_t>(s) * stage_bytes,
-                                   x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s], pol);
-                else
-                    bulk_load(ring + static_cast<size_t>(s) * stage_bytes,
-                              x + static_cast<size_t>(t0) * row_bytes + col, total, &full[s]);
-            }
-        }
-        if (j >= kLag) {
-            // consume item c: wait for its rows, then fan each row out to its K destinations
-            const int64_t c = j - kLag;
-            const int s = static_cast<int>(c % kStages);
-            ok = mbar_wait(&full[s], static_cast<uint32_t>((c / kStages) & 1));
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (ok) {
-                int64_t t0; int n_rows; uint32_t col, bytes;
-                item_tokens(first + c * step, t0, n_rows, col, bytes);
-                const int32_t row = rows_sm[s][lane];
-                if (row >= 0 && row < P) {
-                    const int r = lane / K;
-                    void* dst = send + static_cast<size_t>(row) * row_bytes + col;
-                    const void* src = ring + static_cast<size_t>(s) * stage_bytes + static_cast<size_t>(r) * row_bytes;
-                    if (kHint) bulk_store_hint(dst, src, bytes, pol);
-                    else bulk_store(dst, src, bytes);
-                } else if (row >= P) {
-                    flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
-                }
-            }
-            bulk_commit();
-        }
-    }
-    bulk_wait_all();
-    if (!ok) {
-        if (lane == 0) flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
-        // give loads still in flight a bounded chance to land before the ring is released
-        for (int s = 0; s < kStages; ++s) {
-            (void)mbar_wait(&full[s], 0);
-            (void)mbar_wait(&full[s], 1);
-        }
-    }
-}
 
 // One work item per single-warp CTA, no ring: the block scheduler keeps many small CTAs in
 // flight per SM (shared memory for one item each) and hands out items in order.
@@ -565,7 +428,7 @@ int launch_row_gather_scatter(const void* src, const int32_t* src_row, const int
     int rc = device_error_word(&err_word);
     if (rc != COBALT_OK) return rc;
     const uint32_t row_bytes = static_cast<uint32_t>(H) * 2u;
-    const int max_seg = g_tune.rows_item_bytes;
+    const int max_seg = kRowsItemBytes;
     int n_seg = (row_bytes + max_seg - 1) / max_seg;
     uint32_t seg_bytes = static_cast<uint32_t>(round_up((row_bytes + n_seg - 1) / n_seg, 16));
     n_seg = (row_bytes + seg_bytes - 1) / seg_bytes;
@@ -599,8 +462,7 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
 
     if (impl == COBALT_IMPL_VECTOR) {
         const int n_vec = H / 8;
-        const int64_t max_grid = g_tune.rows_vec_per_sm > 0 ? static_cast<int64_t>(g_tune.rows_vec_per_sm) * n_sm : 0x7FFFFFFFll;
-        const unsigned grid = static_cast<unsigned>(T < max_grid ? T : max_grid);
+        const unsigned grid = static_cast<unsigned>(T < 0x7FFFFFFFll ? T : 0x7FFFFFFFll);   // one CTA per token
         const uint4* xs = static_cast<const uint4*>(x);
         uint4* out = static_cast<uint4*>(send);
 #define COBALT_ROWS_CASE(KT)                                                                              \
@@ -622,8 +484,7 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     }
 
     // bulk variant: pick the work-item shape
-    const Tuning& tune = g_tune;
-    const int max_stage = (impl == COBALT_IMPL_BULK) ? tune.rows_item_bytes : tune.rows_stage_bytes;
+    const int max_stage = kRowsItemBytes;
     int rows_per_item = 1, n_seg = 1;
     uint32_t seg_bytes = row_bytes;
     if (row_bytes <= static_cast<uint32_t>(max_stage)) {
@@ -640,48 +501,12 @@ static int launch_rows(const void* x, const int32_t* row_of_pair, int64_t T, int
     const int64_t n_items = (n_seg == 1) ? (T + rows_per_item - 1) / rows_per_item : T * n_seg;
 
     if (n_items > 0x7FFFFFFFll) return COBALT_ERR_UNSUPPORTED;
-    if (impl == COBALT_IMPL_BULK) {
-        const size_t smem1 = stage_bytes;
-        const int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(perm_rows_bulk_oneshot_kernel), smem1, false);
-        if (rc_attr != COBALT_OK) return rc_attr;
-        perm_rows_bulk_oneshot_kernel<<<static_cast<unsigned>(n_items), 32, smem1, stream>>>(
-            static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
-            static_cast<uint8_t*>(send), err_word);
-        COBALT_CUDA_TRY(cudaGetLastError());
-        return COBALT_OK;
-    }
-
-    using Kernel = void (*)(const uint8_t*, const int32_t*, int64_t, int, int64_t, uint32_t, int, int, uint32_t,
-                            uint32_t, int64_t, uint8_t*, uint32_t*);
-    Kernel kernel = nullptr;
-    int stages = tune.rows_stages;
-    const bool hint = tune.rows_hint != 0;
-#define COBALT_BULK_CASE(NS, LAG)                                                                      \
-    case NS:                                                                                           \
-        kernel = hint ? perm_rows_bulk_kernel<NS, LAG, true> : perm_rows_bulk_kernel<NS, LAG, false>;  \
-        break
-    switch (stages) {
-        COBALT_BULK_CASE(3, 1);
-        COBALT_BULK_CASE(4, 2);
-        COBALT_BULK_CASE(8, 4);
-        COBALT_BULK_CASE(12, 6);
-        default:
-            stages = 6;
-            kernel = hint ? perm_rows_bulk_kernel<6, 3, true> : perm_rows_bulk_kernel<6, 3, false>;
-    }
-#undef COBALT_BULK_CASE
-    const size_t smem = static_cast<size_t>(stages) * stage_bytes;
-    if (smem > 224 * 1024) return COBALT_ERR_UNSUPPORTED;
-    COBALT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    int per_sm = static_cast<int>((220 * 1024) / (smem + 2048));
-    if (per_sm < 1) per_sm = 1;
-    if (per_sm > 8) per_sm = 8;
-    if (tune.rows_per_sm > 0 && tune.rows_per_sm < per_sm) per_sm = tune.rows_per_sm;
-    int64_t grid = static_cast<int64_t>(n_sm) * per_sm;
-    if (grid > n_items) grid = n_items;
-    kernel<<<static_cast<unsigned>(grid), 32, smem, stream>>>(
+    const size_t smem1 = stage_bytes;
+    const int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(perm_rows_bulk_oneshot_kernel), smem1, false);
+    if (rc_attr != COBALT_OK) return rc_attr;
+    perm_rows_bulk_oneshot_kernel<<<static_cast<unsigned>(n_items), 32, smem1, stream>>>(
         static_cast<const uint8_t*>(x), row_of_pair, T, K, P, row_bytes, rows_per_item, n_seg, seg_bytes,
-        stage_bytes, n_items, static_cast<uint8_t*>(send), err_word);
+        static_cast<uint8_t*>(send), err_word);
     COBALT_CUDA_TRY(cudaGetLastError());
     return COBALT_OK;
 }
@@ -857,7 +682,7 @@ int cobalt_permute_rows_block(const void* x, const int32_t* row_of_pair, int64_t
     if (!x || !row_of_pair || !send) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send) || !aligned16(row_of_pair)) return COBALT_ERR_INVALID_ARG;
     const uint32_t impl = flags & COBALT_IMPL_MASK;
-    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK && impl != COBALT_IMPL_BULK_RING)
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK)
         return COBALT_ERR_INVALID_ARG;
     return launch_rows(x, row_of_pair, T, K, H, send, total_rows, flags, static_cast<cudaStream_t>(stream));
 }
@@ -880,7 +705,7 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
     if (T > 0 && (!x || !send)) return COBALT_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(send)) return COBALT_ERR_INVALID_ARG;
     const uint32_t impl = flags & COBALT_IMPL_MASK;
-    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK && impl != COBALT_IMPL_BULK_RING)
+    if (impl != 0 && impl != COBALT_IMPL_VECTOR && impl != COBALT_IMPL_BULK)
         return COBALT_ERR_INVALID_ARG;
     int rc = cobalt_permute_index(assigned_slot, T, K, D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
                                   workspace, workspace_bytes, stream);

@@ -388,7 +388,7 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
     int64_t want = (T + kRouteChunkTokens - 1) / kRouteChunkTokens;   // one chunk per CTA while CTAs last
     if (want < 16) want = 16;      // a full cluster at least: CTAs without tokens still share the merge
     if (want > n_sm) want = n_sm;
-    const auto key = std::make_tuple(dev, lv.E, lv.D, want * 1024 + lv.words % 1024);
+    const auto key = std::make_tuple(dev, static_cast<int>(smem), lv.D, want);
     {
         std::lock_guard<std::mutex> guard(cache_lock);
         auto it = cache.find(key);
@@ -598,12 +598,12 @@ static ChunkPlan route_chunks(int64_t T, int32_t K)
 }
 
 // 0: the triangle does not fit beside the tables, 1: it fits with 32-bit counters, 2: with 16-bit ones
-static int fused_mode(const LayoutView& lv)
+static int fused_mode(const LayoutView& lv, uint32_t tile_flags)
 {
     // from about 180 experts on the 16-bit triangle is taken even where the 32-bit one fits: the merge
     // is bound by the bytes that cross distributed shared memory
     const bool large_tile = tri_entries(lv.E) * sizeof(uint32_t) >= 64 * 1024;
-    if (large_tile && g_tune.stats_packed != 0 && route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
+    if (large_tile && !(tile_flags & COBALT_STATS_TILE32) && route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
     if (route_smem(lv, false).bytes() <= kRouteMaxSmem) return 1;
     if (route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
     return 0;
@@ -619,7 +619,7 @@ size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t
 {
     if (!layout || T < 0 || K < 1 || K > COBALT_MAX_TOPK || T * static_cast<int64_t>(K) >= (1ll << 31)) return 0;
     const LayoutView& lv = layout->view;
-    const int mode = fused_mode(lv);
+    const int mode = fused_mode(lv, 0);
     if (mode == 0 || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
     const ChunkPlan c = route_chunks(T, K);
     const size_t fused = round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
@@ -645,7 +645,8 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         !aligned16(assigned_slot) || !aligned16(totals) || !aligned16(dest_counts) || !aligned16(dest_offsets) ||
         !aligned16(row_of_pair) || !aligned16(pair_of_row) || !aligned16(workspace))
         return COBALT_ERR_INVALID_ARG;
-    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_SEED_ON_DEVICE)) return COBALT_ERR_INVALID_ARG;
+    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_SEED_ON_DEVICE | COBALT_STATS_TILE32 | COBALT_ROUTE_GENERAL_KERNELS))
+        return COBALT_ERR_INVALID_ARG;
     const bool seed_on_device = (flags & COBALT_SEED_ON_DEVICE) != 0;
     if (seed_on_device && (seed == 0 || (seed & 7u) != 0)) return COBALT_ERR_INVALID_ARG;
     const size_t need = cobalt_route_index_workspace_bytes(layout, T, K);
@@ -655,7 +656,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     if (dev != layout->device) return COBALT_ERR_INVALID_ARG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int mode = fused_mode(lv);
+    const int mode = fused_mode(lv, flags & COBALT_STATS_TILE32);
     bool launched = false;
     const ChunkPlan c = route_chunks(T, K);
     // The kernel is compiled for K = 1, 2, 4, 6, 8, 10, 12, 16 with the K ids of a token in registers; its variant
@@ -678,7 +679,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         if (rc != COBALT_OK) return rc;
         rc = sm_count(&a.n_sm);
         if (rc != COBALT_OK) return rc;
-        if (g_tune.route_small != 0 && K <= 8) {
+        if (!(flags & COBALT_ROUTE_GENERAL_KERNELS) && K <= 8) {
             const SmallArgs b = {dest_counts, dest_offsets, row_of_pair, pair_of_row, (flags & COBALT_STATS_ACCUMULATE) != 0};
             bool small = false;
             switch (K) {

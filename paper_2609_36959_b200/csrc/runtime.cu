@@ -1,17 +1,15 @@
 // Status codes, the device error word and the expert-layout handle.
 #include <stdlib.h>
-#include <string.h>
 
 #include <map>
 #include <mutex>
+#include <new>
 #include <utility>
 #include <vector>
 
 #include "common.cuh"
 
 namespace cobalt {
-
-Tuning g_tune;
 
 static thread_local int g_last_cuda_error = 0;
 
@@ -85,7 +83,7 @@ static int build_tables(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
                         const int32_t* primary_in, LayoutView* view, std::vector<uint32_t>* blob)
 {
     if (!slot_expert || N < 1 || Q < 1 || S < 1 || E < 1) return COBALT_ERR_INVALID_ARG;
-    if (N > COBALT_MAX_NODES || E > COBALT_MAX_EXPERTS || Q > 255) return COBALT_ERR_UNSUPPORTED;
+    if (N > COBALT_MAX_NODES || E > COBALT_MAX_EXPERTS || Q > COBALT_MAX_RANKS_PER_NODE) return COBALT_ERR_UNSUPPORTED;
     const int64_t D64 = static_cast<int64_t>(N) * Q * S;
     if (D64 > COBALT_MAX_DESTS) return COBALT_ERR_UNSUPPORTED;
     const int32_t G = N * Q, D = static_cast<int32_t>(D64);
@@ -168,31 +166,12 @@ const char* cobalt_status_string(int status)
         case COBALT_ERR_UNSUPPORTED: return "outside the supported size envelope";
         case COBALT_ERR_CUDA: return "CUDA runtime error";
         case COBALT_ERR_SCRATCH_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
+        case COBALT_ERR_HOST_ALLOC: return "host memory allocation failed";
         default: return "unknown status";
     }
 }
 
 int cobalt_version(void) { return COBALT_VERSION; }
-
-// Not part of the public header: sets one of the sweep knobs of cobalt::Tuning by name.
-int cobalt_internal_tune(const char* key, int value)
-{
-    if (!key) return COBALT_ERR_INVALID_ARG;
-    if (!strcmp(key, "rows_item_bytes")) g_tune.rows_item_bytes = value;
-    else if (!strcmp(key, "rows_stages")) g_tune.rows_stages = value;
-    else if (!strcmp(key, "rows_stage_bytes")) g_tune.rows_stage_bytes = value;
-    else if (!strcmp(key, "rows_per_sm")) g_tune.rows_per_sm = value;
-    else if (!strcmp(key, "rows_vec_per_sm")) g_tune.rows_vec_per_sm = value;
-    else if (!strcmp(key, "rows_hint")) g_tune.rows_hint = value;
-    else if (!strcmp(key, "stats_max_ctas")) g_tune.stats_max_ctas = value;
-    else if (!strcmp(key, "stats_cluster")) g_tune.stats_cluster = value;
-    else if (!strcmp(key, "stats_packed")) g_tune.stats_packed = value;
-    else if (!strcmp(key, "route_small")) g_tune.route_small = value;
-    else if (!strcmp(key, "stats_tokens_per_cta")) g_tune.stats_tokens_per_cta = value;
-    else if (!strcmp(key, "combine_per_sm")) g_tune.combine_per_sm = value;
-    else return COBALT_ERR_INVALID_ARG;
-    return COBALT_OK;
-}
 
 int cobalt_last_cuda_error(void) { return g_last_cuda_error; }
 
@@ -200,7 +179,11 @@ int cobalt_layout_check(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
                         const int32_t* primary_slot_host)
 {
     LayoutView view;
-    return build_tables(N, Q, S, E, slot_expert_host, primary_slot_host, &view, nullptr);
+    try {
+        return build_tables(N, Q, S, E, slot_expert_host, primary_slot_host, &view, nullptr);
+    } catch (const std::bad_alloc&) {
+        return COBALT_ERR_HOST_ALLOC;
+    }
 }
 
 int cobalt_layout_create(cobalt_layout_t** out, int32_t N, int32_t Q, int32_t S, int32_t E,
@@ -210,7 +193,12 @@ int cobalt_layout_create(cobalt_layout_t** out, int32_t N, int32_t Q, int32_t S,
     *out = nullptr;
     LayoutView view;
     std::vector<uint32_t> blob;
-    int rc = build_tables(N, Q, S, E, slot_expert_host, primary_slot_host, &view, &blob);
+    int rc = COBALT_OK;
+    try {
+        rc = build_tables(N, Q, S, E, slot_expert_host, primary_slot_host, &view, &blob);
+    } catch (const std::bad_alloc&) {
+        return COBALT_ERR_HOST_ALLOC;
+    }
     if (rc != COBALT_OK) return rc;
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
@@ -224,7 +212,7 @@ int cobalt_layout_create(cobalt_layout_t** out, int32_t N, int32_t Q, int32_t S,
     cobalt_layout* h = static_cast<cobalt_layout*>(malloc(sizeof(cobalt_layout)));
     if (!h) {
         cudaFree(dptr);
-        return COBALT_ERR_INVALID_ARG;
+        return COBALT_ERR_HOST_ALLOC;
     }
     view.blob = static_cast<const uint32_t*>(dptr);
     h->view = view;

@@ -37,10 +37,20 @@ def test_library_exports_every_declared_symbol(lib_path, cb):
     assert sorted(cb.EXPORTS) == names
 
 
+def test_library_exports_nothing_beyond_the_header(lib_path):
+    """The dynamic symbol table lists exactly the header's cobalt_* functions: no tuning hooks or
+    other undeclared entry points ship in the library."""
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", lib_path], capture_output=True, text=True, check=True).stdout
+    exported = sorted({line.split()[-1] for line in out.splitlines()
+                       if line.split() and line.split()[-1].startswith("cobalt_") and " T " in line})
+    assert exported == declared_symbols()
+
+
 def test_version_and_status_strings(cb):
     assert cb.version() == 100
-    seen = {cb.status_string(s) for s in (0, -1, -2, -3, -4)}
-    assert len(seen) == 5 and "unknown status" not in seen
+    seen = {cb.status_string(s) for s in (0, -1, -2, -3, -4, -5, -6)}
+    assert len(seen) == 7 and "unknown status" not in seen
     assert cb.status_string(-99) == "unknown status"
 
 

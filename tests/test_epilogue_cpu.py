@@ -43,3 +43,13 @@ def test_rebalancer_with_ties_and_empty_slots(cb):
         new, moved, kept = cb.rebalance_intra_node(N, Q, S, E, w.slot_expert.tolist(), load.tolist())
         ref_new, ref_moved, ref_kept = O.rebalance_intra_node(N, Q, S, w.slot_expert, load)
         assert new == ref_new.tolist() and moved == ref_moved.tolist() and kept == len(ref_kept)
+
+
+@pytest.mark.parametrize("bad", [float("nan"), float("inf"), -1.0])
+def test_rebalancer_refuses_loads_that_cannot_be_ordered(cb, bad):
+    """A NaN load would leave the longest-first sort without a strict weak order: such inputs are
+    refused as invalid arguments instead (empty slots may hold anything)."""
+    with pytest.raises(cb.CobaltError) as err:
+        cb.rebalance_intra_node(1, 2, 2, 4, [0, 1, 2, 3], [10, bad, 5, 3])
+    assert err.value.status == cb.ERR_INVALID_ARG
+    assert cb.rebalance_intra_node(1, 2, 2, 3, [0, 1, 2, -1], [3, 2, 1, bad])[2] == 0

@@ -57,7 +57,7 @@ def test_config_full_elementwise(cb, name):
     r, p = check_index_stages(cb, w, step, w.seed)
 
     x = w.hidden_rows()
-    for impl in (cb.IMPL_BULK, cb.IMPL_BULK_RING, cb.IMPL_VECTOR, 0):
+    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR, 0):
         step.send.zero_()
         step.permute(flags=impl)
         torch.cuda.synchronize()
@@ -114,10 +114,28 @@ def test_config_full_size_sampled(cb, name):
     # every send row equals the row of the token its pair belongs to (checked on the device)
     tok_of_row = (step.pair_of_row // w.K).long()
     n_chunk = 1 << 16
-    for r0 in range(0, w.P, n_chunk * 16):
+    for r0 in range(0, w.P, n_chunk):
         r1 = min(w.P, r0 + n_chunk)
         same = step.send[r0:r1].view(torch.int16) == step.x[tok_of_row[r0:r1]].view(torch.int16)
         assert bool(same.all())
+    del diff, bound, same
+
+    # the combine once more at this full shape with expert outputs of their own (not the send buffer):
+    # seeded N(0,1) rows drawn on the device; only the sampled tokens' rows come back for the oracle
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(int(w.seed) + 7)
+    expert_out = torch.empty_like(step.send)
+    blk = 1 << 16
+    for r0 in range(0, w.P, blk):
+        r1 = min(w.P, r0 + blk)
+        expert_out[r0:r1] = torch.randn((r1 - r0, w.H), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    step.y.zero_()
+    cb.combine(expert_out, step.row_of_pair, step.gate_w, step.y)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    rows_needed = bits_from_bf16_tensor(expert_out[torch.from_numpy(rop.ravel()).cuda()])
+    y_ref = O.combine(rows_needed, np.arange(rop.size, dtype=np.int32), w.gate_w[tokens])
+    assert_combine_close(bits_from_bf16_tensor(step.y[torch.from_numpy(tokens).cuda()]), y_ref)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -148,7 +166,7 @@ def test_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     layout, step = make_step(w, alias_expert_out=False)
     r, p = check_index_stages(cb, w, step, 4242)
     x = w.hidden_rows()
-    for impl in (cb.IMPL_BULK, cb.IMPL_BULK_RING, cb.IMPL_VECTOR):
+    for impl in (cb.IMPL_BULK, cb.IMPL_VECTOR):
         step.send.zero_()
         step.permute(flags=impl)
         torch.cuda.synchronize()
@@ -216,23 +234,19 @@ def test_statistics_many_tokens_and_a_large_triangle(cb, E, K, T, tile):
 def test_statistics_with_sixteen_bit_tiles_forced(cb, E, K, T):
     """The 16-bit tile, chosen by default only where the 32-bit one does not fit, gives the same counts
     at every size; T = 700000 exceeds what it may count and must take the 32-bit tile by itself."""
-    import ctypes
-    tune = cb.binding._lib.cobalt_internal_tune
-    tune.argtypes = [ctypes.c_char_p, ctypes.c_int]
     model = W.configs.ClusterModel(E, K, 4, 0.7, np.full(4, 1 / 4), np.ones(E))
     ids = W.sample_topk_ids(model, T, seed=3 * E + K)
     ids_d = torch.from_numpy(ids).cuda()
     coact = torch.full((E, E), 7, dtype=torch.int32, device="cuda")
     load = torch.full((E,), 7, dtype=torch.int32, device="cuda")
-    assert tune(b"stats_packed", 1) == 0
-    try:
-        cb.coact_stats(ids_d, E, coact, load)
-        torch.cuda.synchronize()
-    finally:
-        assert tune(b"stats_packed", -1) == 0
-    assert cb.read_and_clear_device_error() == 0
     ref_coact, ref_load = O.coact_stats(ids, E)
-    assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
+    for flags in (cb.STATS_TILE16, cb.STATS_TILE32):
+        coact.fill_(7)
+        load.fill_(7)
+        cb.coact_stats(ids_d, E, coact, load, flags=flags)
+        torch.cuda.synchronize()
+        assert cb.read_and_clear_device_error() == 0
+        assert (u32(coact) == ref_coact).all() and (u32(load) == ref_load).all()
 
 
 @pytest.mark.parametrize("E,K,T", [(256, 8, 3000), (64, 6, 1), (300, 4, 4096), (400, 8, 2500)])
@@ -292,7 +306,7 @@ def test_naive_rule_and_uniform_source(cb):
     assert (out.cpu().numpy() == r["assigned_slot"]).all()
 
 
-def run_fused_and_compare(cb, w, step, seed):
+def run_fused_and_compare(cb, w, step, seed, flags=0):
     coact, load = O.coact_stats(w.topk_ids, w.E)
     r = oracle_assign(w, seed)
     p = O.permute(r["assigned_slot"], w.D)
@@ -301,7 +315,7 @@ def run_fused_and_compare(cb, w, step, seed):
         buf.fill_(77)
     cb.route_index(step.layout, step.topk_ids, step.src_rank, seed, step.coact, step.load, step.assigned_slot,
                    step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
-                   remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+                   remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row, flags=flags)
     torch.cuda.synchronize()
     assert cb.read_and_clear_device_error() == 0
     assert (u32(step.coact) == coact).all() and (u32(step.load) == load).all()
@@ -361,21 +375,14 @@ def test_step_with_statistics_on_a_side_stream(cb):
 def test_fused_pass_in_a_single_cluster(cb, T, E, K, N, Q, S, empty):
     """Up to 16 chunks of 256 tokens the fused entry runs ONE kernel in one cluster (histograms
     exchanged through distributed shared memory, statistics stored instead of added).  Same results
-    as the oracle, as the general kernels (switched to with the sweep knob), and with the
+    as the oracle, as the general kernels (COBALT_ROUTE_GENERAL_KERNELS), and with the
     accumulate flag on top of what is already there."""
-    import ctypes
-    tune = cb.binding._lib.cobalt_internal_tune
-    tune.argtypes = [ctypes.c_char_p, ctypes.c_int]
     w = W.make_custom(T, E, K, 8, N, Q, S, seed=900 + T, C=2, p_in=0.7, n_empty=empty)
     layout, step = make_step(w, with_x=False)
     run_fused_and_compare(cb, w, step, 321)
     small = {k: getattr(step, k).clone() for k in ("coact", "load", "assigned_slot", "dest_counts", "dest_offsets",
                                                      "row_of_pair", "pair_of_row", "remote_nodes", "totals")}
-    assert tune(b"route_small", 0) == 0
-    try:
-        run_fused_and_compare(cb, w, step, 321)
-    finally:
-        assert tune(b"route_small", 1) == 0
+    run_fused_and_compare(cb, w, step, 321, flags=cb.ROUTE_GENERAL_KERNELS)
     for k, v in small.items():
         assert torch.equal(getattr(step, k), v), k
     cb.route_index(layout, step.topk_ids, step.src_rank, 321, step.coact, step.load, step.assigned_slot,
@@ -546,7 +553,7 @@ def test_results_do_not_depend_on_the_run(cb):
     step.route(w.seed)
     torch.cuda.synchronize()
     ref = [t.clone() for t in (step.coact, step.assigned_slot, step.row_of_pair, step.pair_of_row, step.send, step.y)]
-    for _ in range(5):
+    for _ in range(20):
         step.route(w.seed)
         torch.cuda.synchronize()
         for a, b in zip(ref, (step.coact, step.assigned_slot, step.row_of_pair, step.pair_of_row, step.send, step.y)):

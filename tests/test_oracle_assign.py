@@ -128,7 +128,7 @@ def test_fig1_naive_rule(fig1):
     assert (r["assigned_slot"] == np.array(g["primary_slot"])[ids]).all()
 
 
-# ---------------------------------------------------------------- tie-break of lines 5-8 --
+# ------------------------------------------------- tie-break among covers of equal size --
 def _layout_from_nodes(expert_nodes, N):
     """One rank per node (Q = 1), S = number of experts: expert e sits on the listed nodes."""
     E = len(expert_nodes)
@@ -253,6 +253,39 @@ def test_alg1_matches_bruteforce_minimum(N, Q, S, E, K, seed):
         assert r["remote_nodes"][t] == best, t
 
 
+@pytest.mark.parametrize("N,Q,S,E,K,seed", [(5, 1, 3, 12, 4, 11), (6, 1, 3, 15, 4, 12), (7, 1, 2, 12, 4, 13),
+                                           (8, 1, 2, 14, 4, 14), (8, 2, 1, 14, 4, 15)])
+def test_alg1_matches_bruteforce_minimum_with_many_nodes(N, Q, S, E, K, seed):
+    """The same pin with five to eight nodes, where covers of three and four remote nodes occur
+    (most experts sit on a single node, so four experts can need four nodes)."""
+    w = W.make_custom(150, E, K, 8, N, Q, S, seed=seed, C=1)
+    r = O.assign(N, Q, S, E, w.slot_expert, None, w.topk_ids, w.src_rank, 99)
+    seen = set()
+    for t in range(w.T):
+        best = O.min_remote_nodes_bruteforce(w.slot_expert.tolist(), S, Q, w.topk_ids[t].tolist(),
+                                             int(w.src_rank[t]))
+        assert r["remote_nodes"][t] == best, t
+        seen.add(best)
+    assert {3, 4} <= seen or (N == 5 and 3 in seen), seen     # the larger covers really are exercised
+
+
+def test_cover_of_every_remote_node():
+    """Eight nodes, seven experts each alone on its own remote node: the only cover is all of them.
+    Adding a replica of two of them on one node brings the cover down by one."""
+    N, Q, S, E = 8, 1, 2, 7
+    slot = -np.ones(N * Q * S, np.int32)
+    for e in range(7):
+        slot[(e + 1) * S] = e                       # expert e alone on node e + 1
+    ids = np.arange(7, dtype=np.int32)[None, :]
+    src = np.zeros(1, np.int32)
+    r = O.assign(N, Q, S, E, slot, None, ids, src, 1)
+    assert r["remote_nodes"][0] == 7 and (r["assigned_slot"][0] == (np.arange(7) + 1) * S).all()
+    slot[1 * S + 1] = 6                             # expert 6 also on node 1 (which holds expert 0)
+    r = O.assign(N, Q, S, E, slot, None, ids, src, 1)
+    assert r["remote_nodes"][0] == 6 and r["assigned_slot"][0][6] == 1 * S + 1
+    assert O.min_remote_nodes_bruteforce(slot.tolist(), S, Q, list(range(7)), 0) == 6
+
+
 def test_bruteforce_on_fig1(fig1):
     g = fig1
     for tk in g["tokens"]:
@@ -261,7 +294,8 @@ def test_bruteforce_on_fig1(fig1):
 
 # ---------------------------------------------------------------- randomness --------------
 def test_replica_pick_is_uniform_within_node():
-    """'Replicas of the same expert within a node receive equal workloads in expectation'."""
+    """The replica pick inside a node is uniform (Section 3.3, Step 2): every replica of an expert on
+    one node gets the same share of its tasks up to sampling noise."""
     # one node, 4 ranks, expert 0 on all four ranks, expert 1 on ranks 0 and 2
     slot = np.array([0, 1, 0, -1, 0, 1, 0, -1], np.int32)
     T = 8000
