@@ -70,7 +70,7 @@ extern "C" {
 #define COBALT_DEVERR_DUPLICATE_ID 0x2u      /* an expert listed twice in one token */
 #define COBALT_DEVERR_BAD_SRC_RANK 0x4u      /* source rank outside [0, G) */
 #define COBALT_DEVERR_BAD_SLOT 0x8u          /* assigned slot / row index outside its range */
-#define COBALT_DEVERR_WAIT_TIMEOUT 0x10u     /* a bounded on-chip wait ran out (copy pipeline) */
+#define COBALT_DEVERR_WAIT_TIMEOUT 0x10u     /* a bounded wait ran out (copy pipeline, grid barrier of the fused pass) */
 
 /* flag bits */
 #define COBALT_STATS_ACCUMULATE 0x1u         /* add to coact/load instead of overwriting them */
@@ -83,7 +83,7 @@ extern "C" {
                                                 they cannot overflow (default: only where that is faster or the
                                                 32-bit tile does not fit) */
 #define COBALT_STATS_TILE32 0x20u            /* cobalt_coact_stats, cobalt_route_index: 32-bit counters wherever the tile fits */
-#define COBALT_ROUTE_GENERAL_KERNELS 0x40u   /* cobalt_route_index: do not take the single-cluster kernel for small batches */
+#define COBALT_ROUTE_SEPARATE_KERNELS 0x40u  /* cobalt_route_index: run the three separate calls instead of the fused kernel */
 #define COBALT_IMPL_MASK 0xF00u              /* row-kernel variant override, 0 = library default */
 #define COBALT_IMPL_VECTOR 0x100u            /* row movement with plain 16-byte loads/stores */
 #define COBALT_IMPL_BULK 0x200u              /* row movement with bulk async copies, one work item per CTA (default) */
@@ -201,13 +201,18 @@ int cobalt_permute(const int32_t* assigned_slot, int64_t T, int32_t K, int32_t D
 /* ---- stages 1 + 2 + index half of stage 3 in one pass over the ids ---------------------------
  * Same outputs, bit for bit, as cobalt_coact_stats, cobalt_assign (Algorithm 1, hashed replica
  * pick) and cobalt_permute_index called one after the other, with dest_counts = slot_load = w_er.
- * The top-k ids are read once and the co-activation triangle, the layout tables and the chunk
- * histograms of the permutation share one cluster-launched kernel; the scan and stable-rank
- * kernels follow.  (Section 3.2 Stage 1, Section 3.3 Algorithm 1, Fig. 1 "Dispatch".)
- * The one-pass kernel exists for K = 1, 2, 4, 6, 8, 10, 12, 16 and for layouts whose triangle fits beside the
- * tables (up to about 440 experts); every other case runs the three separate calls internally,
- * with the same results.  The workspace query covers both.
- * flags: COBALT_STATS_ACCUMULATE, COBALT_SEED_ON_DEVICE, COBALT_STATS_TILE32, COBALT_ROUTE_GENERAL_KERNELS
+ * (Section 3.2 Stage 1, Section 3.3 Algorithm 1, Fig. 1 "Dispatch".)  ONE kernel does it: a grid of
+ * at most one CTA per SM, launched cooperatively, reads the top-k ids once, keeps the co-activation
+ * triangle, the layout tables and the lane masks that rank the pairs in shared memory, exchanges
+ * per-CTA partial results through the workspace across one grid-wide barrier (bounded wait:
+ * COBALT_DEVERR_WAIT_TIMEOUT if it ever ran out) and stores every output; nothing is cleared
+ * beforehand and no output is written with atomics unless COBALT_STATS_ACCUMULATE is set.
+ * The kernel serves K = 1 .. 16, D <= 1024 and layouts whose triangle fits beside the other tables
+ * (about 400 experts at D = 288, fewer with more destinations), on devices that support
+ * cooperative launches; every other case runs the three separate calls internally, with the same
+ * results.  The workspace query covers both (about 10 MB at E = 256, D = 288).  Two calls that
+ * run on the GPU at the same time need a workspace each.
+ * flags: COBALT_STATS_ACCUMULATE, COBALT_SEED_ON_DEVICE, COBALT_STATS_TILE32, COBALT_ROUTE_SEPARATE_KERNELS
  * (the last two select kernel variants, not results).  remote_nodes, totals, pair_of_row may be NULL.
  * Follow with cobalt_permute_rows to fill the send buffer. */
 size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t T, int32_t K);

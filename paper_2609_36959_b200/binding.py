@@ -37,7 +37,7 @@ ASSIGN_ROUND_ROBIN = 0x2
 SEED_ON_DEVICE = 0x4
 STATS_TILE16 = 0x10
 STATS_TILE32 = 0x20
-ROUTE_GENERAL_KERNELS = 0x40
+ROUTE_SEPARATE_KERNELS = 0x40
 EMA_INITIALISE = 0x1
 IMPL_VECTOR = 0x100
 IMPL_BULK = 0x200

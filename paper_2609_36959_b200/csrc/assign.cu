@@ -112,8 +112,8 @@ assign_round_robin_kernel(LayoutView lv, const int32_t* __restrict__ group_rank,
         const int32_t key = key_to_slot[p];
         if (key < 0) continue;                       // a token that failed its checks
         const uint32_t e_n = tv.ent[key];
-        const uint32_t j = static_cast<uint32_t>(__ldg(group_rank + p)) % (e_n & 0xFFu);
-        const int32_t slot = static_cast<int32_t>(tv.rlist[(e_n >> 8) + j]);
+        const uint32_t j = static_cast<uint32_t>(__ldg(group_rank + p)) % ent_count(e_n);
+        const int32_t slot = static_cast<int32_t>(tv.rlist[ent_offset(e_n) + j]);
         key_to_slot[p] = slot;
         if (slot_load) atomicAdd(&hist[slot], 1u);
     }

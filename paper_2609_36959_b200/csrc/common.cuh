@@ -40,19 +40,28 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Device tables built from a layout (Section 3.3: R_{e,n} and N_e), one contiguous blob of
 // 32-bit words that kernels copy into shared memory:
-//   ent[e*N + n]   = (offset into rlist << 8) | |R_{e,n}|
-//   primary[e]     = slot of e's primary replica | (its node << 24)
+//   ent[e*N + n]   bits 0-7   |R_{e,n}|
+//                  bits 8-20  offset of R_{e,n} in rlist
+//                  bits 21-27 m_{e,n}: the remote-node mask of e seen from source node n (bit j = j-th
+//                             node in ascending id with n skipped); 0 when n itself holds e
+//                  bits 28-30 node of e's primary replica
+//   primary[e]     = slot of e's primary replica
 //   rlist[...]     = slots of R_{e,n}, ascending, all (e, n) groups back to back
-//   nodes[e]       = bitmask over nodes holding e (one word each)
+//   cover[...]     = 128 bytes, only for N <= 4: the smallest cover b* for every set of mask values that
+//                    can occur in a token (bit v-1 of the index set iff some expert of U_t has mask v)
+constexpr int kEntCountBits = 8, kEntOffsetBits = 13, kEntMaskShift = 21, kEntPrimaryNodeShift = 28;
+constexpr int kCoverTableWords = 32;
+
 struct LayoutView {
     int32_t N, Q, S, E, G, D;
     int32_t n_replicas;       // entries of rlist
     int32_t words;            // total 32-bit words of the blob
+    uint32_t q_inverse;       // floor(s * q_inverse / 2^20) = s / Q for every source rank s in [0, G)
     const uint32_t* blob;     // device
     __host__ __device__ int ent_off() const { return 0; }
     __host__ __device__ int primary_off() const { return E * N; }
     __host__ __device__ int rlist_off() const { return E * N + E; }
-    __host__ __device__ int nodes_off() const { return E * N + E + n_replicas; }
+    __host__ __device__ int cover_off() const { return E * N + E + n_replicas; }
 };
 
 }  // namespace cobalt

@@ -1,115 +1,298 @@
-// Fused index pass: statistics (stage 1), assignment (stage 2) and the per-chunk destination
-// histograms of the permutation (first kernel of stage 3) in ONE pass over the top-k ids.
+// Fused index pass: statistics (stage 1), assignment (stage 2) and the index half of the permutation
+// (stage 3) in ONE kernel and one pass over the top-k ids.
 //
-// The separate entry points read the ids three times and launch six kernels before the scan;
-// for the few megabytes involved those launches, not the bytes, set the time.  Here one
-// cluster-launched kernel keeps, per CTA, the co-activation triangle, the layout tables and the
-// chunk histograms in shared memory; every thread owns one token per round: it adds the token's
-// K(K+1)/2 pairs to the triangle, runs Algorithm 1, stores the K slots and counts them in the
-// histogram of its permutation chunk (256 consecutive tokens = 8 warps).  The triangle is then
-// merged over the cluster exactly as in the stand-alone statistics kernel; the scan and rank
-// kernels of the permutation follow.  Batches of at most 16 chunks run in a second kernel that does
-// all of it, scan and rank included, in one cluster (route_small_kernel).  Results are bit-identical
-// to the separate calls.
-#include <cooperative_groups.h>
-
+// The separate entry points read the ids three times and launch seven kernels; for the few megabytes
+// involved those launches and the dependent-latency chains between them, not the bytes, set the time.
+// Here a grid of at most one CTA per SM (1024 threads, launched cooperatively so that all of it is
+// resident) does everything:
+//
+//   phase 1  every CTA owns a contiguous range of tokens, one token per thread and round: the
+//            token's K(K+1)/2 pairs go into the CTA's private co-activation triangle in shared
+//            memory, Algorithm 1 picks its K slots (stored, and counted per destination).
+//   publish  the CTA writes its triangle, its destination counts and its Eq. 1 sums to the
+//            workspace (plain coalesced stores).  Then ONE grid-wide barrier (bounded wait).
+//   phase 2  every CTA sums a slice of the triangle over all CTAs' partials and STORES coact / load
+//            (no atomics on the outputs, nothing to clear beforehand); it derives, from all CTAs'
+//            destination counts, the offsets and the first row of its own tokens inside every
+//            destination; and ranks its pairs.  A token sends at most one pair to a destination
+//            (its experts, hence its slots, are distinct), so the rows of one destination inside a
+//            warp's 32 tokens are ordered by lane: each lane ORs its bit into a per-destination lane
+//            mask, and a pair's rank is the popcount of the lower lanes -- no sorting, no position
+//            atomics, and the result is the stable order by construction.  The inverse map is
+//            staged in shared memory in row order, so that its stores run along rows.
+//
+// Results are bit-identical to cobalt_coact_stats + cobalt_assign + cobalt_permute_index.
 #include <algorithm>
+#include <atomic>
 #include <map>
 #include <mutex>
-#include <tuple>
 #include <utility>
 
 #include "permute_index.cuh"
 #include "token_core.cuh"
 
-namespace cg = cooperative_groups;
-
 namespace cobalt {
 
 constexpr int kRouteThreads = 1024;
-constexpr int kRouteChunkTokens = 256;                              // tokens per permutation chunk
-constexpr int kRouteChunksPerRound = kRouteThreads / kRouteChunkTokens;
+constexpr int kRouteWarps = kRouteThreads / 32;
 constexpr size_t kRouteMaxSmem = 220 * 1024;
+constexpr int kRouteMaxCtas = 160;                  // the workspace is sized for grids up to this
+constexpr int kRouteMaxDests = kRouteThreads;       // one destination per thread in the scans over d
+constexpr uint32_t kBarrierSpinLimit = 1u << 22;    // polls of the grid barrier before giving up (about a second)
 
+// Shared memory of one CTA, in 32-bit words.
 struct RouteSmem {
-    size_t tri_words, tab_words, hist_words;
-    size_t bytes() const { return (tri_words + tab_words + hist_words) * sizeof(uint32_t); }
+    size_t tri_words;     // co-activation triangle (16- or 32-bit counters), whole 16-byte vectors; after the
+                          // grid barrier: the sums of this CTA's slice, then partial destination sums
+    size_t stage_words;   // the inverse map of one round in row order (1024 K entries)
+    size_t tab_words;     // layout tables
+    size_t dest_words;    // D rounded up to a multiple of 8
+    size_t lane_stride;   // entries per warp of the lane-mask table: D rounded up to an odd number
+    // tri | stage | tab | cnt[dest] | base[dest] | excl[dest] | wm[warps][lane_stride] (two words each)
+    size_t words() const { return tri_words + stage_words + tab_words + 3 * dest_words + 2 * kRouteWarps * lane_stride; }
+    size_t bytes() const { return words() * sizeof(uint32_t); }
 };
 
-static RouteSmem route_smem(const LayoutView& lv, bool packed)
+static RouteSmem route_smem(const LayoutView& lv, int K, bool packed)
 {
     RouteSmem r;
     r.tri_words = ((packed ? (tri_entries(lv.E) + 1) / 2 : tri_entries(lv.E)) + 3) / 4 * 4;
+    r.stage_words = static_cast<size_t>(kRouteThreads) * K;
     r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
-    r.hist_words = static_cast<size_t>(kRouteChunksPerRound) * lv.D;
+    r.dest_words = static_cast<size_t>(lv.D + 7) / 8 * 8;
+    r.lane_stride = static_cast<size_t>(lv.D) | 1u;
     return r;
 }
 
-// kPacked: 16-bit counters in the triangle (see the statistics kernel); the launcher allows it only
-// while one cluster sees at most 65535 tokens.
+// Workspace of the fused kernel (byte offsets, 256-byte aligned).
+struct RouteWorkspace {
+    size_t barrier_off, cnt_off, tot_off, tri_off, total;
+};
+
+static RouteWorkspace route_workspace(const LayoutView& lv, bool packed)
+{
+    const RouteSmem sm = route_smem(lv, 1, packed);
+    RouteWorkspace w;
+    size_t off = 0;
+    w.barrier_off = off; off += 256;
+    w.cnt_off = off;     off += round_up(sizeof(uint16_t) * kRouteMaxCtas * sm.dest_words, 256);
+    w.tot_off = off;     off += round_up(sizeof(unsigned long long) * 2 * kRouteMaxCtas, 256);
+    w.tri_off = off;     off += round_up(sizeof(uint32_t) * kRouteMaxCtas * sm.tri_words, 256);
+    w.total = off;
+    return w;
+}
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide barrier on one 64-bit word of the workspace: epoch (high half) and arrival count.
+// The word may hold anything when the kernel starts.  CTA 0 sets it to (epoch, 0) first thing; a CTA
+// arrives by adding one and learns from the value it gets back whether the word already carried
+// this launch's epoch.  If not (it arrived before CTA 0's store landed: its increment is lost with
+// the old contents), it waits for the epoch to appear and adds again.  Every CTA of the grid is
+// resident (cooperative launch), so the wait ends as soon as the slowest CTA has arrived; it is
+// bounded all the same, and a wait that runs out reports COBALT_DEVERR_WAIT_TIMEOUT and makes the
+// CTA return.  After the wait every CTA signs off on the same word and the last one clears it, so
+// that a replay of a captured launch (same epoch) starts from a word that differs from its epoch.
+// All three are called by all threads of the CTA.
+__device__ __forceinline__ void grid_barrier_init(unsigned long long* word, uint32_t epoch)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicExch(word, static_cast<unsigned long long>(epoch) << 32);
+}
+
+// Returns false on a timeout.
+__device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t n_ctas,
+                                             uint32_t* err_word)
+{
+    __shared__ int barrier_ok;
+    __syncthreads();                       // this CTA's writes are done ...
+    if (threadIdx.x == 0) {
+        __threadfence();                   // ... and visible to the grid before the arrival is
+        const unsigned long long target = (static_cast<unsigned long long>(epoch) << 32) | n_ctas;
+        bool counted = (atomicAdd(word, 1ull) >> 32) == epoch;
+        bool ok = false;
+        for (uint32_t spin = 0; spin < kBarrierSpinLimit; ++spin) {
+            const unsigned long long v = ld_acquire_u64(word);
+            if ((v >> 32) == epoch) {
+                if (!counted) {
+                    counted = (atomicAdd(word, 1ull) >> 32) == epoch;
+                    continue;
+                }
+                if (v >= target) {
+                    ok = true;
+                    break;
+                }
+            }
+            __nanosleep(40);
+        }
+        if (ok) {
+            // sign off; the last CTA to do so leaves the word cleared
+            const unsigned long long before = atomicAdd(word, 1ull);
+            if (static_cast<uint32_t>(before) + 1u == 2u * n_ctas) atomicExch(word, 0ull);
+        } else {
+            flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
+        }
+        __threadfence();
+        barrier_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return barrier_ok != 0;
+}
+
+struct RouteParams {
+    LayoutView lv;
+    const int32_t* topk_ids;
+    const int32_t* src_rank;
+    int32_t src_uniform;
+    int64_t T;
+    int32_t K_rt;
+    uint32_t seed_lo, seed_hi;
+    const unsigned long long* seed_on_device;
+    uint32_t* coact;
+    uint32_t* load;
+    int32_t* assigned_slot;
+    uint8_t* remote_nodes;
+    unsigned long long* totals;
+    uint32_t* dest_counts;
+    uint32_t* dest_offsets;
+    int32_t* row_of_pair;
+    int32_t* pair_of_row;
+    // workspace
+    unsigned long long* barrier;
+    uint16_t* ws_cnt;                  // [CTAs][dest_words], 16-bit: a CTA sends at most one pair per token to a destination
+    unsigned long long* ws_tot;        // [CTAs][2]
+    uint32_t* ws_tri;                  // [CTAs][tri_words]
+    uint32_t epoch;
+    int tri_words, stage_words, tab_words, dest_words, lane_stride;
+    int tokens_per_cta;                // a multiple of 32
+    int accumulate;                    // add to coact / load instead of overwriting them
+    uint32_t* err_word;
+};
+
+// Exclusive scan over d of one value per thread (threads >= D pass 0); returns the sum of the
+// values of lower threads.  `total` receives the sum of all values.  Two block barriers.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t value, uint32_t* warp_sums, uint32_t* total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = value;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    __syncthreads();                      // warp_sums may still be read from the previous scan
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    uint32_t before = incl - value, all = 0;
+#pragma unroll
+    for (int w = 0; w < kRouteWarps; ++w) {
+        const uint32_t s = warp_sums[w];
+        if (w < warp) before += s;
+        all += s;
+    }
+    *total = all;
+    return before;
+}
+
+// One entry of the staged inverse map / of a thread's saved ranks: destination in the low bits, the
+// rest above it.
+constexpr int kDestBits = 10;
+static_assert(kRouteMaxDests <= (1 << kDestBits), "destinations must fit the packed entry");
+static_assert(kRouteThreads * COBALT_MAX_TOPK <= (1 << (32 - kDestBits - 1)), "a round's pairs must fit the packed entry");
+
 template <int KT, bool kPacked>
 __global__ void __launch_bounds__(kRouteThreads)
-route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ src_rank,
-                   int32_t src_uniform, int64_t T, int32_t K_rt, uint32_t seed_lo, uint32_t seed_hi,
-                   uint32_t* __restrict__ coact, uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot,
-                   uint8_t* __restrict__ remote_nodes, unsigned long long* __restrict__ totals,
-                   uint32_t* __restrict__ chunk_ws, int n_chunks, int tri_words, int tab_words,
-                   int chunks_per_cta, const unsigned long long* __restrict__ seed_on_device,
-                   uint32_t* __restrict__ err_word)
+route_fused_kernel(const RouteParams p)
 {
-    if (seed_on_device) {                               // the seed of this run, not of the capture
-        const unsigned long long sd = __ldg(seed_on_device);
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* tri = smem;                                      // later: acc (phase 2a), part (phase 2b)
+    uint32_t* stage = tri + p.tri_words;                       // [1024 K] the inverse map of one round, in row order
+    uint32_t* tab = stage + p.stage_words;
+    uint32_t* cnt = tab + p.tab_words;                         // [D] pairs of this CTA (round) per destination
+    uint32_t* base = cnt + p.dest_words;                       // [D] first row of this CTA's (round's) pairs inside d
+    uint32_t* excl = base + p.dest_words;                      // [D] pairs of this round in lower destinations
+    uint2* wm = reinterpret_cast<uint2*>(excl + p.dest_words); // [warps][lane_stride] x: lanes (tokens) of the warp that
+                                                               //   send to d, y: the round's pairs to d in lower warps
+    __shared__ unsigned long long cta_totals[2];
+    __shared__ uint32_t warp_sums[kRouteWarps];
+
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    const int K = (KT > 0) ? KT : p.K_rt;
+    const int D = p.lv.D, E = p.lv.E;
+    const int dest_words = p.dest_words;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = static_cast<int>(blockIdx.x), n_ctas = static_cast<int>(gridDim.x);
+    uint2* my_wm = wm + warp * p.lane_stride;
+    const uint32_t lower_lanes = (1u << lane) - 1u;
+
+    uint32_t seed_lo = p.seed_lo, seed_hi = p.seed_hi;
+    if (p.seed_on_device) {                                   // the seed of this run, not of the capture
+        const unsigned long long sd = __ldg(p.seed_on_device);
         seed_lo = static_cast<uint32_t>(sd);
         seed_hi = static_cast<uint32_t>(sd >> 32);
     }
-    extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t* tri = smem;
-    uint32_t* tab = smem + tri_words;
-    uint32_t* chist = tab + tab_words;            // [kRouteChunksPerRound][D]
-    __shared__ unsigned long long cta_totals[2];
-    constexpr int KMAX = TokenShape<KT>::KMAX;
-    const int K = (KT > 0) ? KT : K_rt;
-    const int D = lv.D;
-    cg::cluster_group cluster = cg::this_cluster();
 
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the scan kernel may be scheduled early
-    // a CTA owns chunks_per_cta consecutive chunks of 256 tokens (the batch cut evenly over the grid)
-    // and takes them in rounds of up to four, one token per thread
-    const int chunk_lo = min(n_chunks, static_cast<int>(blockIdx.x) * chunks_per_cta);
-    const int chunk_hi = min(n_chunks, chunk_lo + chunks_per_cta);
-    const int n_rounds = (chunk_hi - chunk_lo + kRouteChunksPerRound - 1) / kRouteChunksPerRound;
+    grid_barrier_init(p.barrier, p.epoch);
+    const int64_t t_lo = min(p.T, static_cast<int64_t>(cta) * p.tokens_per_cta);
+    const int64_t t_hi = min(p.T, t_lo + p.tokens_per_cta);
+    const int n_rounds = static_cast<int>((t_hi - t_lo + kRouteThreads - 1) / kRouteThreads);
+    // One round (at most 1024 tokens per CTA): the lane masks that rank the pairs are built while the
+    // slots are assigned, and everything about the ranks that needs no other CTA is done before the
+    // grid barrier is waited for.  More rounds: the slots are counted, and the ranks are worked out
+    // round by round after the barrier.
+    const bool single = n_rounds <= 1;
+
     // the first round's loads go out before the shared-memory set-up so that the two overlap
     int32_t id[KMAX], out[KMAX];
-    int32_t s_t = src_uniform;
-    {
-        const int64_t t0 = static_cast<int64_t>(chunk_lo) * kRouteChunkTokens + threadIdx.x;
-        if (static_cast<int>(threadIdx.x) < (chunk_hi - chunk_lo) * kRouteChunkTokens && t0 < T) {
-            load_token_ids<KT>(topk_ids, t0, K, id);
-            if (src_rank) s_t = __ldg(src_rank + t0);
-        }
+    int32_t s_t = p.src_uniform;
+    if (t_lo + tid < t_hi) {
+        load_token_ids<KT>(p.topk_ids, t_lo + tid, K, id);
+        if (p.src_rank) s_t = __ldg(p.src_rank + t_lo + tid);
     }
-    for (int i = threadIdx.x; i < tri_words / 4; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = threadIdx.x; i < kRouteChunksPerRound * D; i += blockDim.x) chist[i] = 0;
-    if (threadIdx.x < 2) cta_totals[threadIdx.x] = 0;
-    const TableView tv = stage_tables(lv, tab);
+    // the layout tables travel to shared memory asynchronously, behind the clearing of the other arrays
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(p.lv.blob);
+        const int n_vec = (p.lv.words + 3) / 4;
+        for (int i = tid; i < n_vec; i += kRouteThreads)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(
+                             reinterpret_cast<uint4*>(tab) + i))),
+                         "l"(src + i)
+                         : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int i = tid; i < p.tri_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < dest_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(cnt)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < kRouteWarps * p.lane_stride; i += kRouteThreads) wm[i] = make_uint2(0, 0);
+    if (tid < 2) cta_totals[tid] = 0;
+    const TableView tv = table_view(p.lv, tab);
+    asm volatile("cp.async.wait_all;" ::: "memory");      // the tables have arrived behind the clearing
     __syncthreads();
 
+    // ---- phase 1: statistics, Algorithm 1, destination counts ---------------------------------
     uint32_t cost_sum = 0, naive_sum = 0;
     for (int round = 0; round < n_rounds; ++round) {
-        const int first_chunk = chunk_lo + round * kRouteChunksPerRound;
-        const int chunks_this_round = min(kRouteChunksPerRound, chunk_hi - first_chunk);
-        const int64_t t = static_cast<int64_t>(first_chunk) * kRouteChunkTokens + threadIdx.x;
-        if (static_cast<int>(threadIdx.x) < chunks_this_round * kRouteChunkTokens && t < T) {
+        const int64_t t = t_lo + static_cast<int64_t>(round) * kRouteThreads + tid;
+        const bool has_token = t < t_hi;
+        uint32_t bad = 0;
+        if (has_token) {
             if (round > 0) {
-                load_token_ids<KT>(topk_ids, t, K, id);
-                if (src_rank) s_t = __ldg(src_rank + t);
+                load_token_ids<KT>(p.topk_ids, t, K, id);
+                if (p.src_rank) s_t = __ldg(p.src_rank + t);
             }
-            const uint32_t bad_ids = check_token_ids<KT>(id, K, lv.E);
-            uint32_t bad = bad_ids;
-            if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
-            if (bad) flag_error(err_word, bad);
+            int32_t sorted[KMAX];
+            sort_token_ids<KT>(id, K, sorted);
+            const uint32_t bad_ids = check_sorted_ids<KT>(sorted, K, E);
+            bad = bad_ids;
+            if (s_t < 0 || s_t >= p.lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
+            if (bad) flag_error(p.err_word, bad);
             // the statistics only need valid ids, as in the stand-alone statistics call
-            if (!bad_ids) add_token_to_triangle<KT, kPacked>(tri, id, K);
+            if (!bad_ids) add_sorted_token_to_triangle<KT, kPacked>(tri, sorted, K);
+        }
+        if (has_token) {
             uint32_t cost = 0, naive_cost = 0;
             if (bad) {
 #pragma unroll
@@ -117,278 +300,347 @@ route_fused_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const in
             } else {
                 assign_token<KT, kAssignSlot>(tv, id, K, s_t, static_cast<uint32_t>(t), seed_lo, seed_hi, out, cost,
                                               naive_cost);
-                uint32_t* mine = chist + (threadIdx.x / kRouteChunkTokens) * D;
+                if (single) {
 #pragma unroll
-                for (int a = 0; a < KMAX; ++a)
-                    if (a < K) atomicAdd(&mine[out[a]], 1u);
+                    for (int a = 0; a < KMAX; ++a)
+                        if (a < K) atomicOr(&my_wm[out[a]].x, 1u << lane);
+                } else {
+#pragma unroll
+                    for (int a = 0; a < KMAX; ++a)
+                        if (a < K) atomicAdd(&cnt[out[a]], 1u);
+                }
             }
-            store_token_slots<KT>(assigned_slot + t * K, out, K);
-            if (remote_nodes) remote_nodes[t] = static_cast<uint8_t>(cost);
+            store_token_slots<KT>(p.assigned_slot + t * K, out, K);
+            if (p.remote_nodes) p.remote_nodes[t] = static_cast<uint8_t>(cost);
             cost_sum += cost;
             naive_sum += naive_cost;
         }
-        __syncthreads();
-        // hand this round's chunk histograms to the scan (every chunk row is written, zeros included)
-        for (int i = threadIdx.x; i < chunks_this_round * D; i += blockDim.x) {
-            const int g = i / D, d = i - g * D;
-            chunk_ws[static_cast<size_t>(d) * n_chunks + first_chunk + g] = chist[i];
-            chist[i] = 0;
-        }
-        __syncthreads();
     }
-
-    if (totals) {
+    if (p.totals) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             cost_sum += __shfl_xor_sync(0xFFFFFFFFu, cost_sum, off);
             naive_sum += __shfl_xor_sync(0xFFFFFFFFu, naive_sum, off);
         }
-        if ((threadIdx.x & 31) == 0) {
+        if (lane == 0) {
             if (cost_sum) atomicAdd(&cta_totals[0], static_cast<unsigned long long>(cost_sum));
             if (naive_sum) atomicAdd(&cta_totals[1], static_cast<unsigned long long>(naive_sum));
         }
     }
-    cluster.sync();            // every triangle of the cluster is complete (also orders cta_totals)
-    wait_for_prior_kernel();   // coact / load / totals may still be being cleared by the kernel before this one
-    merge_triangle_over_cluster<kPacked>(tri, lv.E, coact, load);
-    if (totals && threadIdx.x < 2 && cta_totals[threadIdx.x])
-        atomicAdd(&totals[threadIdx.x], cta_totals[threadIdx.x]);
-    cluster.sync();            // no CTA may exit while a peer still reads its triangle
-}
-
-// ---- batches of at most 16 chunks: everything in ONE kernel, one cluster --------------------------
-// Every CTA owns one chunk of 256 tokens.  The per-chunk destination histograms are exchanged through
-// distributed shared memory instead of a workspace in global memory, so the scan across chunks and
-// the stable rank run in the same kernel (two cluster barriers, no further launches), and with a
-// single cluster the statistics can be stored instead of added, so nothing is cleared beforehand.
-constexpr int kSmallMaxChunks = 16;
-constexpr int kSmallMaxDests = 992;        // one destination per thread in the scan over d; the last warp sums the totals
-constexpr int kSmallWarps = kRouteThreads / 32;
-
-struct SmallSmem {
-    size_t tri_words, tab_words, dest_words, slot_words, rank_words;
-    size_t bytes() const { return (tri_words + tab_words + 2 * dest_words + slot_words + rank_words) * sizeof(uint32_t); }
-};
-
-static SmallSmem small_smem(const LayoutView& lv, int K)
-{
-    SmallSmem r;
-    // 16-bit counters (a cluster sees at most 4096 tokens): the merge is bound by the bytes that cross
-    // distributed shared memory, and these are half as many
-    r.tri_words = ((tri_entries(lv.E) + 1) / 2 + 3) / 4 * 4;
-    r.tab_words = static_cast<size_t>(lv.words + 3) / 4 * 4;
-    r.dest_words = static_cast<size_t>(lv.D + 3) / 4 * 4;                   // chist, and the totals per destination
-    r.slot_words = static_cast<size_t>(kRouteChunkTokens) * K;              // this chunk's slots, in pair order
-    r.rank_words = static_cast<size_t>(1 + kSmallWarps) * r.dest_words;     // base[d] and the per-warp counters
-    return r;
-}
-
-template <int KT, bool kAccumulate>
-__global__ void __launch_bounds__(kRouteThreads)
-route_small_kernel(LayoutView lv, const int32_t* __restrict__ topk_ids, const int32_t* __restrict__ src_rank,
-                   int32_t src_uniform, int64_t T, uint32_t seed_lo, uint32_t seed_hi, uint32_t* __restrict__ coact,
-                   uint32_t* __restrict__ load, int32_t* __restrict__ assigned_slot, uint8_t* __restrict__ remote_nodes,
-                   unsigned long long* __restrict__ totals, uint32_t* __restrict__ dest_counts,
-                   uint32_t* __restrict__ dest_offsets, int32_t* __restrict__ row_of_pair,
-                   int32_t* __restrict__ pair_of_row, int tri_words, int tab_words, int dest_words, int key_bits,
-                   const unsigned long long* __restrict__ seed_on_device, uint32_t* __restrict__ err_word)
-{
-    if (seed_on_device) {                               // the seed of this run, not of the capture
-        const unsigned long long sd = __ldg(seed_on_device);
-        seed_lo = static_cast<uint32_t>(sd);
-        seed_hi = static_cast<uint32_t>(sd >> 32);
-    }
-    extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t* tri = smem;
-    uint32_t* tab = tri + tri_words;
-    uint32_t* chist = tab + tab_words;             // [D] this chunk's pairs per destination
-    uint32_t* tot = chist + dest_words;            // [D] all chunks' pairs per destination
-    int32_t* slots = reinterpret_cast<int32_t*>(tot + dest_words);      // [256 * K]
-    uint32_t* base = reinterpret_cast<uint32_t*>(slots) + kRouteChunkTokens * KT;   // [D]
-    uint32_t* wcnt = base + dest_words;            // [kSmallWarps][dest_words]
-    __shared__ unsigned long long cta_totals[2];
-    __shared__ uint32_t warp_sums[kSmallWarps];
-    constexpr int K = KT;
-    const int D = lv.D;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int chunk = static_cast<int>(cluster.block_rank());
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    // threads 0..255 run Algorithm 1 for the chunk's tokens, threads 256..511 add the same tokens to
-    // the triangle: two short instruction chains side by side instead of one long one
-    const int64_t t = static_cast<int64_t>(chunk) * kRouteChunkTokens + (tid & (kRouteChunkTokens - 1));
-    const bool has_token = tid < kRouteChunkTokens && t < T;
-    const bool counts_token = tid >= kRouteChunkTokens && tid < 2 * kRouteChunkTokens && t < T;
-    int32_t id[K], out[K];
-    int32_t s_t = src_uniform;
-    if (has_token || counts_token) {
-        load_token_ids<KT>(topk_ids, t, K, id);
-        if (has_token && src_rank) s_t = __ldg(src_rank + t);
-    }
-    for (int i = tid; i < tri_words / 4; i += blockDim.x) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < dest_words; i += blockDim.x) chist[i] = 0;
-    for (int i = tid; i < kSmallWarps * dest_words; i += blockDim.x) wcnt[i] = 0;
-    if (tid < 2) cta_totals[tid] = 0;
-    const TableView tv = stage_tables(lv, tab);
     __syncthreads();
 
-    uint32_t cost = 0, naive_cost = 0;
-    if (has_token) {
-        const uint32_t bad_ids = check_token_ids<KT>(id, K, lv.E);
-        uint32_t bad = bad_ids;
-        if (s_t < 0 || s_t >= lv.G) bad |= COBALT_DEVERR_BAD_SRC_RANK;
-        if (bad) flag_error(err_word, bad);
-        if (bad) {
+    // Per destination, the pairs of the lower warps of a round (and the round's pairs in all): one warp
+    // per destination, lane w holding the pairs of warp w, an exclusive scan across the lanes.  The odd
+    // stride of the table keeps the lanes on different banks.  Needs the lane masks of the round.
+    auto count_round = [&]() {
+        // two destinations share a scan (16-bit halves: a warp sends at most 32 pairs to a destination, a
+        // round at most 1024), and two such scans are in flight per iteration
+        for (int d0 = warp; d0 < D; d0 += 4 * kRouteWarps) {
+            uint32_t c[2], incl[2];
 #pragma unroll
-            for (int a = 0; a < K; ++a) out[a] = -1;
+            for (int h = 0; h < 2; ++h) {
+                const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
+                const uint32_t ca = (da < D) ? __popc(wm[lane * p.lane_stride + da].x) : 0u;
+                const uint32_t cb = (db < D) ? __popc(wm[lane * p.lane_stride + db].x) : 0u;
+                c[h] = ca | (cb << 16);
+                incl[h] = c[h];
+            }
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl[h], off);
+                    if (lane >= off) incl[h] += up;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
+                const uint32_t before = incl[h] - c[h];
+                if (da < D) {
+                    wm[lane * p.lane_stride + da].y = before & 0xFFFFu;
+                    if (lane == 31) cnt[da] = incl[h] & 0xFFFFu;
+                }
+                if (db < D) {
+                    wm[lane * p.lane_stride + db].y = before >> 16;
+                    if (lane == 31) cnt[db] = incl[h] >> 16;
+                }
+            }
+        }
+    };
+    // The rank of each of the thread's pairs inside its destination among the pairs of the round (packed
+    // with the destination into out[], -1 for a pair without one), and the pair's entry in the staged
+    // inverse map.  Needs count_round and the scan of its counts over d (excl).
+    auto rank_round = [&](bool has_token) {
+        if (!has_token) return;
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a) {
+            if (a < K && out[a] >= 0) {
+                const uint32_t d = static_cast<uint32_t>(out[a]);
+                const uint2 v = my_wm[d];
+                const uint32_t r = v.y + __popc(v.x & lower_lanes);
+                if (p.pair_of_row) stage[excl[d] + r] = d | (static_cast<uint32_t>(tid * K + a) << kDestBits);
+                out[a] = static_cast<int32_t>(d | (r << kDestBits));
+            }
+        }
+    };
+    // Rows of the thread's pairs (the rank of rank_round on top of the first row of the round's pairs
+    // inside the destination), and the round's part of the inverse map in row order: consecutive
+    // threads write consecutive rows of a destination.
+    auto write_round = [&](bool has_token, int64_t t_round, uint32_t round_pairs) {
+        if (has_token) {
+            int32_t row[KMAX];
+#pragma unroll
+            for (int a = 0; a < KMAX; ++a) {
+                row[a] = -1;
+                if (a < K && out[a] >= 0)
+                    row[a] = static_cast<int32_t>(base[out[a] & ((1 << kDestBits) - 1)] + (static_cast<uint32_t>(out[a]) >> kDestBits));
+            }
+            store_token_slots<KT>(p.row_of_pair + (t_round + tid) * K, row, K);
+        }
+        if (p.pair_of_row) {
+            for (uint32_t j = tid; j < round_pairs; j += kRouteThreads) {
+                const uint32_t v = stage[j];
+                const uint32_t d = v & ((1u << kDestBits) - 1u);
+                p.pair_of_row[base[d] + (j - excl[d])] = static_cast<int32_t>(t_round * K + (v >> kDestBits));
+            }
+        }
+    };
+
+    if (single) count_round();               // cnt[d] from the lane masks
+    __syncthreads();
+
+    // ---- publish this CTA's partial results ------------------------------------------------------
+    {
+        uint4* dst = reinterpret_cast<uint4*>(p.ws_tri + static_cast<size_t>(cta) * p.tri_words);
+        for (int v = tid; v < p.tri_words / 4; v += kRouteThreads) dst[v] = reinterpret_cast<const uint4*>(tri)[v];
+        uint32_t* dst_cnt = reinterpret_cast<uint32_t*>(p.ws_cnt + static_cast<size_t>(cta) * dest_words);
+        for (int i = tid; i < dest_words / 2; i += kRouteThreads) dst_cnt[i] = cnt[2 * i] | (cnt[2 * i + 1] << 16);
+        if (p.totals && tid < 2) p.ws_tot[2 * cta + tid] = cta_totals[tid];
+    }
+    // while those stores drain: what the ranks need from this CTA alone
+    uint32_t round_pairs = 0;
+    if (single) {
+        const uint32_t lower_dests = block_exclusive_scan((tid < D) ? cnt[tid] : 0u, warp_sums, &round_pairs);
+        if (tid < D) excl[tid] = lower_dests;
+        __syncthreads();
+        rank_round(t_lo + tid < t_hi);
+    }
+    if (!grid_barrier(p.barrier, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word)) return;
+
+    // ---- phase 2a and 2b side by side: both wait on loads of what the other CTAs published, so the
+    // upper half of the CTA's warps sums this CTA's slice of the triangle over all partials (2a) while
+    // the lower half sums the destination counts of all CTAs (2b) ---------------------------------
+    constexpr int kHalf = kRouteThreads / 2;
+    constexpr int kPerWord = kPacked ? 2 : 1;
+    const int n_tri = static_cast<int>(tri_entries(E));
+    const int n_vec = p.tri_words / 4;                                // 16-byte vectors of a triangle
+    const int slice = (n_vec + n_ctas - 1) / n_ctas;                  // vectors of a CTA's slice
+    const int v0 = min(n_vec, cta * slice), v1 = min(n_vec, v0 + slice);
+    const int n_mine = v1 - v0;
+    const int n_acc = 4 * n_mine * kPerWord;                          // sums of the slice, 32 bits each
+    // 2b: the CTAs' counts are split over `parts` groups of threads; a thread sums eight consecutive
+    // destinations of its share of the CTAs and leaves its sums (all CTAs, lower CTAs) where the
+    // triangle was, behind the sums of the slice; one thread per destination adds them up.
+    const int octs = dest_words / 8;
+    int parts = max(1, kHalf / octs);
+    parts = min(parts, n_ctas);
+    if (parts > 1) parts = max(1, min(parts, (p.tri_words - n_acc) / (2 * dest_words)));
+    uint32_t* acc = tri;
+    uint32_t* part_all = tri + (n_acc + 3) / 4 * 4;                   // [parts][dest_words]
+    uint32_t* part_lower = part_all + parts * dest_words;             // [parts][dest_words]
+    if ((n_acc + 3) / 4 * 4 + 2 * parts * dest_words > p.tri_words) {   // a tiny triangle: one group, sums straight into cnt / base
+        parts = 1;
+        part_all = cnt;
+        part_lower = base;
+    }
+    for (int i = tid; i < n_acc; i += kRouteThreads) acc[i] = 0;
+    __syncthreads();
+    if (tid >= kHalf) {
+        // 2a: `groups` threads share a vector of the slice, each summing every groups-th partial in
+        // registers (loads in flight together, lanes along consecutive vectors), then shared-memory adds
+        constexpr int kBatch = 5;
+        const int ht = tid - kHalf;
+        if (n_mine > 0) {
+            const int groups = max(1, kHalf / n_mine);
+            for (int j = ht; j < groups * n_mine; j += kHalf) {          // one pass unless n_mine > 512
+                const int g = j / n_mine, v = j - g * n_mine;
+                const uint4* src = reinterpret_cast<const uint4*>(p.ws_tri) + v0 + v;
+                uint32_t sum[4 * kPerWord];
+#pragma unroll
+                for (int i = 0; i < 4 * kPerWord; ++i) sum[i] = 0;
+                for (int c = g; c < n_ctas; c += groups * kBatch) {
+                    uint4 q[kBatch];
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u) {
+                        const int cc = c + u * groups;
+                        q[u] = (cc < n_ctas) ? __ldcg(src + static_cast<size_t>(cc) * n_vec) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u) {
+                        const uint32_t word[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            if (kPacked) {
+                                sum[2 * i] += word[i] & 0xFFFFu;
+                                sum[2 * i + 1] += word[i] >> 16;
+                            } else {
+                                sum[i] += word[i];
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4 * kPerWord; ++i)
+                    if (sum[i]) atomicAdd(&acc[4 * kPerWord * v + i], sum[i]);
+            }
+        }
+        if (p.totals && cta == 0 && ht < 2) {
+            unsigned long long sum = 0;
+            for (int c = 0; c < n_ctas; ++c) sum += __ldcg(p.ws_tot + 2 * c + ht);
+            p.totals[ht] = sum;
+        }
+    } else {
+        constexpr int kBatch = 6;
+        const int part = tid / octs, oct = tid - part * octs;
+        if (part < parts) {
+            const uint4* src = reinterpret_cast<const uint4*>(p.ws_cnt) + oct;
+            uint32_t all[8], lower[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) all[i] = lower[i] = 0;
+            for (int c = part; c < n_ctas; c += parts * kBatch) {
+                uint4 q[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int cc = c + u * parts;
+                    q[u] = (cc < n_ctas) ? __ldcg(src + static_cast<size_t>(cc) * octs) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const bool below = c + u * parts < cta;
+                    const uint32_t word[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t lo = word[i] & 0xFFFFu, hi = word[i] >> 16;
+                        all[2 * i] += lo;
+                        all[2 * i + 1] += hi;
+                        if (below) {
+                            lower[2 * i] += lo;
+                            lower[2 * i + 1] += hi;
+                        }
+                    }
+                }
+            }
+            uint4* dst_all = reinterpret_cast<uint4*>(part_all + part * dest_words + 8 * oct);
+            uint4* dst_lower = reinterpret_cast<uint4*>(part_lower + part * dest_words + 8 * oct);
+            dst_all[0] = make_uint4(all[0], all[1], all[2], all[3]);
+            dst_all[1] = make_uint4(all[4], all[5], all[6], all[7]);
+            dst_lower[0] = make_uint4(lower[0], lower[1], lower[2], lower[3]);
+            dst_lower[1] = make_uint4(lower[4], lower[5], lower[6], lower[7]);
+        }
+    }
+    __syncthreads();
+    // 2a: the sums of the slice go out to coact / load (plain stores unless accumulating)
+    for (int i = tid; i < n_acc; i += kRouteThreads) {
+        const int flat = 4 * v0 * kPerWord + i;
+        if (flat >= n_tri) continue;
+        const int hi = tri_row(flat), lo = flat - hi * (hi + 1) / 2;
+        const uint32_t v = acc[i];
+        if (p.accumulate) {
+            if (v) {
+                atomicAdd(&p.coact[static_cast<size_t>(hi) * E + lo], v);
+                if (lo != hi) atomicAdd(&p.coact[static_cast<size_t>(lo) * E + hi], v);
+                else atomicAdd(&p.load[hi], v);
+            }
         } else {
-            assign_token<KT, kAssignSlot>(tv, id, K, s_t, static_cast<uint32_t>(t), seed_lo, seed_hi, out, cost, naive_cost);
-#pragma unroll
-            for (int a = 0; a < K; ++a) atomicAdd(&chist[out[a]], 1u);
-        }
-        store_token_slots<KT>(assigned_slot + t * K, out, K);
-#pragma unroll
-        for (int a = 0; a < K; ++a) slots[tid * K + a] = out[a];
-        if (remote_nodes) remote_nodes[t] = static_cast<uint8_t>(cost);
-    } else if (counts_token) {
-        // the statistics only need valid ids, as in the stand-alone statistics call
-        if (!check_token_ids<KT>(id, K, lv.E)) add_token_to_triangle<KT, true>(tri, id, K);
-    }
-    if (totals && tid < kRouteChunkTokens) {      // the first eight warps hold the tokens
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            cost += __shfl_xor_sync(0xFFFFFFFFu, cost, off);
-            naive_cost += __shfl_xor_sync(0xFFFFFFFFu, naive_cost, off);
-        }
-        if (lane == 0) {
-            if (cost) atomicAdd(&cta_totals[0], static_cast<unsigned long long>(cost));
-            if (naive_cost) atomicAdd(&cta_totals[1], static_cast<unsigned long long>(naive_cost));
+            p.coact[static_cast<size_t>(hi) * E + lo] = v;
+            if (lo != hi) p.coact[static_cast<size_t>(lo) * E + hi] = v;
+            else p.load[hi] = v;
         }
     }
-    cluster.sync();            // every triangle, chunk histogram and cost sum of the cluster is complete
-
-    merge_triangle_over_cluster<true, !kAccumulate>(tri, lv.E, coact, load);
-    // scan across chunks, one destination per thread: pairs of lower chunks, and of all chunks
-    // (the cluster always has kSmallMaxChunks CTAs: all remote loads are issued before the first is used)
-    uint32_t mine_total = 0;
-    if (tid < D) {
-        uint32_t c[kSmallMaxChunks];
-#pragma unroll
-        for (int r = 0; r < kSmallMaxChunks; ++r) c[r] = cluster.map_shared_rank(chist, r)[tid];
-        uint32_t before = 0;
-#pragma unroll
-        for (int r = 0; r < kSmallMaxChunks; ++r) {
-            if (r < chunk) before += c[r];
-            mine_total += c[r];
+    {
+        // 2b: totals over all CTAs, their exclusive scan over d (the offsets), first row of this CTA
+        uint32_t mine = 0, lower = 0;
+        if (tid < D) {
+            for (int g = 0; g < parts; ++g) {
+                mine += part_all[g * dest_words + tid];
+                lower += part_lower[g * dest_words + tid];
+            }
         }
-        base[tid] = before;
-        tot[tid] = mine_total;
-    } else if (totals && chunk == 0 && tid >= kSmallMaxDests && tid < kSmallMaxDests + 2) {
-        const int which = tid - kSmallMaxDests;
-        unsigned long long part[kSmallMaxChunks];
-#pragma unroll
-        for (int r = 0; r < kSmallMaxChunks; ++r) part[r] = cluster.map_shared_rank(cta_totals, r)[which];
-        unsigned long long sum = 0;
-#pragma unroll
-        for (int r = 0; r < kSmallMaxChunks; ++r) sum += part[r];
-        totals[which] = sum;
-    }
-    cluster.sync();            // no CTA may exit, nor may shared memory change, while a peer still reads it
-    // exclusive scan of the totals over d (one destination per thread, D <= blockDim.x)
-    uint32_t incl = mine_total;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= off) incl += up;
-    }
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    uint32_t offset = incl - mine_total;
-    for (int w = 0; w < warp; ++w) offset += warp_sums[w];
-    if (tid < D) {
-        base[tid] += offset;                    // first row of this chunk inside destination d
-        if (chunk == 0) {
-            dest_counts[tid] = mine_total;
-            dest_offsets[tid] = offset;
-            if (tid == D - 1) dest_offsets[D] = offset + mine_total;
+        uint32_t total = 0;
+        const uint32_t before = block_exclusive_scan(mine, warp_sums, &total);
+        if (tid < D) {
+            if (cta == 0) {
+                p.dest_counts[tid] = mine;
+                p.dest_offsets[tid] = before;
+            }
+            base[tid] = before + lower;
         }
+        if (cta == 0 && tid == 0) p.dest_offsets[D] = total;
     }
     __syncthreads();
 
-    // stable rank of the chunk's pairs: each warp owns 8 K consecutive pairs (at most four 32-pair steps)
-    const int n_tok = static_cast<int>(min(static_cast<int64_t>(kRouteChunkTokens),
-                                           max(static_cast<int64_t>(0), T - static_cast<int64_t>(chunk) * kRouteChunkTokens)));
-    const int n_pairs = n_tok * K;
-    constexpr int kSub = kRouteChunkTokens * K / kSmallWarps;
-    constexpr int kSteps = (kSub + 31) / 32;
-    const int w0 = warp * kSub, w1 = min(n_pairs, w0 + kSub);
-    const int64_t p0 = static_cast<int64_t>(chunk) * kRouteChunkTokens * K;
-    uint32_t* mine = wcnt + warp * dest_words;
-    int32_t dreg[kSteps];
-    uint32_t preg[kSteps];
-#pragma unroll
-    for (int st = 0; st < kSteps; ++st) {
-        const int p = w0 + st * 32 + lane;
-        const int32_t d = (st * 32 + lane < kSub && p < w1) ? slots[p] : -1;
-        const uint32_t key = static_cast<uint32_t>(d < 0 ? D : d);
-        uint32_t peers = 0xFFFFFFFFu;
-        for (int b = 0; b < key_bits; ++b) {
-            const uint32_t bit = (key >> b) & 1u;
-            const uint32_t vote = __ballot_sync(0xFFFFFFFFu, bit);
-            peers &= bit ? vote : ~vote;
-        }
-        dreg[st] = d;
-        preg[st] = peers;
-        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);   // highest lane of the group
-        __syncwarp();
+    // ---- phase 2c: rows of this CTA's pairs ------------------------------------------------------
+    if (single) {
+        write_round(t_lo + tid < t_hi, t_lo, round_pairs);
+        return;
     }
-    __syncthreads();
-    if (tid < D) {                              // per destination: per-warp counts -> starting rows, in warp order
-        uint32_t run = base[tid];
-#pragma unroll 8
-        for (int w = 0; w < kSmallWarps; ++w) {
-            const uint32_t c = wcnt[w * dest_words + tid];
-            wcnt[w * dest_words + tid] = run;
-            run += c;
-        }
-    }
-    __syncthreads();
+    for (int round = 0; round < n_rounds; ++round) {
+        const int64_t t_round = t_lo + static_cast<int64_t>(round) * kRouteThreads;
+        const int64_t t = t_round + tid;
+        const bool has_token = t < t_hi;
+        if (has_token) {
+            // the slots come back from memory (this thread wrote them in phase 1)
+            const int32_t* slots = p.assigned_slot + t * K;
+            if (KT > 0 && KT % 4 == 0) {
 #pragma unroll
-    for (int st = 0; st < kSteps; ++st) {
-        const int p = w0 + st * 32 + lane;
-        const bool in_range = st * 32 + lane < kSub && p < w1;
-        const int32_t d = dreg[st];
-        const uint32_t peers = preg[st];
-        if (d >= 0) {
-            const uint32_t row = mine[d] + __popc(peers & ((1u << lane) - 1u));
-            row_of_pair[p0 + p] = static_cast<int32_t>(row);
-            if (pair_of_row) pair_of_row[row] = static_cast<int32_t>(p0 + p);
-        } else if (in_range) {
-            row_of_pair[p0 + p] = -1;
+                for (int a = 0; a < KT / 4; ++a) {
+                    const int4 v = reinterpret_cast<const int4*>(slots)[a];
+                    out[4 * a] = v.x; out[4 * a + 1] = v.y; out[4 * a + 2] = v.z; out[4 * a + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int a = 0; a < KMAX; ++a)
+                    if (a < K) out[a] = slots[a];
+            }
+#pragma unroll
+            for (int a = 0; a < KMAX; ++a)
+                if (a < K && out[a] >= 0) atomicOr(&my_wm[out[a]].x, 1u << lane);
         }
-        __syncwarp();
-        if (d >= 0 && (peers >> lane) == 1u) mine[d] += __popc(peers);
-        __syncwarp();
+        __syncthreads();
+        count_round();
+        __syncthreads();
+        const uint32_t round_total = (tid < D) ? cnt[tid] : 0u;
+        const uint32_t lower_dests = block_exclusive_scan(round_total, warp_sums, &round_pairs);
+        if (tid < D) excl[tid] = lower_dests;
+        // the masks are cleared through the still unpacked slots before rank_round packs them
+        __syncthreads();
+        uint32_t touched[KMAX];
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a) touched[a] = (has_token && a < K && out[a] >= 0) ? static_cast<uint32_t>(out[a]) : 0xFFFFFFFFu;
+        rank_round(has_token);
+        __syncthreads();
+        write_round(has_token, t_round, round_pairs);
+        __syncthreads();
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a)
+            if (touched[a] != 0xFFFFFFFFu) my_wm[touched[a]].x = 0;
+        if (tid < D) base[tid] += round_total;
+        __syncthreads();
     }
 }
 
-struct RouteLaunch {
-    int cluster;
-    int ctas;
-};
-
+// The grid the device can hold for this kernel and shared-memory size (one CTA per SM in practice),
+// asked once per (device, kernel, bytes); 0 if the device cannot launch it cooperatively.
 template <int KT, bool kPacked>
-static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n_sm, RouteLaunch* out)
+static int max_resident_ctas(size_t smem, int* out)
 {
     auto kernel = route_fused_kernel<KT, kPacked>;
     static std::mutex cache_lock;
-    static std::map<std::tuple<int, int, int, int64_t>, RouteLaunch> cache;
+    static std::map<std::pair<int, size_t>, int> cache;
     int dev = 0;
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
-    int64_t want = (T + kRouteChunkTokens - 1) / kRouteChunkTokens;   // one chunk per CTA while CTAs last
-    if (want < 16) want = 16;      // a full cluster at least: CTAs without tokens still share the merge
-    if (want > n_sm) want = n_sm;
-    const auto key = std::make_tuple(dev, static_cast<int>(smem), lv.D, want);
+    const auto key = std::make_pair(dev, smem);
     {
         std::lock_guard<std::mutex> guard(cache_lock);
         auto it = cache.find(key);
@@ -397,44 +649,17 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
             return COBALT_OK;
         }
     }
-    int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), smem, true);
+    int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), smem, false);
     if (rc_attr != COBALT_OK) return rc_attr;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    cfg.blockDim = dim3(kRouteThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    int cand_cs[5], cand_cta[5], n_cand = 0, most = 0;
-    for (int cs = 16; cs >= 1; cs >>= 1) {
-        if (cs > want) continue;
-        attr[0].val.clusterDim.x = cs;
-        cfg.gridDim = dim3(cs);
-        int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess) {
-            (void)cudaGetLastError();
-            continue;
-        }
-        int n_cta = static_cast<int>(want) / cs * cs;
-        if (n_cta > max_clusters * cs) n_cta = max_clusters * cs;
-        if (n_cta < cs) continue;
-        cand_cs[n_cand] = cs;
-        cand_cta[n_cand] = n_cta;
-        ++n_cand;
-        if (n_cta > most) most = n_cta;
-    }
-    RouteLaunch best = {0, 0};
-    for (int i = 0; i < n_cand; ++i) {
-        if (cand_cta[i] * 4 >= most * 3) {
-            best.cluster = cand_cs[i];
-            best.ctas = cand_cta[i];
-            break;
-        }
-    }
-    if (best.cluster == 0) return COBALT_ERR_UNSUPPORTED;
+    int best = 0, cooperative = 0, n_sm = 0, per_sm = 0;
+    COBALT_CUDA_TRY(cudaDeviceGetAttribute(&cooperative, cudaDevAttrCooperativeLaunch, dev));
+    rc_attr = sm_count(&n_sm);
+    if (rc_attr != COBALT_OK) return rc_attr;
+    if (cooperative &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kRouteThreads, smem) == cudaSuccess && per_sm >= 1)
+        best = std::min(n_sm, kRouteMaxCtas);          // one CTA per SM: more would only share the SM's issue slots
+    else
+        (void)cudaGetLastError();
     {
         std::lock_guard<std::mutex> guard(cache_lock);
         cache[key] = best;
@@ -444,141 +669,86 @@ static int pick_route_launch(const LayoutView& lv, int64_t T, size_t smem, int n
 }
 
 struct RouteArgs {
-    const LayoutView* lv;
-    const int32_t* ids;
-    const int32_t* src;
-    int32_t src_uniform;
-    int64_t T;
-    int32_t K;
-    uint64_t seed;
-    const unsigned long long* seed_on_device;
-    uint32_t* coact;
-    uint32_t* load;
-    int32_t* assigned_slot;
-    uint8_t* remote_nodes;
-    uint64_t* totals;
-    uint32_t* chunk_ws;
-    int n_chunks;
-    uint32_t* err_word;
-    ZeroList zero;
-    int n_sm;
+    RouteParams p;
+    int K;
+    void* workspace;
     cudaStream_t stream;
 };
 
-// *launched stays false (and nothing has been enqueued) when 16-bit counters would be needed but one
-// cluster would see more than 65535 tokens: the caller then takes the separate calls.
-template <int KT, bool kPacked>
-static int launch_route(const RouteArgs& a, bool* launched)
+// Epochs of the grid barrier: distinct for consecutive launches and never 0 (a cleared word).
+static uint32_t next_epoch()
 {
-    *launched = false;
-    const LayoutView& lv = *a.lv;
-    const RouteSmem sm = route_smem(lv, kPacked);
-    RouteLaunch how;
-    int rc = pick_route_launch<KT, kPacked>(lv, a.T, sm.bytes(), a.n_sm, &how);
-    if (rc != COBALT_OK) return rc;
-    const int chunks_per_cta = (a.n_chunks + how.ctas - 1) / how.ctas;
-    if (kPacked && static_cast<int64_t>(chunks_per_cta) * kRouteChunkTokens * how.cluster > 65535) return COBALT_OK;
-    bool after_zeroing = false;
-    rc = launch_zero_list(a.zero, a.stream, &after_zeroing);
-    if (rc != COBALT_OK) return rc;
-    auto kernel = route_fused_kernel<KT, kPacked>;
-    rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), sm.bytes(), true);
-    if (rc != COBALT_OK) return rc;
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[2];
-    cfg.blockDim = dim3(kRouteThreads);
-    cfg.gridDim = dim3(static_cast<unsigned>(how.ctas));
-    cfg.dynamicSmemBytes = sm.bytes();
-    cfg.stream = a.stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = how.cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    set_programmatic_launch(&attr[1], after_zeroing);
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T, a.K,
-                                       static_cast<uint32_t>(a.seed & 0xFFFFFFFFu),
-                                       static_cast<uint32_t>(a.seed >> 32), a.coact, a.load, a.assigned_slot,
-                                       a.remote_nodes, reinterpret_cast<unsigned long long*>(a.totals), a.chunk_ws,
-                                       a.n_chunks, static_cast<int>(sm.tri_words), static_cast<int>(sm.tab_words),
-                                       chunks_per_cta, a.seed_on_device, a.err_word));
-    *launched = true;
-    return COBALT_OK;
+    static std::atomic<uint32_t> counter{0};
+    uint32_t x = counter.fetch_add(1) + 1u;
+    x *= 0x9E3779B9u;                 // odd multiplier: a bijection, so consecutive launches differ
+    return x ? x : 0x5bd1e995u;
 }
 
-struct SmallArgs {
-    uint32_t* dest_counts;
-    uint32_t* dest_offsets;
-    int32_t* row_of_pair;
-    int32_t* pair_of_row;
-    bool accumulate;
-};
-
-// *launched stays false (nothing enqueued) when the batch, the layout or the device does not qualify.
-template <int KT>
-static int launch_route_small(const RouteArgs& a, const SmallArgs& b, bool* launched)
+// *launched stays false (and nothing has been enqueued) when the kernel does not fit this layout,
+// batch or device: the caller then takes the separate calls.
+template <int KT, bool kPacked>
+static int launch_route(RouteArgs a, bool* launched)
 {
     *launched = false;
-    const LayoutView& lv = *a.lv;
-    if (a.T < 1 || a.n_chunks > kSmallMaxChunks || lv.D > kSmallMaxDests) return COBALT_OK;
-    const SmallSmem sm = small_smem(lv, KT);
+    RouteParams& p = a.p;
+    if (p.lv.D > kRouteMaxDests) return COBALT_OK;
+    const RouteSmem sm = route_smem(p.lv, a.K, kPacked);
     if (sm.bytes() > kRouteMaxSmem) return COBALT_OK;
-    // always a full cluster: CTAs without tokens still take their share of the clearing and the merge
-    const int cluster = kSmallMaxChunks;
-    using Kernel = void (*)(LayoutView, const int32_t*, const int32_t*, int32_t, int64_t, uint32_t, uint32_t, uint32_t*,
-                            uint32_t*, int32_t*, uint8_t*, unsigned long long*, uint32_t*, uint32_t*, int32_t*, int32_t*,
-                            int, int, int, int, const unsigned long long*, uint32_t*);
-    Kernel kernel = b.accumulate ? route_small_kernel<KT, true> : route_small_kernel<KT, false>;
-    int rc = ensure_kernel_attributes(reinterpret_cast<const void*>(kernel), sm.bytes(), true);
+    int max_ctas = 0;
+    int rc = max_resident_ctas<KT, kPacked>(sm.bytes(), &max_ctas);
     if (rc != COBALT_OK) return rc;
+    if (max_ctas < 1) return COBALT_OK;
+    // 256 tokens per CTA until the resident CTAs run out
+    int64_t want = (p.T + 255) / 256;
+    if (want > max_ctas) want = max_ctas;
+    // with 16-bit counters the sums of a slice (32-bit) are kept where the triangle was: at least two slices
+    const int min_ctas = kPacked ? 2 : 1;
+    if (want < min_ctas) want = min_ctas;
+    if (want > max_ctas) return COBALT_OK;
+    const int n_ctas = static_cast<int>(want);
+    const int64_t per = static_cast<int64_t>(round_up(static_cast<size_t>((p.T + n_ctas - 1) / n_ctas), 32));
+    if (per > 0x7FFFFFFFll) return COBALT_OK;
+    if (per > 65535) return COBALT_OK;     // the CTA's 16-bit counters (destination counts, packed triangle) could overflow
+    p.tokens_per_cta = static_cast<int>(per);
+    p.tri_words = static_cast<int>(sm.tri_words);
+    p.stage_words = static_cast<int>(sm.stage_words);
+    p.tab_words = static_cast<int>(sm.tab_words);
+    p.dest_words = static_cast<int>(sm.dest_words);
+    p.lane_stride = static_cast<int>(sm.lane_stride);
+    const RouteWorkspace w = route_workspace(p.lv, kPacked);
+    uint8_t* ws = static_cast<uint8_t*>(a.workspace);
+    p.barrier = reinterpret_cast<unsigned long long*>(ws + w.barrier_off);
+    p.ws_cnt = reinterpret_cast<uint16_t*>(ws + w.cnt_off);
+    p.ws_tot = reinterpret_cast<unsigned long long*>(ws + w.tot_off);
+    p.ws_tri = reinterpret_cast<uint32_t*>(ws + w.tri_off);
+    p.epoch = next_epoch();
+
+    auto kernel = route_fused_kernel<KT, kPacked>;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     cfg.blockDim = dim3(kRouteThreads);
-    cfg.gridDim = dim3(static_cast<unsigned>(cluster));
+    cfg.gridDim = dim3(static_cast<unsigned>(n_ctas));
     cfg.dynamicSmemBytes = sm.bytes();
     cfg.stream = a.stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    {   // can the device hold one such cluster at all?  asked once per (device, kernel, cluster, bytes)
-        static std::mutex lock;
-        static std::map<std::tuple<int, const void*, int, size_t>, bool> fits;
-        int dev = 0;
-        COBALT_CUDA_TRY(cudaGetDevice(&dev));
-        const auto key = std::make_tuple(dev, reinterpret_cast<const void*>(kernel), cluster, sm.bytes());
-        bool known = false, ok = false;
-        {
-            std::lock_guard<std::mutex> guard(lock);
-            auto it = fits.find(key);
-            if (it != fits.end()) { known = true; ok = it->second; }
-        }
-        if (!known) {
-            int max_clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess) {
-                (void)cudaGetLastError();
-                max_clusters = 0;
-            }
-            ok = max_clusters >= 1;
-            std::lock_guard<std::mutex> guard(lock);
-            fits[key] = ok;
-        }
-        if (!ok) return COBALT_OK;
-    }
-    int key_bits = 1;
-    while ((1 << key_bits) <= lv.D) ++key_bits;          // keys 0..D
-    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, lv, a.ids, a.src, a.src_uniform, a.T,
-                                       static_cast<uint32_t>(a.seed & 0xFFFFFFFFu), static_cast<uint32_t>(a.seed >> 32),
-                                       a.coact, a.load, a.assigned_slot, a.remote_nodes,
-                                       reinterpret_cast<unsigned long long*>(a.totals), b.dest_counts, b.dest_offsets,
-                                       b.row_of_pair, b.pair_of_row, static_cast<int>(sm.tri_words),
-                                       static_cast<int>(sm.tab_words), static_cast<int>(sm.dest_words), key_bits,
-                                       a.seed_on_device, a.err_word));
+    attr[0].id = cudaLaunchAttributeCooperative;     // all CTAs resident together: the grid barrier cannot starve
+    attr[0].val.cooperative = 1;
+    COBALT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, p));
     *launched = true;
     return COBALT_OK;
+}
+
+// 0: the triangle does not fit beside the other arrays, 1: it fits with 32-bit counters, 2: with 16-bit ones
+static int fused_mode(const LayoutView& lv, int K, uint32_t tile_flags)
+{
+    // from about 180 experts on the 16-bit triangle is taken even where the 32-bit one fits: the
+    // exchange is bound by the bytes of the partial triangles
+    const bool large_tile = tri_entries(lv.E) * sizeof(uint32_t) >= 64 * 1024;
+    if (large_tile && !(tile_flags & COBALT_STATS_TILE32) && route_smem(lv, K, true).bytes() <= kRouteMaxSmem) return 2;
+    if (route_smem(lv, K, false).bytes() <= kRouteMaxSmem) return 1;
+    if (route_smem(lv, K, true).bytes() <= kRouteMaxSmem) return 2;
+    return 0;
 }
 
 template <int KT>
@@ -587,26 +757,27 @@ static int launch_route_any(const RouteArgs& a, bool packed, bool* launched)
     return packed ? launch_route<KT, true>(a, launched) : launch_route<KT, false>(a, launched);
 }
 
-static ChunkPlan route_chunks(int64_t T, int32_t K)
+static int dispatch_route(const RouteArgs& a, bool packed, bool* launched)
 {
-    ChunkPlan c;
-    c.P = T * K;
-    c.chunk = kRouteChunkTokens * K;
-    c.n_chunks = static_cast<int>((T + kRouteChunkTokens - 1) / kRouteChunkTokens);
-    if (c.n_chunks < 1) c.n_chunks = 1;
-    return c;
-}
-
-// 0: the triangle does not fit beside the tables, 1: it fits with 32-bit counters, 2: with 16-bit ones
-static int fused_mode(const LayoutView& lv, uint32_t tile_flags)
-{
-    // from about 180 experts on the 16-bit triangle is taken even where the 32-bit one fits: the merge
-    // is bound by the bytes that cross distributed shared memory
-    const bool large_tile = tri_entries(lv.E) * sizeof(uint32_t) >= 64 * 1024;
-    if (large_tile && !(tile_flags & COBALT_STATS_TILE32) && route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
-    if (route_smem(lv, false).bytes() <= kRouteMaxSmem) return 1;
-    if (route_smem(lv, true).bytes() <= kRouteMaxSmem) return 2;
-    return 0;
+    switch (a.K) {
+        case 1: return launch_route_any<1>(a, packed, launched);
+        case 2: return launch_route_any<2>(a, packed, launched);
+        case 3: return launch_route_any<3>(a, packed, launched);
+        case 4: return launch_route_any<4>(a, packed, launched);
+        case 5: return launch_route_any<5>(a, packed, launched);
+        case 6: return launch_route_any<6>(a, packed, launched);
+        case 7: return launch_route_any<7>(a, packed, launched);
+        case 8: return launch_route_any<8>(a, packed, launched);
+        case 9: return launch_route_any<9>(a, packed, launched);
+        case 10: return launch_route_any<10>(a, packed, launched);
+        case 11: return launch_route_any<11>(a, packed, launched);
+        case 12: return launch_route_any<12>(a, packed, launched);
+        case 13: return launch_route_any<13>(a, packed, launched);
+        case 14: return launch_route_any<14>(a, packed, launched);
+        case 15: return launch_route_any<15>(a, packed, launched);
+        case 16: return launch_route_any<16>(a, packed, launched);
+        default: *launched = false; return COBALT_OK;
+    }
 }
 
 }  // namespace cobalt
@@ -619,13 +790,12 @@ size_t cobalt_route_index_workspace_bytes(const cobalt_layout_t* layout, int64_t
 {
     if (!layout || T < 0 || K < 1 || K > COBALT_MAX_TOPK || T * static_cast<int64_t>(K) >= (1ll << 31)) return 0;
     const LayoutView& lv = layout->view;
-    const int mode = fused_mode(lv, 0);
-    if (mode == 0 || T == 0) return cobalt_permute_workspace_bytes(T, K, lv.D);
-    const ChunkPlan c = route_chunks(T, K);
-    const size_t fused = round_up(sizeof(uint32_t) * static_cast<size_t>(lv.D) * c.n_chunks, 256);
-    // the call may still take the separate calls (K without a compiled variant, 16-bit counters not
-    // allowed for this T): room for them as well
-    return std::max(fused, cobalt_permute_workspace_bytes(T, K, lv.D));
+    // room for the separate calls as well: the pass falls back to them when the fused kernel does not
+    // fit the layout, the batch or the device
+    size_t need = cobalt_permute_workspace_bytes(T, K, lv.D);
+    if (route_smem(lv, K, false).bytes() <= kRouteMaxSmem) need = std::max(need, route_workspace(lv, false).total);
+    if (route_smem(lv, K, true).bytes() <= kRouteMaxSmem) need = std::max(need, route_workspace(lv, true).total);
+    return need;
 }
 
 int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, const int32_t* src_rank,
@@ -645,7 +815,7 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
         !aligned16(assigned_slot) || !aligned16(totals) || !aligned16(dest_counts) || !aligned16(dest_offsets) ||
         !aligned16(row_of_pair) || !aligned16(pair_of_row) || !aligned16(workspace))
         return COBALT_ERR_INVALID_ARG;
-    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_SEED_ON_DEVICE | COBALT_STATS_TILE32 | COBALT_ROUTE_GENERAL_KERNELS))
+    if (flags & ~(COBALT_STATS_ACCUMULATE | COBALT_SEED_ON_DEVICE | COBALT_STATS_TILE32 | COBALT_ROUTE_SEPARATE_KERNELS))
         return COBALT_ERR_INVALID_ARG;
     const bool seed_on_device = (flags & COBALT_SEED_ON_DEVICE) != 0;
     if (seed_on_device && (seed == 0 || (seed & 7u) != 0)) return COBALT_ERR_INVALID_ARG;
@@ -655,74 +825,39 @@ int cobalt_route_index(const cobalt_layout_t* layout, const int32_t* topk_ids, c
     COBALT_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != layout->device) return COBALT_ERR_INVALID_ARG;
 
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int mode = fused_mode(lv, flags & COBALT_STATS_TILE32);
+    const int mode = fused_mode(lv, K, flags & COBALT_STATS_TILE32);
     bool launched = false;
-    const ChunkPlan c = route_chunks(T, K);
-    // The kernel is compiled for K = 1, 2, 4, 6, 8, 10, 12, 16 with the K ids of a token in registers; its variant
-    // for any other K (loops to 16, spills) measured slower than the separate calls (K = 10: 85 us
-    // against 58 us at T = 65536, E = 256), so those take the separate calls.
-    const bool k_compiled = K == 1 || K == 2 || K == 4 || K == 6 || K == 8 || K == 10 || K == 12 || K == 16;
-    if (mode != 0 && T > 0 && k_compiled) {
+    if (mode != 0 && T > 0 && !(flags & COBALT_ROUTE_SEPARATE_KERNELS)) {
         RouteArgs a;
-        a.zero = ZeroList{{nullptr, nullptr, reinterpret_cast<uint32_t*>(totals), nullptr}, {0, 0, 4, 0}};
-        if (!(flags & COBALT_STATS_ACCUMULATE)) {
-            a.zero.ptr[0] = coact; a.zero.n[0] = lv.E * lv.E;
-            a.zero.ptr[1] = load;  a.zero.n[1] = lv.E;
-        }
-        a.lv = &lv; a.ids = topk_ids; a.src = src_rank; a.src_uniform = src_rank_uniform; a.T = T; a.K = K;
-        a.seed = seed_on_device ? 0 : seed;
-        a.seed_on_device = seed_on_device ? reinterpret_cast<const unsigned long long*>(static_cast<uintptr_t>(seed)) : nullptr;
-        a.coact = coact; a.load = load; a.assigned_slot = assigned_slot; a.remote_nodes = remote_nodes; a.totals = totals;
-        a.chunk_ws = static_cast<uint32_t*>(workspace); a.n_chunks = c.n_chunks; a.stream = s;
-        int rc = device_error_word(&a.err_word);
+        RouteParams& p = a.p;
+        p.lv = lv;
+        p.topk_ids = topk_ids; p.src_rank = src_rank; p.src_uniform = src_rank_uniform; p.T = T; p.K_rt = K;
+        p.seed_lo = seed_on_device ? 0u : static_cast<uint32_t>(seed & 0xFFFFFFFFu);
+        p.seed_hi = seed_on_device ? 0u : static_cast<uint32_t>(seed >> 32);
+        p.seed_on_device = seed_on_device ? reinterpret_cast<const unsigned long long*>(static_cast<uintptr_t>(seed)) : nullptr;
+        p.coact = coact; p.load = load; p.assigned_slot = assigned_slot; p.remote_nodes = remote_nodes;
+        p.totals = reinterpret_cast<unsigned long long*>(totals);
+        p.dest_counts = dest_counts; p.dest_offsets = dest_offsets; p.row_of_pair = row_of_pair; p.pair_of_row = pair_of_row;
+        p.accumulate = (flags & COBALT_STATS_ACCUMULATE) ? 1 : 0;
+        a.K = K; a.workspace = workspace; a.stream = static_cast<cudaStream_t>(stream);
+        int rc = device_error_word(&p.err_word);
         if (rc != COBALT_OK) return rc;
-        rc = sm_count(&a.n_sm);
-        if (rc != COBALT_OK) return rc;
-        if (!(flags & COBALT_ROUTE_GENERAL_KERNELS) && K <= 8) {
-            const SmallArgs b = {dest_counts, dest_offsets, row_of_pair, pair_of_row, (flags & COBALT_STATS_ACCUMULATE) != 0};
-            bool small = false;
-            switch (K) {
-                case 1: rc = launch_route_small<1>(a, b, &small); break;
-                case 2: rc = launch_route_small<2>(a, b, &small); break;
-                case 4: rc = launch_route_small<4>(a, b, &small); break;
-                case 6: rc = launch_route_small<6>(a, b, &small); break;
-                default: rc = launch_route_small<8>(a, b, &small);
-            }
-            if (rc != COBALT_OK || small) return rc;     // the single kernel has done everything
-        }
-        auto launch_general = [&](bool packed) {
-            switch (K) {
-                case 1: return launch_route_any<1>(a, packed, &launched);
-                case 2: return launch_route_any<2>(a, packed, &launched);
-                case 4: return launch_route_any<4>(a, packed, &launched);
-                case 6: return launch_route_any<6>(a, packed, &launched);
-                case 8: return launch_route_any<8>(a, packed, &launched);
-                case 10: return launch_route_any<10>(a, packed, &launched);
-                case 12: return launch_route_any<12>(a, packed, &launched);
-                case 16: return launch_route_any<16>(a, packed, &launched);
-                default: return static_cast<int>(COBALT_ERR_UNSUPPORTED);
-            }
-        };
-        rc = launch_general(mode == 2);
+        rc = dispatch_route(a, mode == 2, &launched);
         // 16-bit counters refused for this many tokens: the 32-bit triangle, if it fits
-        if (rc == COBALT_OK && !launched && mode == 2 && route_smem(lv, false).bytes() <= kRouteMaxSmem)
-            rc = launch_general(false);
-        if (rc != COBALT_OK) return rc;
+        if (rc == COBALT_OK && !launched && mode == 2 && route_smem(lv, K, false).bytes() <= kRouteMaxSmem)
+            rc = dispatch_route(a, false, &launched);
+        if (rc != COBALT_OK || launched) return rc;
     }
-    if (!launched) {
-        // the co-activation triangle does not fit beside the tables (or there is nothing to route):
-        // same results from the separate calls
-        int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags & COBALT_STATS_ACCUMULATE, nullptr, 0, stream);
-        if (rc != COBALT_OK) return rc;
-        rc = cobalt_assign(layout, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot, nullptr,
-                           remote_nodes, totals, flags & COBALT_SEED_ON_DEVICE, nullptr, 0, stream);
-        if (rc != COBALT_OK) return rc;
-        return cobalt_permute_index(assigned_slot, T, K, lv.D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
-                                    workspace, workspace_bytes, stream);
-    }
-    return launch_scan_and_rank(assigned_slot, T * K, lv.D, c, static_cast<uint32_t*>(workspace), dest_counts, dest_offsets,
-                                row_of_pair, pair_of_row, 0, s);
+    // the fused kernel does not fit (or there is nothing to route, or the caller asked for it): the
+    // same results from the separate calls
+    int rc = cobalt_coact_stats(topk_ids, T, K, lv.E, coact, load, flags & (COBALT_STATS_ACCUMULATE | COBALT_STATS_TILE32),
+                                nullptr, 0, stream);
+    if (rc != COBALT_OK) return rc;
+    rc = cobalt_assign(layout, topk_ids, src_rank, src_rank_uniform, T, K, seed, assigned_slot, nullptr,
+                       remote_nodes, totals, flags & COBALT_SEED_ON_DEVICE, nullptr, 0, stream);
+    if (rc != COBALT_OK) return rc;
+    return cobalt_permute_index(assigned_slot, T, K, lv.D, dest_counts, dest_offsets, row_of_pair, pair_of_row,
+                                workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

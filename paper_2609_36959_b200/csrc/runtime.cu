@@ -122,16 +122,21 @@ static int build_tables(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
 
     view->N = N; view->Q = Q; view->S = S; view->E = E; view->G = G; view->D = D;
     view->n_replicas = n_replicas;
-    view->words = E * N + E + n_replicas + E;
+    view->words = E * N + E + n_replicas + kCoverTableWords;
     view->blob = nullptr;
+    // s / Q by multiplication, verified for every source rank
+    view->q_inverse = (1u << 20) / static_cast<uint32_t>(Q) + 1u;
+    for (int32_t s = 0; s < G; ++s)
+        if (static_cast<int32_t>((static_cast<uint64_t>(s) * view->q_inverse) >> 20) != s / Q) return COBALT_ERR_UNSUPPORTED;
     if (!blob) return COBALT_OK;
 
     blob->assign(static_cast<size_t>(view->words + 3) / 4 * 4, 0u);   // whole 16-byte vectors
     uint32_t* ent = blob->data() + view->ent_off();
     uint32_t* primary = blob->data() + view->primary_off();
     uint32_t* rlist = blob->data() + view->rlist_off();
-    uint32_t* nodes = blob->data() + view->nodes_off();
+    uint8_t* cover = reinterpret_cast<uint8_t*>(blob->data() + view->cover_off());
     std::vector<int32_t> fill(static_cast<size_t>(E) * N, 0);
+    std::vector<uint32_t> nodes(static_cast<size_t>(E), 0u);          // N_e as a bitmask over nodes
     for (int32_t e = 0; e < E; ++e) primary[e] = 0xFFFFFFFFu;
     for (int32_t d = 0; d < D; ++d) {  // ascending slot id => every R_{e,n} list is ascending
         const int32_t e = slot_expert[d];
@@ -143,11 +148,37 @@ static int build_tables(int32_t N, int32_t Q, int32_t S, int32_t E, const int32_
         nodes[e] |= 1u << n;
         if (primary[e] == 0xFFFFFFFFu) primary[e] = static_cast<uint32_t>(d);
     }
-    for (size_t en = 0; en < static_cast<size_t>(E) * N; ++en)
-        ent[en] = (static_cast<uint32_t>(offset[en]) << 8) | static_cast<uint32_t>(count[en]);
     if (primary_in)
         for (int32_t e = 0; e < E; ++e) primary[e] = static_cast<uint32_t>(primary_in[e]);
-    for (int32_t e = 0; e < E; ++e) primary[e] |= (primary[e] / static_cast<uint32_t>(S * Q)) << 24;
+    for (int32_t e = 0; e < E; ++e) {
+        const uint32_t primary_node = primary[e] / static_cast<uint32_t>(S * Q);
+        for (int32_t n = 0; n < N; ++n) {
+            // the remote mask of e for a token whose source node is n: the nodes holding e with node n
+            // taken out of the numbering; 0 when n holds e (the expert then runs on the source node)
+            uint32_t m = 0;
+            if (!(nodes[e] & (1u << n))) m = ((nodes[e] >> (n + 1)) << n) | (nodes[e] & ((1u << n) - 1u));
+            const size_t en = static_cast<size_t>(e) * N + n;
+            ent[en] = static_cast<uint32_t>(count[en]) | (static_cast<uint32_t>(offset[en]) << kEntCountBits) |
+                      (m << kEntMaskShift) | (primary_node << kEntPrimaryNodeShift);
+        }
+    }
+    // Smallest cover for every set of mask values (N <= 4: values 1 .. 2^(N-1)-1, at most seven), found
+    // with Algorithm 1's own search: candidates b ascend from 0, a candidate replaces the best so far
+    // only when it covers every mask of the set with strictly fewer nodes; the search starts from the
+    // set of all remote nodes.
+    if (N <= 4) {
+        const uint32_t full = (1u << (N - 1)) - 1u;
+        for (uint32_t present = 0; present < 128u; ++present) {
+            uint32_t best = full;
+            for (uint32_t b = 0; b < full; ++b) {
+                bool covers = true;
+                for (uint32_t v = 1; v <= 7u; ++v)
+                    if ((present & (1u << (v - 1))) && v <= full && (b & v) == 0) covers = false;
+                if (covers && __builtin_popcount(b) < __builtin_popcount(best)) best = b;
+            }
+            cover[present] = static_cast<uint8_t>(best);
+        }
+    }
     return COBALT_OK;
 }
 

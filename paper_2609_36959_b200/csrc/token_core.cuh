@@ -81,14 +81,73 @@ __device__ __forceinline__ void store_token_slots(int32_t* __restrict__ dst, con
     }
 }
 
+// The K ids of a token in ascending order (a compare-exchange network, fully unrolled; entries past K
+// are padded with a value above every id so that they stay at the end).
+template <int KT>
+__device__ __forceinline__ void sort_token_ids(const int32_t (&id)[TokenShape<KT>::KMAX], int K,
+                                               int32_t (&s)[TokenShape<KT>::KMAX])
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) s[a] = (a < K) ? id[a] : 0x7FFFFFFF;
+#pragma unroll
+    for (int pass = 0; pass < KMAX; ++pass) {
+#pragma unroll
+        for (int a = pass & 1; a + 1 < KMAX; a += 2) {
+            const int32_t lo = min(s[a], s[a + 1]), hi = max(s[a], s[a + 1]);
+            s[a] = lo;
+            s[a + 1] = hi;
+        }
+    }
+}
+
+// The same checks as check_token_ids on ids that are already sorted: the range is decided by the two
+// ends, a repeated id by its neighbour.
+template <int KT>
+__device__ __forceinline__ uint32_t check_sorted_ids(const int32_t (&s)[TokenShape<KT>::KMAX], int K, int E)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+    uint32_t bad = 0;
+    bool high = false, twice = false;
+#pragma unroll
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            high = high || s[a] >= E;
+            if (a > 0) twice = twice || s[a] == s[a - 1];
+        }
+    }
+    if (s[0] < 0 || high) bad |= COBALT_DEVERR_BAD_EXPERT_ID;
+    if (twice) bad |= COBALT_DEVERR_DUPLICATE_ID;
+    return bad;
+}
+
 // Layout tables staged in shared memory (see LayoutView for the word layout).
 struct TableView {
     const uint32_t* ent;
     const uint32_t* primary;
     const uint32_t* rlist;
-    const uint32_t* nodes;
-    int N, Q, G, E;
+    const uint8_t* cover;
+    int N, G, E;
+    uint32_t q_inverse;
 };
+
+__device__ __forceinline__ uint32_t ent_count(uint32_t w) { return w & ((1u << kEntCountBits) - 1u); }
+__device__ __forceinline__ uint32_t ent_offset(uint32_t w) { return (w >> kEntCountBits) & ((1u << kEntOffsetBits) - 1u); }
+__device__ __forceinline__ uint32_t ent_remote_mask(uint32_t w) { return (w >> kEntMaskShift) & 0x7Fu; }
+__device__ __forceinline__ uint32_t ent_primary_node(uint32_t w) { return w >> kEntPrimaryNodeShift; }
+
+// The view of tables that are (or will be) staged at `tab`.
+__device__ __forceinline__ TableView table_view(const LayoutView& lv, const uint32_t* tab)
+{
+    TableView tv;
+    tv.ent = tab + lv.ent_off();
+    tv.primary = tab + lv.primary_off();
+    tv.rlist = tab + lv.rlist_off();
+    tv.cover = reinterpret_cast<const uint8_t*>(tab + lv.cover_off());
+    tv.N = lv.N; tv.G = lv.G; tv.E = lv.E;
+    tv.q_inverse = lv.q_inverse;
+    return tv;
+}
 
 __device__ __forceinline__ TableView stage_tables(const LayoutView& lv, uint32_t* tab)
 {
@@ -98,18 +157,12 @@ __device__ __forceinline__ TableView stage_tables(const LayoutView& lv, uint32_t
     const int n_vec = (lv.words + 3) / 4;
 #pragma unroll 4
     for (int i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = __ldg(src + i);
-    TableView tv;
-    tv.ent = tab + lv.ent_off();
-    tv.primary = tab + lv.primary_off();
-    tv.rlist = tab + lv.rlist_off();
-    tv.nodes = tab + lv.nodes_off();
-    tv.N = lv.N; tv.Q = lv.Q; tv.G = lv.G; tv.E = lv.E;
-    return tv;
+    return table_view(lv, tab);
 }
 
 // What assign_token writes per task.
 enum AssignMode {
-    kAssignSlot = 0,      // Algorithm 1 with the hashed uniform replica pick (lines 14-15)
+    kAssignSlot = 0,      // Algorithm 1 with the hashed uniform replica pick (Step 2)
     kAssignNaive = 1,     // every task to its expert's primary replica
     kAssignGroupKey = 2,  // Step 1 only: out = e * N + n_te (the replica is picked later, in task order)
 };
@@ -124,74 +177,94 @@ __device__ __forceinline__ void assign_token(const TableView& tv, const int32_t 
 {
     constexpr int KMAX = TokenShape<KT>::KMAX;
     const int N = tv.N;
-    const int n_s = s_t / tv.Q;                       // N(s_t)
+    const int n_s = static_cast<int>(__umulhi(static_cast<uint32_t>(s_t) << 12, tv.q_inverse));   // N(s_t) = s_t / Q
     const uint32_t src_bit = 1u << n_s;
-    const uint32_t low = src_bit - 1u;
 
-    // the naive rule's term of Eq. 1: distinct nodes of the primaries, source excluded
+    // One table word per expert, read for the token's own source node: the remote mask m_{t,e} (0 if
+    // the expert is present on the source node, i.e. not in U_t), the replicas on the source node,
+    // and the node of the primary replica (for the naive rule's term of Eq. 1).
+    uint32_t w[KMAX];
     uint32_t naive_nodes = 0;
 #pragma unroll
-    for (int a = 0; a < KMAX; ++a)
-        if (a < K) naive_nodes |= 1u << (tv.primary[id[a]] >> 24);
+    for (int a = 0; a < KMAX; ++a) {
+        if (a < K) {
+            w[a] = tv.ent[id[a] * N + n_s];
+            naive_nodes |= 1u << ent_primary_node(w[a]);
+        }
+    }
     naive_cost = __popc(naive_nodes & ~src_bit);
 
     if (MODE == kAssignNaive) {
 #pragma unroll
         for (int a = 0; a < KMAX; ++a)
-            if (a < K) out[a] = static_cast<int32_t>(tv.primary[id[a]] & 0xFFFFFFu);
+            if (a < K) out[a] = static_cast<int32_t>(tv.primary[id[a]]);
         cost = naive_cost;
         return;
     }
 
-    // lines 3-4: U_t and the remote masks; bit j <-> j-th node after skipping n_s.
-    // m[a] == 0 marks an expert that is present on the source node.
-    uint32_t m[KMAX];
-    uint32_t any_remote = 0, common = 0xFFFFFFFFu;
-#pragma unroll
-    for (int a = 0; a < KMAX; ++a) {
-        if (a < K) {
-            const uint32_t held = tv.nodes[id[a]];
-            m[a] = (held & src_bit) ? 0u : (((held >> (n_s + 1)) << n_s) | (held & low));
-            any_remote |= m[a];
-            if (m[a]) common &= m[a];
-        }
-    }
-    // lines 5-8: ascending b, strictly smaller popcount replaces b*.  A single node covers U_t
-    // iff every mask has its bit, and the lowest such bit is the smallest one-bit b; only
-    // otherwise are the masks with two or more bits enumerated.
+    // b*: the fewest remote nodes that meet every mask, the numerically smallest among equals (the
+    // outcome of scanning all (N-1)-bit masks in ascending order and replacing the candidate only on
+    // a strictly smaller node count).  Up to four nodes a mask is one of seven values, and the answer
+    // for every set of values present is looked up in a table built once per layout by that very
+    // scan.  Beyond that: a single node covers U_t iff every mask has its bit, and the lowest such
+    // bit is the smallest one-bit candidate; only otherwise are the candidates with two or more bits
+    // scanned.
     uint32_t b_star = 0;
-    cost = 0;
-    if (any_remote) {
-        if (common) {
-            b_star = common & (0u - common);
-        } else {
-            const uint32_t full = (1u << (N - 1)) - 1u;
-            b_star = full;
-            int best = N - 1;
-            for (uint32_t b = 3; b < full; ++b) {
-                const int pc = __popc(b);
-                if (pc >= best) continue;
-                bool feasible = true;
+    if (N <= 4) {
+        uint32_t present = 0;
 #pragma unroll
-                for (int a = 0; a < KMAX; ++a)
-                    if (a < K) feasible = feasible && (m[a] == 0 || (b & m[a]) != 0);
-                if (feasible) {
-                    b_star = b;
-                    best = pc;
-                    if (pc == 2) break;  // one node is known not to suffice
+        for (int a = 0; a < KMAX; ++a)
+            if (a < K) present |= 1u << ent_remote_mask(w[a]);
+        b_star = tv.cover[present >> 1];                 // bit 0 (mask 0: a local expert) drops out
+    } else {
+        uint32_t any_remote = 0, common = 0xFFFFFFFFu;
+#pragma unroll
+        for (int a = 0; a < KMAX; ++a) {
+            if (a < K) {
+                const uint32_t m = ent_remote_mask(w[a]);
+                any_remote |= m;
+                if (m) common &= m;
+            }
+        }
+        if (any_remote) {
+            if (common) {
+                b_star = common & (0u - common);
+            } else {
+                const uint32_t full = (1u << (N - 1)) - 1u;
+                b_star = full;
+                int best = N - 1;
+                for (uint32_t b = 3; b < full; ++b) {
+                    const int pc = __popc(b);
+                    if (pc >= best) continue;
+                    bool feasible = true;
+#pragma unroll
+                    for (int a = 0; a < KMAX; ++a) {
+                        if (a < K) {
+                            const uint32_t m = ent_remote_mask(w[a]);
+                            feasible = feasible && (m == 0 || (b & m) != 0);
+                        }
+                    }
+                    if (feasible) {
+                        b_star = b;
+                        best = pc;
+                        if (pc == 2) break;  // one node is known not to suffice
+                    }
                 }
             }
         }
-        cost = __popc(b_star);
     }
-    // lines 9-16: node per expert, then a replica inside the node
+    cost = __popc(b_star);
+
+    // node per expert (Step 1), then a replica inside the node (Step 2)
 #pragma unroll
     for (int a = 0; a < KMAX; ++a) {
         if (a < K) {
             int node = n_s;
-            if (m[a] != 0) {
+            uint32_t e_n = w[a];                         // R_{e,N(s_t)} for an expert that stays local
+            const uint32_t m = ent_remote_mask(w[a]);
+            if (m != 0) {
                 // RandomNode: the i-th set bit of b* & m; a single candidate needs no draw
-                uint32_t c = b_star & m[a];
+                uint32_t c = b_star & m;
                 const uint32_t n_c = __popc(c);
                 if (n_c > 1) {
                     const uint32_t i = hash_index(route_hash(seed_lo, seed_hi, t, id[a], 0u), n_c);
@@ -199,15 +272,35 @@ __device__ __forceinline__ void assign_token(const TableView& tv, const int32_t 
                 }
                 const int bit = __ffs(c) - 1;
                 node = bit + (bit >= n_s ? 1 : 0);
+                if (MODE != kAssignGroupKey) e_n = tv.ent[id[a] * N + node];
             }
             if (MODE == kAssignGroupKey) {
                 out[a] = id[a] * N + node;
             } else {
                 // UniformChoice over R_{e,node}; floor(x * 1 / 2^32) = 0, so one replica needs no draw
-                const uint32_t e_n = tv.ent[id[a] * N + node];
-                const uint32_t n_r = e_n & 0xFFu;
+                const uint32_t n_r = ent_count(e_n);
                 const uint32_t i = (n_r > 1) ? hash_index(route_hash(seed_lo, seed_hi, t, id[a], 1u), n_r) : 0u;
-                out[a] = static_cast<int32_t>(tv.rlist[(e_n >> 8) + i]);
+                out[a] = static_cast<int32_t>(tv.rlist[ent_offset(e_n) + i]);
+            }
+        }
+    }
+}
+
+// Adds the K(K+1)/2 unordered pairs of one token (diagonal included) to a lower-triangle tile, from
+// ids in ascending order: entry (s[b], s[a]) with a <= b sits at s[b](s[b]+1)/2 + s[a].
+template <int KT, bool kPacked>
+__device__ __forceinline__ void add_sorted_token_to_triangle(uint32_t* tri, const int32_t (&s)[TokenShape<KT>::KMAX], int K)
+{
+    constexpr int KMAX = TokenShape<KT>::KMAX;
+#pragma unroll
+    for (int b = 0; b < KMAX; ++b) {
+        if (b < K) {
+            const int row = s[b] * (s[b] + 1) / 2;
+#pragma unroll
+            for (int a = 0; a <= b; ++a) {
+                const int idx = row + s[a];
+                if (kPacked) atomicAdd(&tri[idx >> 1], (idx & 1) ? 0x10000u : 1u);
+                else atomicAdd(&tri[idx], 1u);
             }
         }
     }

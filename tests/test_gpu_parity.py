@@ -341,14 +341,44 @@ def test_fused_route_index_on_configs(cb, name):
     (1000, 20, 5, 8, 8, 1, 5, 0), (2049, 40, 8, 8, 2, 4, 6, 0), (4099, 100, 16, 8, 4, 8, 5, 7),
     (5000, 257, 7, 8, 4, 4, 20, 0), (6000, 700, 8, 8, 4, 8, 24, 0), (200000, 6, 2, 8, 4, 2, 1, 0),
     (1100000, 40, 4, 8, 4, 2, 6, 0),
-    # E = 320..440: the fused pass keeps the triangle in 16-bit counters; with 600000 tokens a cluster
-    # would see more than 65535 of them and the separate calls take over
+    # 200000 and 1100000 tokens: several rounds of 1024 tokens per CTA (the ranks are worked out round by
+    # round after the barrier).  E = 320..440: the triangle only fits with 16-bit counters; with 600000
+    # tokens the 32-bit triangle (E = 330) takes over; E = 1024 or D = 4096: the separate calls
     (20000, 384, 8, 8, 4, 8, 13, 0), (131072, 320, 8, 8, 4, 8, 11, 3), (9000, 440, 6, 8, 2, 4, 56, 0),
     (600000, 330, 2, 8, 4, 2, 42, 0), (3000, 1024, 16, 8, 8, 8, 64, 0)])
 def test_fused_route_index_edge_shapes(cb, T, E, K, H, N, Q, S, empty):
     w = W.make_custom(T, E, K, H, N, Q, S, seed=2000 + T + E, C=3, p_in=0.6, n_empty=empty)
     layout, step = make_step(w, with_x=False)
     run_fused_and_compare(cb, w, step, 31337)
+
+
+def test_fused_pass_starts_from_any_workspace_contents_and_runs_beside_itself(cb):
+    """The grid barrier of the fused kernel lives in the workspace and must not depend on what it finds
+    there: all ones, all zeros, what the previous call left, a word that looks like a barrier of
+    another launch.  Two calls on two streams, each with its own workspace, may overlap."""
+    w = W.make_config("3", T=20000)
+    layout, step = make_step(w, with_x=False)
+    for fill in (0xFF, 0x00, None, 0x5A):
+        if fill is not None:
+            step.workspace.fill_(fill)
+        run_fused_and_compare(cb, w, step, 99)
+    step.workspace.view(torch.int64)[0] = (12345 << 32) | 7          # epoch 12345, seven arrivals
+    run_fused_and_compare(cb, w, step, 99)
+    ref = {k: getattr(step, k).clone() for k in ("coact", "assigned_slot", "row_of_pair", "pair_of_row", "dest_offsets")}
+    layout2, other = make_step(w, with_x=False)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(10):
+        for st, stream in ((step, s1), (other, s2)):
+            with torch.cuda.stream(stream):
+                cb.route_index(st.layout, st.topk_ids, st.src_rank, 99, st.coact, st.load, st.assigned_slot,
+                               st.dest_counts, st.dest_offsets, st.row_of_pair, st.workspace,
+                               remote_nodes=st.remote_nodes, totals=st.totals, pair_of_row=st.pair_of_row)
+    torch.cuda.synchronize()
+    assert cb.read_and_clear_device_error() == 0
+    for st in (step, other):
+        for k, v in ref.items():
+            assert torch.equal(getattr(st, k), v), k
 
 
 def test_step_with_statistics_on_a_side_stream(cb):
@@ -372,17 +402,17 @@ def test_step_with_statistics_on_a_side_stream(cb):
 @pytest.mark.parametrize("T,E,K,N,Q,S,empty", [(4096, 256, 8, 4, 8, 9, 0), (4095, 64, 6, 4, 8, 3, 2), (257, 16, 2, 2, 4, 3, 0),
                                                (1, 8, 1, 1, 2, 4, 0), (3000, 100, 4, 8, 4, 4, 5), (2049, 24, 8, 3, 2, 5, 0),
                                                (4000, 384, 8, 4, 8, 13, 0), (4096, 420, 6, 2, 4, 60, 7)])
-def test_fused_pass_in_a_single_cluster(cb, T, E, K, N, Q, S, empty):
-    """Up to 16 chunks of 256 tokens the fused entry runs ONE kernel in one cluster (histograms
-    exchanged through distributed shared memory, statistics stored instead of added).  Same results
-    as the oracle, as the general kernels (COBALT_ROUTE_GENERAL_KERNELS), and with the
-    accumulate flag on top of what is already there."""
+def test_fused_pass_on_small_batches(cb, T, E, K, N, Q, S, empty):
+    """Small batches run the fused kernel on a few CTAs (256 tokens each, down to a single CTA), large
+    triangles beside many destinations fall back to the separate calls.  Same results as the oracle,
+    as the separate calls (COBALT_ROUTE_SEPARATE_KERNELS), and with the accumulate flag on top of
+    what is already there."""
     w = W.make_custom(T, E, K, 8, N, Q, S, seed=900 + T, C=2, p_in=0.7, n_empty=empty)
     layout, step = make_step(w, with_x=False)
     run_fused_and_compare(cb, w, step, 321)
     small = {k: getattr(step, k).clone() for k in ("coact", "load", "assigned_slot", "dest_counts", "dest_offsets",
                                                      "row_of_pair", "pair_of_row", "remote_nodes", "totals")}
-    run_fused_and_compare(cb, w, step, 321, flags=cb.ROUTE_GENERAL_KERNELS)
+    run_fused_and_compare(cb, w, step, 321, flags=cb.ROUTE_SEPARATE_KERNELS)
     for k, v in small.items():
         assert torch.equal(getattr(step, k), v), k
     cb.route_index(layout, step.topk_ids, step.src_rank, 321, step.coact, step.load, step.assigned_slot,
@@ -688,8 +718,8 @@ def test_bad_data_sets_the_error_word(cb):
 
 @pytest.mark.parametrize("T", [2000, 9000])
 def test_bad_data_through_the_fused_entry(cb, T):
-    """The one-pass kernels (single cluster at T = 2000, general at T = 9000) treat bad tokens exactly as
-    the separate calls do: same error bits, slots of -1, rows of -1, counts without them."""
+    """The fused kernel (a few CTAs at T = 2000, 36 at T = 9000) treats bad tokens exactly as the
+    separate calls do: same error bits, slots of -1, rows of -1, counts without them."""
     w = W.make_config("3", T=T)
     layout, step = make_step(w, with_x=False)
     ids = w.topk_ids.copy()
