@@ -255,32 +255,34 @@ __device__ __forceinline__ void assign_token(const TableView& tv, const int32_t 
     }
     cost = __popc(b_star);
 
-    // node per expert (Step 1), then a replica inside the node (Step 2)
+    // Node per expert (Step 1), then a replica inside the node (Step 2).  Written without branches, so
+    // that the K experts' chains (table loads, hashes) are independent straight-line code that the
+    // scheduler can interleave: a draw among one candidate is floor(x * 1 / 2^32) = 0 whatever x is, and
+    // an expert that stays local simply reads its own table word again.
+    const bool few_nodes = N <= 4;                       // at most three remote nodes: two bits to drop at most
 #pragma unroll
     for (int a = 0; a < KMAX; ++a) {
         if (a < K) {
-            int node = n_s;
-            uint32_t e_n = w[a];                         // R_{e,N(s_t)} for an expert that stays local
             const uint32_t m = ent_remote_mask(w[a]);
-            if (m != 0) {
-                // RandomNode: the i-th set bit of b* & m; a single candidate needs no draw
-                uint32_t c = b_star & m;
-                const uint32_t n_c = __popc(c);
-                if (n_c > 1) {
-                    const uint32_t i = hash_index(route_hash(seed_lo, seed_hi, t, id[a], 0u), n_c);
-                    for (uint32_t j = 0; j < i; ++j) c &= c - 1u;   // drop the i lowest set bits
-                }
-                const int bit = __ffs(c) - 1;
-                node = bit + (bit >= n_s ? 1 : 0);
-                if (MODE != kAssignGroupKey) e_n = tv.ent[id[a] * N + node];
+            // RandomNode: the i-th set bit of b* & m, i uniform over the candidates
+            uint32_t c = b_star & m;
+            const uint32_t i = hash_index(route_hash(seed_lo, seed_hi, t, id[a], 0u), __popc(c));
+            if (few_nodes) {
+#pragma unroll
+                for (uint32_t j = 0; j < 2; ++j) c = (j < i) ? (c & (c - 1u)) : c;
+            } else {
+#pragma unroll
+                for (uint32_t j = 0; j < COBALT_MAX_NODES - 2; ++j) c = (j < i) ? (c & (c - 1u)) : c;
             }
+            const int bit = __ffs(c) - 1;
+            const int node = (m != 0) ? bit + (bit >= n_s ? 1 : 0) : n_s;
             if (MODE == kAssignGroupKey) {
                 out[a] = id[a] * N + node;
             } else {
-                // UniformChoice over R_{e,node}; floor(x * 1 / 2^32) = 0, so one replica needs no draw
-                const uint32_t n_r = ent_count(e_n);
-                const uint32_t i = (n_r > 1) ? hash_index(route_hash(seed_lo, seed_hi, t, id[a], 1u), n_r) : 0u;
-                out[a] = static_cast<int32_t>(tv.rlist[ent_offset(e_n) + i]);
+                // UniformChoice over R_{e,node}
+                const uint32_t e_n = tv.ent[id[a] * N + node];
+                const uint32_t r = hash_index(route_hash(seed_lo, seed_hi, t, id[a], 1u), ent_count(e_n));
+                out[a] = static_cast<int32_t>(tv.rlist[ent_offset(e_n) + r]);
             }
         }
     }
