@@ -39,9 +39,41 @@ def kernels_per_step(T):
     (at most 16 CTAs of 256 tokens) store their sums and need no clearing kernel."""
     return KERNELS_PER_STEP - (1 if 0 < T <= 4096 else 0)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (bytes per pair, measured on a reduced token count and scaled by the pairs of a launch)
-NCU_TRAFFIC_BYTES_PER_PAIR = {"permute_rows": 15683.4, "combine": 15972.4}   # profiles/perm_rows_and_combine_T16384.md
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "row_kernels_traffic.json")
+COUNTERS_JSON = os.path.join(ROOT, "profiles", "index_kernels_counters.json")
+
+
+def load_json(path):
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return {}
+
+
+def traffic_from_ncu_csv(csv_path, tokens, K, H, command):
+    """Turns `ncu -i <report> --page raw --csv` of a reduced-size capture into the per-pair DRAM
+    traffic of the two row kernels and writes it where the benchmark reads it."""
+    import csv
+    with open(csv_path) as f:
+        rows = list(csv.reader(f))
+    hdr = rows[0]
+    out = load_json(TRAFFIC_JSON)
+    names = {"perm_rows_bulk_oneshot_kernel": "permute_rows", "combine_kernel": "combine"}
+    for r in rows[2:]:
+        d = dict(zip(hdr, r))
+        stage = next((v for k, v in names.items() if k in d.get("Kernel Name", "")), None)
+        if stage is None or "backward" in d.get("Kernel Name", ""):
+            continue
+        total = float(d["dram__bytes_read.sum"]) + float(d["dram__bytes_write.sum"])
+        unit = hdr.index("dram__bytes_read.sum")
+        scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}.get(rows[1][unit], 1.0)
+        out[stage] = {"bytes_per_pair": total * scale / (tokens * K), "captured_tokens": tokens, "K": K, "H": H,
+                      "kernel": d["Kernel Name"], "command": command}
+    with open(TRAFFIC_JSON, "w") as f:
+        json.dump(out, f, indent=1, sort_keys=True)
+        f.write("\n")
+    return out
 
 
 def parse_args():
@@ -54,10 +86,21 @@ def parse_args():
     ap.add_argument("--hidden", type=int, default=None, help="override H (tiny rows isolate the index stages)")
     ap.add_argument("--impl", default="cobalt", choices=["cobalt", "reference"])
     ap.add_argument("--cpu-sample-tokens", type=int, default=None,
-                    help="tokens of the workload the CPU oracle is timed on (default 32768; 8192 for --impl reference)")
+                    help="tokens of the workload the CPU oracle is timed on (default 32768 in both legs)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="only the timed step loop (for launch lists under a profiler)")
+    ap.add_argument("--clock-period-ms", type=float, default=8.0,
+                    help="period of the SM clock / throttle-reason sampling during the timed region (0 = no sampling)")
+    ap.add_argument("--traffic-from", default=None, metavar="CSV",
+                    help="no benchmark: read `ncu -i <report> --page raw --csv` of a reduced-size capture of the row "
+                         "kernels (taken with --tokens T) and write profiles/row_kernels_traffic.json")
+    ap.add_argument("--counters-from", default=None, metavar="CSV",
+                    help="no benchmark: read `ncu -i <report> --page raw --csv` of the index kernels and write "
+                         "profiles/index_kernels_counters.json")
+    ap.add_argument("--traffic-command", default="", help="the command that made the capture, recorded beside the figures")
+    ap.add_argument("--summarise", nargs="+", default=None, metavar="JSON",
+                    help="no benchmark: print a markdown table (per-stage times and fractions) of earlier output lines")
     return ap.parse_args()
 
 
@@ -102,35 +145,62 @@ def oracle_step(w, x_bits):
     return time.perf_counter() - t0
 
 
-def cpu_sample(config, tokens):
+CPU_SAMPLE_TOKENS = 32768          # the oracle is timed on the first tokens of the workload, in both legs
+
+
+def cpu_sample(config, tokens, hidden=None):
     import workloads as W
     w = W.make_config(config, T=tokens)
+    if hidden is not None:
+        w.H = hidden
     return w, w.hidden_rows()
+
+
+def cpu_sample_text(ws, extra=""):
+    return (f"first {ws.T} tokens of the workload ({ws.P} pairs), all four stages of the oracle as it stands, "
+            f"single thread{extra}")
+
+
+def config_dict(name_T, w):
+    """The `config` object of the JSON line: the same for both arms (the reference arm describes the
+    workload it samples, not the sample; that is in cpu_baseline.sample)."""
+    cold = name_T * w.K * w.H * 2 > (1 << 28)
+    return {"workload": workload_name(w, T=name_T), "seed": int(w.seed),
+            "l2": ("no explicit flush: each step streams the send buffer (larger than L2) through L2 twice, "
+                   "so every stage starts cold") if cold else "inputs smaller than L2: stages run warm",
+            "parallelism": "replicas only (no cross-GPU step on this path)"}
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w, x_bits = cpu_sample(args.config, args.cpu_sample_tokens or 8192)
-    for _ in range(max(0, min(args.warmup, 1))):
+    full_T = args.tokens or _default_T(args.config)
+    w, x_bits = cpu_sample(args.config, min(args.cpu_sample_tokens or CPU_SAMPLE_TOKENS, full_T), args.hidden)
+    budget_s = 150.0
+    t_begin = time.perf_counter()
+    warm = 0
+    for _ in range(max(0, args.warmup)):
         oracle_step(w, x_bits)
-    budget_s = 120.0
+        warm += 1
+        if time.perf_counter() - t_begin > budget_s / 2:
+            break
     times = []
     for _ in range(max(1, args.steps)):
         times.append(oracle_step(w, x_bits))
-        if sum(times) > budget_s:
+        if time.perf_counter() - t_begin > budget_s:
             break
     sec = sum(times) / len(times)
     value = w.P / sec
-    name = workload_name(w, T=args.tokens or _default_T(args.config))
-    sample = f"first {w.T} tokens of the workload ({w.P} pairs), all four stages, single thread"
+    sample = cpu_sample_text(w, f", mean of {len(times)} runs, {sec:.2f} s each")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": name, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "steps": len(times), "warmup": warm, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "dtype_detail": "bf16 rows moved bit-exactly, fp32 accumulation in the combine, u32 counts, i32 indices",
+        "data": "synthetic", "config": config_dict(full_T, w),
+        "cpu_baseline": dict({"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+                             **host_description()),
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -145,45 +215,96 @@ def _default_T(config):
 # clocks
 # ---------------------------------------------------------------------------------------------
 class ClockSampler:
+    """SM clock, power and throttle reasons of one GPU, sampled while the timed region runs: through
+    NVML from a thread every few milliseconds (reads only), or, without the NVML module, from an
+    nvidia-smi loop."""
     QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
     NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+    PERIOD_S = 0.008
 
     def __init__(self, device_id):
         self.proc = None
-        self.device_index = device_id      # an index or a "GPU-<uuid>" string
+        self.thread = None
+        self.rows = []                      # (epoch seconds, sm MHz, max sm MHz, watts, [reason strings])
+        self.device_index = device_id       # an index or a "GPU-<uuid>" string
+        self.how = None
+
+    def _nvml_loop(self, handle, nv):
+        bits = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        try:
+            max_sm = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+        except Exception:
+            max_sm = float("nan")
+        n_taken, watts = 0, float("nan")
+        while not self._stop:
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM))
+                reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(handle))
+                n_taken += 1
+                if n_taken % 8 == 1:                       # the power reading is the slow one
+                    watts = nv.nvmlDeviceGetPowerUsage(handle) / 1000.0
+                self.rows.append((time.time(), sm, max_sm, watts,
+                                  ["Active" if reasons & bits[n] else "Not Active" for n in self.NAMES]))
+            except Exception:
+                pass
+            time.sleep(self.PERIOD_S)
 
     def start(self):
         try:
+            import threading
+
+            import pynvml as nv
+            nv.nvmlInit()
+            dev = str(self.device_index)
+            handle = nv.nvmlDeviceGetHandleByUUID(dev) if dev.startswith("GPU-") else nv.nvmlDeviceGetHandleByIndex(int(dev))
+            self._stop = False
+            self.thread = threading.Thread(target=self._nvml_loop, args=(handle, nv), daemon=True)
+            self.thread.start()
+            self.how = f"NVML every {self.PERIOD_S * 1e3:.0f} ms"
+            return
+        except Exception:
+            self.thread = None
+        try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.device_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.how = "nvidia-smi every 20 ms"
         except Exception:
             self.proc = None
 
     def stop(self, t_begin=None, t_end=None):
         """Median SM clock and throttle reasons over the samples taken inside [t_begin, t_end]
         (wall-clock seconds since the epoch); all samples if no window is given or none fall in it."""
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        time.sleep(0.1)
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except Exception:
-            self.proc.kill()
-            out = ""
         rows = []
-        for line in out.splitlines():
-            f = [v.strip() for v in line.split(",")]
-            if len(f) < 8:
-                continue
+        if self.thread is not None:
+            time.sleep(0.02)
+            self._stop = True
+            self.thread.join(timeout=2)
+            rows = list(self.rows)
+        elif self.proc is not None:
+            time.sleep(0.1)
+            self.proc.terminate()
             try:
-                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[4:8]))
-            except ValueError:
-                continue
+                out, _ = self.proc.communicate(timeout=5)
+            except Exception:
+                self.proc.kill()
+                out = ""
+            for line in out.splitlines():
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[1]), float(f[2]), float(f[3]), f[4:8]))
+                except ValueError:
+                    continue
+        else:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
         window = "timed region" if inside else "whole run (no sample fell inside the timed region)"
         use = inside or rows
@@ -193,9 +314,24 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(r[1] for r in use) if use else None,
+                "sm_min_mhz": min(r[1] for r in use) if use else None,
                 "sm_max_mhz": max(r[2] for r in use) if use else None,
-                "power_w_max": max(r[3] for r in use) if use else None,
-                "reasons": sorted(reasons), "samples": len(use), "window": window}
+                "power_w_max": max((r[3] for r in use if r[3] == r[3]), default=None),
+                "reasons": sorted(reasons), "samples": len(use), "window": window, "sampler": self.how}
+
+
+def host_description():
+    """The host the CPU oracle is timed on: logical CPUs, model name, the threads the oracle uses."""
+    model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model, "threads_used": 1}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -309,6 +445,22 @@ def extra_measurements(args, w, step, cb, torch):
     except Exception as exc:
         out["timing_floor_us"] = None
         out["timing_floor_error"] = str(exc)[:200]
+
+    # What binds the statistics and the assignment is not HBM: the rate of shared-memory atomic adds and
+    # of instruction issue, measured here on this device by the measurement kernels of cobalt_peaks.h
+    try:
+        from paper_2609_36959_b200 import peaks
+        out["sm_peaks"] = {
+            "shared_atomic_adds_per_clk_sm_conflict_free": peaks.shared_atomics_conflict_free(),
+            "shared_atomic_adds_per_clk_sm_stats_pattern": (peaks.shared_atomics_stats_pattern(step.topk_ids, w.E)
+                                                            if w.K in (1, 2, 4, 6, 8) and w.E <= 600 else None),
+            "warp_instructions_per_clk_sm": peaks.issue_rate(0),
+            "warp_instructions_per_clk_sm_hash_mix": peaks.issue_rate(1),
+            "how": "one CTA of 1024 threads per SM, SM cycle counter over the slowest CTA, warm; "
+                   "stats pattern = the K(K+1)/2 adds per token of this workload's ids into the 16-bit triangle, nothing else",
+        }
+    except Exception as exc:
+        out["sm_peaks"] = {"error": str(exc)[:200]}
 
     # the same step with stages 1, 2 and the permutation index fused into one pass over the ids
     try:
@@ -532,7 +684,8 @@ def run_cobalt(args):
     except Exception:
         gpu_id = local_rank
     sampler = ClockSampler(gpu_id)
-    if rank == 0:
+    sampler.PERIOD_S = args.clock_period_ms * 1e-3
+    if rank == 0 and args.clock_period_ms > 0:
         sampler.start()
     for _ in range(max(3, args.warmup)):
         one_step()
@@ -597,12 +750,40 @@ def run_cobalt(args):
                          "frac_of_same_run_copy": (gbs / extras["same_run_copy_gbs"]
                                                    if extras.get("same_run_copy_gbs") else None),
                          "pairs_per_s": w.P / (stage_ms[n] * 1e-3)}
+        # second roofline of the two small stages: the SM resource that binds them
+        pk = extras.get("sm_peaks") or {}
+        counters = load_json(COUNTERS_JSON).get(f"config{w.name}", {}) if w.T == _default_T(w.name) else {}
+        n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        sm_hz = (clocks.get("sm_mhz") or 1965.0) * 1e6 if clocks else 1965.0e6
+        if pk.get("shared_atomic_adds_per_clk_sm_conflict_free"):
+            adds = w.T * w.K * (w.K + 1) // 2
+            rate = adds / (stage_ms["coact_stats"] * 1e-3 * sm_hz * n_sm)
+            stages["coact_stats"]["second_bound"] = {
+                "bound": "shared-memory atomic adds", "adds": adds, "unit": "adds per clock per SM", "achieved": rate,
+                "peak_conflict_free": pk["shared_atomic_adds_per_clk_sm_conflict_free"],
+                "frac_of_conflict_free": rate / pk["shared_atomic_adds_per_clk_sm_conflict_free"],
+                "peak_this_pattern": pk.get("shared_atomic_adds_per_clk_sm_stats_pattern"),
+                "frac_of_this_pattern": (rate / pk["shared_atomic_adds_per_clk_sm_stats_pattern"]
+                                         if pk.get("shared_atomic_adds_per_clk_sm_stats_pattern") else None),
+                "note": "whole stage (clearing kernel, launch, merge) against the adds alone"}
+        instr = (counters.get("assign_kernel") or {}).get("warp_instructions")
+        if pk.get("warp_instructions_per_clk_sm") and instr:
+            rate = instr / (stage_ms["assign"] * 1e-3 * sm_hz * n_sm)
+            stages["assign"]["second_bound"] = {
+                "bound": "instruction issue", "warp_instructions": instr, "unit": "warp instructions per clock per SM",
+                "achieved": rate, "peak": pk["warp_instructions_per_clk_sm"], "frac": rate / pk["warp_instructions_per_clk_sm"],
+                "note": "instruction count from the ncu capture in profiles/index_kernels_counters.json; whole stage "
+                        "(clearing kernel, launch) against issue alone"}
         dom = max(("permute_rows", "combine"), key=lambda n: stage_ms[n])
-        # the ncu capture was taken on this shape (H=7168, K=8); traffic scales with the pairs
-        traffic = NCU_TRAFFIC_BYTES_PER_PAIR.get(dom) if (w.H, w.K) == (7168, 8) else None
+        # DRAM bytes per pair from the ncu capture of a reduced token count on this row shape
+        # (profiles/row_kernels_traffic.json); traffic grows in proportion to the pairs of a launch
+        captured = load_json(TRAFFIC_JSON).get(dom, {})
+        traffic = captured.get("bytes_per_pair") if (captured.get("H"), captured.get("K")) == (w.H, w.K) else None
         roofline = {"bound": "hbm", "kernel": dom, "achieved": stages[dom]["gbs"], "peak": peak,
                     "unit": "GB/s", "frac": stages[dom]["frac"], "peak_source": peak_src,
                     "traffic": None if traffic is None else traffic * w.P,
+                    "traffic_source": None if traffic is None else
+                    f"ncu dram__bytes_read+write per pair at T={captured.get('captured_tokens')}, scaled to {w.P} pairs",
                     "algorithmic_bytes": sb[dom], "ms_per_launch": stage_ms[dom]}
         totals = step.totals.cpu().tolist()
         load = step.slot_load.cpu().numpy().astype(np.int64).reshape(w.G, w.S).sum(axis=1)
@@ -612,11 +793,7 @@ def run_cobalt(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "dtype_detail": "bf16 rows moved bit-exactly, fp32 accumulation in the combine, u32 counts, i32 indices",
             "data": "synthetic",
-            "config": {"workload": workload_name(w), "seed": int(w.seed),
-                       "l2": "no explicit flush: each step streams the 15 GB send buffer through L2 twice, "
-                             "so every stage starts cold" if w.P * w.H * 2 > (1 << 28) else
-                             "inputs smaller than L2: stages run warm",
-                       "parallelism": "replicas only (no cross-GPU step on this path)"},
+            "config": config_dict(w.T, w),
             "e2e": e2e, "gpu_launches": kernels_per_step(w.T) * args.steps,
             "roofline": roofline, "stages": stages, "clocks": clocks,
             "traffic_model": {"V_cobalt": totals[0], "V_naive": totals[1],
@@ -627,18 +804,89 @@ def run_cobalt(args):
             "device_error_bits": err_bits, "wall_s_timed_region": t_wall, "extras": extras,
         }
         if not args.no_cpu_baseline and world == 1:
-            ws, xs = cpu_sample(args.config, min(args.cpu_sample_tokens or 32768, w.T))
-            sec = min(oracle_step(ws, xs), oracle_step(ws, xs))
-            line["cpu_baseline"] = {"value": ws.P / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": f"first {ws.T} tokens of the workload ({ws.P} pairs), all four "
-                                              f"stages, single thread, best of 2 runs, {sec:.2f} s each"}
+            ws, xs = cpu_sample(args.config, min(args.cpu_sample_tokens or CPU_SAMPLE_TOKENS, w.T), args.hidden)
+            runs = [oracle_step(ws, xs) for _ in range(3)]
+            sec = min(runs[1:])                      # the first run warms the page cache and the allocator
+            line["cpu_baseline"] = dict({"value": ws.P / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                         "sample": cpu_sample_text(ws, f", best of 2 runs after one warm-up, {sec:.2f} s each")},
+                                        **host_description())
         print(json.dumps(line))
     if distributed:
         dist.destroy_process_group()
 
 
+def counters_from_ncu_csv(csv_path, config, command):
+    """Turns `ncu -i <report> --page raw --csv` of the index kernels (full token count, tiny rows) into
+    profiles/index_kernels_counters.json: warp instructions, shared-memory atomics and their wavefronts,
+    kernel time."""
+    import csv
+    import re
+    with open(csv_path) as f:
+        rows = list(csv.reader(f))
+    hdr = rows[0]
+    out = load_json(COUNTERS_JSON)
+    entry = out.setdefault(f"config{config}", {})
+    want = {"smsp__inst_executed.sum": "warp_instructions", "smsp__thread_inst_executed.sum": "thread_instructions",
+            "smsp__inst_executed_op_shared_atom.sum": "shared_atomic_instructions",
+            "l1tex__data_pipe_lsu_wavefronts_mem_shared_op_atom.sum": "shared_atomic_wavefronts",
+            "l1tex__data_pipe_lsu_wavefronts_mem_shared.sum": "shared_wavefronts",
+            "gpu__time_duration.sum": "time_under_ncu", "launch__grid_size": "grid", "launch__block_size": "block",
+            "launch__registers_per_thread": "registers", "sm__cycles_active.avg": "sm_cycles_active_avg"}
+    for r in rows[2:]:
+        d = dict(zip(hdr, r))
+        name = re.sub(r"^void ", "", d.get("Kernel Name", "")).split("(")[0]
+        short = name.split("<")[0]
+        rec = {"kernel": name, "command": command}
+        for metric, key in want.items():
+            if metric in d and d[metric] not in ("", "nan"):
+                rec[key] = float(d[metric])
+                if metric == "gpu__time_duration.sum":
+                    rec["time_unit"] = rows[1][hdr.index(metric)]
+        entry[short] = rec
+    with open(COUNTERS_JSON, "w") as f:
+        json.dump(out, f, indent=1, sort_keys=True)
+        f.write("\n")
+    return entry
+
+
+def summarise(paths):
+    """Markdown table of benchmark lines written earlier (one file per config)."""
+    rows = []
+    for path in paths:
+        with open(path) as f:
+            d = json.loads(f.read().strip().splitlines()[-1])
+        st, ex, tm = d["stages"], d.get("extras") or {}, d["traffic_model"]
+        e2e = d.get("e2e") or {}
+        rows.append("| {} | {} | {} | {} | {} | {} | {:.3f} | {:.1f} | {} | {:.1f} | {} | {:.1f} % | {:.2f} | {} |".format(
+            d["config"]["workload"].split(":")[0].replace("config ", ""),
+            *("{:.1f} ({:.1f} %)".format(st[n]["ms"] * 1e3, 100 * st[n]["frac"]) for n in
+              ("coact_stats", "assign", "permute_index", "permute_rows", "combine")),
+            d["ms_per_step"], d["value"] / 1e6,
+            "{:.1f}".format(ex["fused_route_index_us"]) if ex.get("fused_route_index_us") else "-",
+            (e2e.get("ms_per_step") or float("nan")), "{:.1f}".format(e2e["value"] / 1e6) if e2e.get("value") else "-",
+            100 * (tm["cross_node_reduction"] or 0.0), tm["rank_load_imbalance"] or float("nan"),
+            "{:.0f}".format(d["clocks"]["sm_mhz"]) if d.get("clocks") and d["clocks"].get("sm_mhz") else "-"))
+    print("| config | coact_stats us (of HBM peak) | assign us | permute_index us | permute_rows us | combine us | step ms | "
+          "M pairs/s | fused index pass us | e2e ms | e2e M pairs/s | cross-node reduction | rank-load imbalance | SM MHz |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(r)
+
+
 def main():
     args = parse_args()
+    if args.summarise:
+        summarise(args.summarise)
+        return
+    if args.counters_from:
+        print(json.dumps(counters_from_ncu_csv(args.counters_from, args.config, args.traffic_command)))
+        return
+    if args.traffic_from:
+        import workloads as W
+        w = W.make_config(args.config, T=16)
+        tokens = args.tokens or _default_T(args.config)
+        print(json.dumps(traffic_from_ncu_csv(args.traffic_from, tokens, w.K, args.hidden or w.H, args.traffic_command)))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -11,6 +11,8 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libcobalt.so")
+PEAKS_SRC = os.path.join(PKG, "peaks", "peaks.cu")
+PEAKS_LIB = os.path.join(PKG, "libcobalt_peaks.so")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -29,7 +31,23 @@ def _newest_dep() -> float:
     return max(os.path.getmtime(p) for p in deps)
 
 
+def build_peaks(force: bool = False) -> str:
+    """The measurement kernels the benchmark uses (shared-atomic and issue rates): a library of their own."""
+    deps = [PEAKS_SRC, os.path.join(ROOT, "include", "cobalt_peaks.h"), os.path.abspath(__file__)]
+    if not force and os.path.exists(PEAKS_LIB) and os.path.getmtime(PEAKS_LIB) >= max(os.path.getmtime(p) for p in deps):
+        return PEAKS_LIB
+    nvcc = os.environ.get("NVCC", "nvcc")
+    cmd = [nvcc, *NVCC_FLAGS, "-shared", "-o", PEAKS_LIB + ".tmp", PEAKS_SRC]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError(f"nvcc failed for {PEAKS_SRC}")
+    os.replace(PEAKS_LIB + ".tmp", PEAKS_LIB)
+    return PEAKS_LIB
+
+
 def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
+    build_peaks(force)
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_dep():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")

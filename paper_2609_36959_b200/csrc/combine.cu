@@ -14,18 +14,6 @@ namespace cobalt {
 
 constexpr int kCombineThreads = 256;
 
-// Threads of a one-token-per-CTA row kernel: whole warps, at most kCombineThreads, and as few as
-// keep the number of passes over the row's 16-byte vectors (H = 7168: 896 vectors, four passes of
-// 224 threads instead of three and a half of 256, so no pass runs half empty).
-static inline int row_kernel_threads(int n_vec)
-{
-    const int passes = (n_vec + kCombineThreads - 1) / kCombineThreads;
-    int threads = ((n_vec + passes - 1) / passes + 31) / 32 * 32;
-    if (threads < 32) threads = 32;
-    if (threads > kCombineThreads) threads = kCombineThreads;
-    return threads;
-}
-
 __device__ __forceinline__ void fma_bf16x2(float& a0, float& a1, uint32_t packed, float w)
 {
     a0 = fmaf(w, __uint_as_float(packed << 16), a0);
@@ -168,11 +156,9 @@ combine_backward_kernel(const uint4* __restrict__ grad_y, const uint4* __restric
         }
         __syncthreads();
         if (threadIdx.x < K) {
-            const int n_warps = blockDim.x >> 5;
             float d = 0.0f;
 #pragma unroll
-            for (int wi = 0; wi < kWarps; ++wi)
-                if (wi < n_warps) d += partial[wi][threadIdx.x];
+            for (int wi = 0; wi < kWarps; ++wi) d += partial[wi][threadIdx.x];
             grad_w[t * K + threadIdx.x] = d;
         }
     }
@@ -206,16 +192,15 @@ static int launch_combine(const void* expert_out, const int32_t* row_of_pair, co
     // one CTA per token: the block scheduler overlaps the per-token index loads of one CTA with
     // the row streaming of the others (measured faster than a persistent grid-stride grid)
     const unsigned grid = static_cast<unsigned>(T < 0x7FFFFFFFll ? T : 0x7FFFFFFFll);
-    const int threads = row_kernel_threads(n_vec);
     const uint4* src = static_cast<const uint4*>(expert_out);
     uint4* dst = static_cast<uint4*>(y);
 #define COBALT_COMBINE_CASE(KT)                                                                         \
     case KT:                                                                                            \
         if (gate_w)                                                                                     \
-            combine_kernel<KT, false><<<grid, threads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, \
+            combine_kernel<KT, false><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst, \
                                                                        err_word);                       \
         else                                                                                            \
-            combine_kernel<KT, true><<<grid, threads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,  \
+            combine_kernel<KT, true><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,  \
                                                                       err_word);                        \
         break
     switch (K) {
@@ -229,10 +214,10 @@ static int launch_combine(const void* expert_out, const int32_t* row_of_pair, co
         COBALT_COMBINE_CASE(16);
         default:
             if (gate_w)
-                combine_kernel<0, false><<<grid, threads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
+                combine_kernel<0, false><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
                                                                           err_word);
             else
-                combine_kernel<0, true><<<grid, threads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
+                combine_kernel<0, true><<<grid, kCombineThreads, 0, s>>>(src, row_of_pair, gate_w, T, K, n_vec, P, dst,
                                                                          err_word);
     }
 #undef COBALT_COMBINE_CASE
@@ -290,13 +275,12 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
     const int n_vec = H / 8;
     const int64_t P = T * K;
     const unsigned grid = static_cast<unsigned>(T);
-    const int threads = row_kernel_threads(n_vec);
     const uint4* gy = static_cast<const uint4*>(grad_y);
     const uint4* out = static_cast<const uint4*>(expert_out);
     uint4* go = static_cast<uint4*>(grad_expert_out);
 #define COBALT_CBWD_CASE(KT)                                                                                   \
     case KT:                                                                                                   \
-        combine_backward_kernel<KT><<<grid, threads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go, \
+        combine_backward_kernel<KT><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go, \
                                                                      grad_gate_w, err_word);                   \
         break
     switch (K) {
@@ -309,7 +293,7 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
         COBALT_CBWD_CASE(12);
         COBALT_CBWD_CASE(16);
         default:
-            combine_backward_kernel<0><<<grid, threads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go,
+            combine_backward_kernel<0><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go,
                                                                         grad_gate_w, err_word);
     }
 #undef COBALT_CBWD_CASE

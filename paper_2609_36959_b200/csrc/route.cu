@@ -48,7 +48,7 @@ struct RouteSmem {
     size_t tab_words;     // layout tables
     size_t dest_words;    // D rounded up to a multiple of 8
     size_t lane_stride;   // entries per warp of the lane-mask table: D rounded up to an odd number
-    // tri | stage | tab | cnt[dest] | base[dest] | excl[dest] | wm[warps][lane_stride] (two words each)
+    // tri | stage | tab | cnt[dest] | base[dest] | excl[dest] | mask[warps][lane_stride] | pre[warps][lane_stride]
     size_t words() const { return tri_words + stage_words + tab_words + 3 * dest_words + 2 * kRouteWarps * lane_stride; }
     size_t bytes() const { return words() * sizeof(uint32_t); }
 };
@@ -215,8 +215,8 @@ route_fused_kernel(const RouteParams p)
     uint32_t* cnt = tab + p.tab_words;                         // [D] pairs of this CTA (round) per destination
     uint32_t* base = cnt + p.dest_words;                       // [D] first row of this CTA's (round's) pairs inside d
     uint32_t* excl = base + p.dest_words;                      // [D] pairs of this round in lower destinations
-    uint2* wm = reinterpret_cast<uint2*>(excl + p.dest_words); // [warps][lane_stride] x: lanes (tokens) of the warp that
-                                                               //   send to d, y: the round's pairs to d in lower warps
+    uint32_t* mask = excl + p.dest_words;                      // [warps][lane_stride] lanes (tokens) of the warp that send to d
+    uint32_t* pre = mask + kRouteWarps * p.lane_stride;        // [warps][lane_stride] the round's pairs to d in lower warps
     __shared__ unsigned long long cta_totals[2];
     __shared__ uint32_t warp_sums[kRouteWarps];
 
@@ -226,7 +226,8 @@ route_fused_kernel(const RouteParams p)
     const int dest_words = p.dest_words;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = static_cast<int>(blockIdx.x), n_ctas = static_cast<int>(gridDim.x);
-    uint2* my_wm = wm + warp * p.lane_stride;
+    uint32_t* my_mask = mask + warp * p.lane_stride;
+    const uint32_t* my_pre = pre + warp * p.lane_stride;
     const uint32_t lower_lanes = (1u << lane) - 1u;
 
     uint32_t seed_lo = p.seed_lo, seed_hi = p.seed_hi;
@@ -266,7 +267,7 @@ route_fused_kernel(const RouteParams p)
     }
     for (int i = tid; i < p.tri_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < dest_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(cnt)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < kRouteWarps * p.lane_stride; i += kRouteThreads) wm[i] = make_uint2(0, 0);
+    for (int i = tid; i < kRouteWarps * p.lane_stride; i += kRouteThreads) mask[i] = 0;
     if (tid < 2) cta_totals[tid] = 0;
     const TableView tv = table_view(p.lv, tab);
     asm volatile("cp.async.wait_all;" ::: "memory");      // the tables have arrived behind the clearing
@@ -303,7 +304,7 @@ route_fused_kernel(const RouteParams p)
                 if (single) {
 #pragma unroll
                     for (int a = 0; a < KMAX; ++a)
-                        if (a < K) atomicOr(&my_wm[out[a]].x, 1u << lane);
+                        if (a < K) atomicOr(&my_mask[out[a]], 1u << lane);
                 } else {
 #pragma unroll
                     for (int a = 0; a < KMAX; ++a)
@@ -340,8 +341,8 @@ route_fused_kernel(const RouteParams p)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
-                const uint32_t ca = (da < D) ? __popc(wm[lane * p.lane_stride + da].x) : 0u;
-                const uint32_t cb = (db < D) ? __popc(wm[lane * p.lane_stride + db].x) : 0u;
+                const uint32_t ca = (da < D) ? __popc(mask[lane * p.lane_stride + da]) : 0u;
+                const uint32_t cb = (db < D) ? __popc(mask[lane * p.lane_stride + db]) : 0u;
                 c[h] = ca | (cb << 16);
                 incl[h] = c[h];
             }
@@ -358,11 +359,11 @@ route_fused_kernel(const RouteParams p)
                 const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
                 const uint32_t before = incl[h] - c[h];
                 if (da < D) {
-                    wm[lane * p.lane_stride + da].y = before & 0xFFFFu;
+                    pre[lane * p.lane_stride + da] = before & 0xFFFFu;
                     if (lane == 31) cnt[da] = incl[h] & 0xFFFFu;
                 }
                 if (db < D) {
-                    wm[lane * p.lane_stride + db].y = before >> 16;
+                    pre[lane * p.lane_stride + db] = before >> 16;
                     if (lane == 31) cnt[db] = incl[h] >> 16;
                 }
             }
@@ -377,8 +378,7 @@ route_fused_kernel(const RouteParams p)
         for (int a = 0; a < KMAX; ++a) {
             if (a < K && out[a] >= 0) {
                 const uint32_t d = static_cast<uint32_t>(out[a]);
-                const uint2 v = my_wm[d];
-                const uint32_t r = v.y + __popc(v.x & lower_lanes);
+                const uint32_t r = my_pre[d] + __popc(my_mask[d] & lower_lanes);
                 if (p.pair_of_row) stage[excl[d] + r] = d | (static_cast<uint32_t>(tid * K + a) << kDestBits);
                 out[a] = static_cast<int32_t>(d | (r << kDestBits));
             }
@@ -605,7 +605,7 @@ route_fused_kernel(const RouteParams p)
             }
 #pragma unroll
             for (int a = 0; a < KMAX; ++a)
-                if (a < K && out[a] >= 0) atomicOr(&my_wm[out[a]].x, 1u << lane);
+                if (a < K && out[a] >= 0) atomicOr(&my_mask[out[a]], 1u << lane);
         }
         __syncthreads();
         count_round();
@@ -624,7 +624,7 @@ route_fused_kernel(const RouteParams p)
         __syncthreads();
 #pragma unroll
         for (int a = 0; a < KMAX; ++a)
-            if (touched[a] != 0xFFFFFFFFu) my_wm[touched[a]].x = 0;
+            if (touched[a] != 0xFFFFFFFFu) my_mask[touched[a]] = 0;
         if (tid < D) base[tid] += round_total;
         __syncthreads();
     }

@@ -47,6 +47,19 @@ def test_library_exports_nothing_beyond_the_header(lib_path):
     assert exported == declared_symbols()
 
 
+def test_measurement_library_exports_its_header():
+    """libcobalt_peaks.so (the benchmark's measurement kernels) exports exactly what cobalt_peaks.h declares."""
+    import subprocess
+    from paper_2609_36959_b200 import build, peaks
+    lib = build.build_peaks()
+    with open(os.path.join(ROOT, "include", "cobalt_peaks.h")) as f:
+        declared = sorted(set(re.findall(r"\b(cobalt_[a-z_0-9]+)\s*\(", f.read())))
+    out = subprocess.run(["nm", "-D", "--defined-only", lib], capture_output=True, text=True, check=True).stdout
+    exported = sorted({line.split()[-1] for line in out.splitlines()
+                       if line.split() and line.split()[-1].startswith("cobalt_") and " T " in line})
+    assert exported == declared == sorted(peaks.EXPORTS)
+
+
 def test_version_and_status_strings(cb):
     assert cb.version() == 100
     seen = {cb.status_string(s) for s in (0, -1, -2, -3, -4, -5, -6)}
