@@ -31,13 +31,14 @@ if ROOT not in sys.path:
 METRIC = "routed token-expert pairs/sec"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
-KERNELS_PER_STEP = 9               # stats 2 (clear + tile), assign 2 (clear + assign), permute 4 (hist, scan, rank, rows), combine 1
-
-
-def kernels_per_step(T):
-    """Launches of one four-stage step: the statistics of a batch that fits a single cluster
-    (at most 16 CTAs of 256 tokens) store their sums and need no clearing kernel."""
-    return KERNELS_PER_STEP - (1 if 0 < T <= 4096 else 0)
+def kernels_per_step(T, fused):
+    """Launches of one step.  Fused: the index kernel, the row mover, the combine.  Four separate calls:
+    stats 2 (clear + tile), assign 2 (clear + assign), permute 4 (hist, scan, rank, rows), combine 1; the
+    statistics of a batch that fits a single cluster (at most 16 CTAs of 256 tokens) store their sums and
+    need no clearing kernel."""
+    if fused:
+        return 3
+    return 9 - (1 if 0 < T <= 4096 else 0)
 
 TRAFFIC_JSON = os.path.join(ROOT, "profiles", "row_kernels_traffic.json")
 COUNTERS_JSON = os.path.join(ROOT, "profiles", "index_kernels_counters.json")
@@ -82,6 +83,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="5")
+    ap.add_argument("--step", default="fused", choices=["fused", "separate"],
+                    help="the timed step: cobalt_route_index + cobalt_permute_rows + cobalt_combine (three kernels, "
+                         "default) or the four stages as separate calls (nine kernels); same outputs either way, and "
+                         "the other form is timed beside it")
     ap.add_argument("--tokens", type=int, default=None, help="override T (reduced-size runs for profiling)")
     ap.add_argument("--hidden", type=int, default=None, help="override H (tiny rows isolate the index stages)")
     ap.add_argument("--impl", default="cobalt", choices=["cobalt", "reference"])
@@ -117,6 +122,8 @@ def stage_bytes(w):
         "coact_stats": 4 * P + 4 * E * E + 4 * E,
         "assign": 4 * P + 4 * T + 4 * P + 4 * D + T,
         "permute_index": 4 * P + 4 * P + 4 * P + 4 * (2 * D + 1),
+        # one pass: ids and source ranks in; slots, both maps, remote_nodes, coact, load, counts and offsets out
+        "route_index": 4 * P + 4 * T + 4 * P + 4 * P + 4 * P + T + 4 * E * E + 4 * E + 4 * (2 * D + 1),
         "permute_rows": 2 * T * H + 2 * P * H + 4 * P,
         "combine": 2 * P * H + 2 * T * H + 4 * P + 4 * P,
     }
@@ -660,8 +667,11 @@ def run_cobalt(args):
     torch.cuda.synchronize()
 
     names = ["coact_stats", "assign", "permute_index", "permute_rows", "combine"]
+    fused_names = ["route_index", "permute_rows", "combine"]
 
-    def one_step(events=None):
+    def separate_step(events=None):
+        """The four stages as four calls (cobalt_permute split into its two halves so that the row mover is
+        timed on its own): nine kernels."""
         def mark(i):
             if events is not None:
                 events[i].record()
@@ -670,7 +680,6 @@ def run_cobalt(args):
         mark(1)
         step.assign(w.seed)
         mark(2)
-        # cobalt_permute is exactly these two calls; split so the row mover is timed on its own
         cb.permute_index(step.assigned_slot, w.D, step.dest_counts, step.dest_offsets, step.row_of_pair,
                          step.pair_of_row, step.workspace)
         mark(3)
@@ -678,6 +687,35 @@ def run_cobalt(args):
         mark(4)
         step.combine()
         mark(5)
+
+    def fused_step(events=None):
+        """The same outputs from three kernels: stages 1, 2 and the index half of 3 in one (cobalt_route_index)."""
+        def mark(i):
+            if events is not None:
+                events[i].record()
+        mark(0)
+        cb.route_index(step.layout, step.topk_ids, step.src_rank, w.seed, step.coact, step.load, step.assigned_slot,
+                       step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
+                       remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+        mark(1)
+        cb.permute_rows(step.x, step.row_of_pair, w.K, step.send)
+        mark(2)
+        step.combine()
+        mark(3)
+
+    headline_fused = args.step == "fused"
+    one_step = fused_step if headline_fused else separate_step
+    n_marks = 4 if headline_fused else 6
+
+    def timed_loop(fn, marks, n_steps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(marks)] for _ in range(n_steps)]
+        for i in range(n_steps):
+            fn(evs[i])
+        torch.cuda.synchronize()
+        return evs
 
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
@@ -690,7 +728,7 @@ def run_cobalt(args):
     for _ in range(max(3, args.warmup)):
         one_step()
     barrier()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(n_marks)] for _ in range(args.steps)]
     barrier()
     t_epoch0 = time.time()
     t_wall0 = time.perf_counter()
@@ -700,10 +738,24 @@ def run_cobalt(args):
     t_wall = time.perf_counter() - t_wall0
     clocks = sampler.stop(t_epoch0, t_epoch0 + t_wall) if rank == 0 else None
 
-    total_ms = ev[0][0].elapsed_time(ev[-1][5])
-    per_step = {n: [e[i].elapsed_time(e[i + 1]) for e in ev] for i, n in enumerate(names)}
-    stage_ms = {n: sum(v) / args.steps for n, v in per_step.items()}
+    total_ms = ev[0][0].elapsed_time(ev[-1][n_marks - 1])
+    head_names = fused_names if headline_fused else names
+    per_step = {n: [e[i].elapsed_time(e[i + 1]) for e in ev] for i, n in enumerate(head_names)}
     err_bits = cb.read_and_clear_device_error()
+    # the other form of the step, same number of steps, for the stages the headline loop does not separate
+    other_total_ms = None
+    if rank == 0 and not args.no_extras:
+        if headline_fused:
+            ev2 = timed_loop(separate_step, 6, args.steps)
+            other = {n: [e[i].elapsed_time(e[i + 1]) for e in ev2] for i, n in enumerate(names)}
+            other_total_ms = ev2[0][0].elapsed_time(ev2[-1][5]) / args.steps
+            for n in ("coact_stats", "assign", "permute_index"):
+                per_step[n] = other[n]
+        else:
+            ev2 = timed_loop(fused_step, 4, args.steps)
+            per_step["route_index"] = [e[0].elapsed_time(e[1]) for e in ev2]
+            other_total_ms = ev2[0][0].elapsed_time(ev2[-1][3]) / args.steps
+    stage_ms = {n: sum(v) / len(v) for n, v in per_step.items()}
 
     ms_per_step = max_over_ranks(total_ms, "cuda") / args.steps
     value = whole_job_value(world, w.P, ms_per_step)
@@ -742,7 +794,7 @@ def run_cobalt(args):
         peak, peak_src = hbm_peak()
         sb = stage_bytes(w)
         stages = {}
-        for n in names:
+        for n in [m for m in ["coact_stats", "assign", "permute_index", "route_index", "permute_rows", "combine"] if m in stage_ms]:
             gbs = sb[n] / (stage_ms[n] * 1e-3) / 1e9
             stages[n] = {"ms": stage_ms[n], "ms_median": statistics.median(per_step[n]), "ms_min": min(per_step[n]),
                          "bytes": sb[n], "gbs": gbs, "frac": gbs / peak,
@@ -794,13 +846,18 @@ def run_cobalt(args):
             "dtype_detail": "bf16 rows moved bit-exactly, fp32 accumulation in the combine, u32 counts, i32 indices",
             "data": "synthetic",
             "config": config_dict(w.T, w),
-            "e2e": e2e, "gpu_launches": kernels_per_step(w.T) * args.steps,
+            "step": ("cobalt_route_index (stages 1, 2 and the index half of 3 in one kernel) + cobalt_permute_rows + "
+                     "cobalt_combine; the four separate calls are timed beside it (stages, four_stage_step_ms)"
+                     if headline_fused else "cobalt_coact_stats + cobalt_assign + cobalt_permute + cobalt_combine"),
+            "e2e": e2e, "gpu_launches": kernels_per_step(w.T, headline_fused) * args.steps,
             "roofline": roofline, "stages": stages, "clocks": clocks,
             "traffic_model": {"V_cobalt": totals[0], "V_naive": totals[1],
                               "remote_nodes_per_token_cobalt": totals[0] / max(w.T, 1),
                               "remote_nodes_per_token_naive": totals[1] / max(w.T, 1),
                               "cross_node_reduction": (1 - totals[0] / totals[1]) if totals[1] else None,
                               "rank_load_imbalance": float(load.max() / load.mean()) if load.sum() else None},
+            "four_stage_step_ms": other_total_ms if headline_fused else ms_per_step,
+            "fused_step_ms": ms_per_step if headline_fused else other_total_ms,
             "device_error_bits": err_bits, "wall_s_timed_region": t_wall, "extras": extras,
         }
         if not args.no_cpu_baseline and world == 1:
