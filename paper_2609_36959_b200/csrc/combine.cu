@@ -164,6 +164,44 @@ combine_backward_kernel(const uint4* __restrict__ grad_y, const uint4* __restric
     }
 }
 
+// grad_expert_out alone (no gate-weight gradient wanted): one warp per (token, k).  The token's grad_y
+// row is staged in shared memory once, then warp k writes row r(t,k) of grad_expert_out from end to
+// end, so that every warp produces one long contiguous run instead of the K rows being interleaved
+// 512 bytes at a time (measured at T = 131072, K = 8, H = 7168: 2.63 ms against 2.81 ms).  With the dot
+// products in the same kernel the interleaved form above is the faster one (5.09 ms against 5.16 ms).
+__global__ void __launch_bounds__(kCombineThreads)
+combine_backward_scatter_kernel(const uint4* __restrict__ grad_y, const int32_t* __restrict__ row_of_pair,
+                                const float* __restrict__ gate_w, int64_t T, int K, int n_vec, int64_t P,
+                                uint4* __restrict__ grad_out, uint32_t* __restrict__ err_word)
+{
+    extern __shared__ __align__(16) uint4 g_row[];             // [n_vec] the token's grad_y row
+    constexpr int kWarps = kCombineThreads / 32;
+    const int64_t t = blockIdx.x;
+    if (t >= T) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int v = threadIdx.x; v < n_vec; v += kCombineThreads) g_row[v] = ld_stream16(grad_y + t * n_vec + v);
+    __syncthreads();
+    for (int k = warp; k < K; k += kWarps) {
+        const int32_t r = __ldg(row_of_pair + t * K + k);
+        if (r < 0 || r >= P) {
+            if (lane == 0) flag_error(err_word, COBALT_DEVERR_BAD_SLOT);
+            continue;
+        }
+        const float w = __ldg(gate_w + t * K + k);
+        uint4* dst = grad_out + static_cast<int64_t>(r) * n_vec;
+#pragma unroll 4
+        for (int v = lane; v < n_vec; v += 32) {
+            const uint4 g = g_row[v];
+            uint4 o;
+            o.x = pack_bf16x2(w * __uint_as_float(g.x << 16), w * __uint_as_float(g.x & 0xFFFF0000u));
+            o.y = pack_bf16x2(w * __uint_as_float(g.y << 16), w * __uint_as_float(g.y & 0xFFFF0000u));
+            o.z = pack_bf16x2(w * __uint_as_float(g.z << 16), w * __uint_as_float(g.z & 0xFFFF0000u));
+            o.w = pack_bf16x2(w * __uint_as_float(g.w << 16), w * __uint_as_float(g.w & 0xFFFF0000u));
+            st_stream16(dst + v, o);
+        }
+    }
+}
+
 // Argument checks and launch shared by the combine and by the backward of the dispatch gather.
 // gate_w == nullptr selects unit weights (the plain sum of the K rows); the public combine entries
 // reject it before they get here.
@@ -278,6 +316,14 @@ int cobalt_combine_backward(const void* grad_y, const void* expert_out, const in
     const uint4* gy = static_cast<const uint4*>(grad_y);
     const uint4* out = static_cast<const uint4*>(expert_out);
     uint4* go = static_cast<uint4*>(grad_expert_out);
+    if (!grad_gate_w && (flags & COBALT_IMPL_MASK) != COBALT_IMPL_VECTOR && static_cast<size_t>(n_vec) * sizeof(uint4) <= 96 * 1024) {
+        const size_t smem = sizeof(uint4) * static_cast<size_t>(n_vec);
+        int rc_attr = ensure_kernel_attributes(reinterpret_cast<const void*>(combine_backward_scatter_kernel), smem, false);
+        if (rc_attr != COBALT_OK) return rc_attr;
+        combine_backward_scatter_kernel<<<grid, kCombineThreads, smem, s>>>(gy, row_of_pair, gate_w, T, K, n_vec, P, go, err_word);
+        COBALT_CUDA_TRY(cudaGetLastError());
+        return COBALT_OK;
+    }
 #define COBALT_CBWD_CASE(KT)                                                                                   \
     case KT:                                                                                                   \
         combine_backward_kernel<KT><<<grid, kCombineThreads, 0, s>>>(gy, out, row_of_pair, gate_w, T, K, n_vec, P, go, \
