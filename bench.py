@@ -596,7 +596,7 @@ def extra_measurements(args, w, step, cb, torch):
         out["stage2_rebalance"] = {"error": str(exc)[:200]}
 
     # Eq. 1 under a layout that co-locates each co-activation cluster (what the paper's global
-    # planner aims for), same ids: reported as context, not judged
+    # planner aims for), same ids: reported as context
     try:
         import workloads as W
         wc = W.make_config(args.config, clustered=True, T=min(w.T, 32768))
