@@ -204,6 +204,37 @@ constexpr int kDestBits = 10;
 static_assert(kRouteMaxDests <= (1 << kDestBits), "destinations must fit the packed entry");
 static_assert(kRouteThreads * COBALT_MAX_TOPK <= (1 << (32 - kDestBits - 1)), "a round's pairs must fit the packed entry");
 
+// Barrier among the 512 threads of one half of the CTA (named barrier 1 for the lower half, 2 for the upper).
+__device__ __forceinline__ void half_barrier(int id)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kRouteThreads / 2) : "memory");
+}
+
+// Exclusive scan over d with two consecutive destinations per thread of the lower half (threads
+// 0 .. 511, D <= 1024); `before` receives the sum of the values below destination 2 * tid.  Uses half
+// barriers only.
+__device__ __forceinline__ uint32_t half_exclusive_scan2(uint32_t pair_sum, uint32_t* warp_sums, uint32_t* total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = pair_sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    half_barrier(1);
+    uint32_t before = incl - pair_sum, all = 0;
+#pragma unroll
+    for (int w = 0; w < kRouteWarps / 2; ++w) {
+        const uint32_t s = warp_sums[w];
+        if (w < warp) before += s;
+        all += s;
+    }
+    *total = all;
+    return before;
+}
+
 template <int KT, bool kPacked>
 __global__ void __launch_bounds__(kRouteThreads)
 route_fused_kernel(const RouteParams p)
@@ -407,13 +438,15 @@ route_fused_kernel(const RouteParams p)
         }
     };
 
-    if (single) count_round();               // cnt[d] from the lane masks
-    __syncthreads();
-
     // ---- publish this CTA's partial results ------------------------------------------------------
+    // The triangle goes first (9.7 MB over the grid: the stores drain while the counts are worked out).
     {
         uint4* dst = reinterpret_cast<uint4*>(p.ws_tri + static_cast<size_t>(cta) * p.tri_words);
         for (int v = tid; v < p.tri_words / 4; v += kRouteThreads) dst[v] = reinterpret_cast<const uint4*>(tri)[v];
+    }
+    if (single) count_round();               // cnt[d] from the lane masks
+    __syncthreads();
+    {
         uint32_t* dst_cnt = reinterpret_cast<uint32_t*>(p.ws_cnt + static_cast<size_t>(cta) * dest_words);
         for (int i = tid; i < dest_words / 2; i += kRouteThreads) dst_cnt[i] = cnt[2 * i] | (cnt[2 * i + 1] << 16);
         if (p.totals && tid < 2) p.ws_tot[2 * cta + tid] = cta_totals[tid];
@@ -539,42 +572,56 @@ route_fused_kernel(const RouteParams p)
             dst_lower[1] = make_uint4(lower[4], lower[5], lower[6], lower[7]);
         }
     }
-    __syncthreads();
-    // 2a: the sums of the slice go out to coact / load (plain stores unless accumulating)
-    for (int i = tid; i < n_acc; i += kRouteThreads) {
-        const int flat = 4 * v0 * kPerWord + i;
-        if (flat >= n_tri) continue;
-        const int hi = tri_row(flat), lo = flat - hi * (hi + 1) / 2;
-        const uint32_t v = acc[i];
-        if (p.accumulate) {
-            if (v) {
-                atomicAdd(&p.coact[static_cast<size_t>(hi) * E + lo], v);
-                if (lo != hi) atomicAdd(&p.coact[static_cast<size_t>(lo) * E + hi], v);
-                else atomicAdd(&p.load[hi], v);
+    // (the two halves go on separately: each only waits for its own half until the rows are written)
+    if (tid >= kHalf) {
+        half_barrier(2);
+        // 2a: the sums of the slice go out to coact / load (plain stores unless accumulating)
+        for (int i = tid - kHalf; i < n_acc; i += kHalf) {
+            const int flat = 4 * v0 * kPerWord + i;
+            if (flat >= n_tri) continue;
+            const int hi = tri_row(flat), lo = flat - hi * (hi + 1) / 2;
+            const uint32_t v = acc[i];
+            if (p.accumulate) {
+                if (v) {
+                    atomicAdd(&p.coact[static_cast<size_t>(hi) * E + lo], v);
+                    if (lo != hi) atomicAdd(&p.coact[static_cast<size_t>(lo) * E + hi], v);
+                    else atomicAdd(&p.load[hi], v);
+                }
+            } else {
+                p.coact[static_cast<size_t>(hi) * E + lo] = v;
+                if (lo != hi) p.coact[static_cast<size_t>(lo) * E + hi] = v;
+                else p.load[hi] = v;
             }
-        } else {
-            p.coact[static_cast<size_t>(hi) * E + lo] = v;
-            if (lo != hi) p.coact[static_cast<size_t>(lo) * E + hi] = v;
-            else p.load[hi] = v;
         }
-    }
-    {
-        // 2b: totals over all CTAs, their exclusive scan over d (the offsets), first row of this CTA
-        uint32_t mine = 0, lower = 0;
-        if (tid < D) {
-            for (int g = 0; g < parts; ++g) {
-                mine += part_all[g * dest_words + tid];
-                lower += part_lower[g * dest_words + tid];
+    } else {
+        half_barrier(1);
+        // 2b: totals over all CTAs, their exclusive scan over d (the offsets), first row of this CTA;
+        // two consecutive destinations per thread
+        uint32_t mine[2] = {0, 0}, lower[2] = {0, 0};
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int d = 2 * tid + j;
+            if (d < D) {
+                for (int g = 0; g < parts; ++g) {
+                    mine[j] += part_all[g * dest_words + d];
+                    lower[j] += part_lower[g * dest_words + d];
+                }
             }
         }
         uint32_t total = 0;
-        const uint32_t before = block_exclusive_scan(mine, warp_sums, &total);
-        if (tid < D) {
-            if (cta == 0) {
-                p.dest_counts[tid] = mine;
-                p.dest_offsets[tid] = before;
+        uint32_t before = half_exclusive_scan2(mine[0] + mine[1], warp_sums, &total);
+        half_barrier(1);                         // the part buffers have been read: base may be written (it can be one of them)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int d = 2 * tid + j;
+            if (d < D) {
+                if (cta == 0) {
+                    p.dest_counts[d] = mine[j];
+                    p.dest_offsets[d] = before;
+                }
+                base[d] = before + lower[j];
             }
-            base[tid] = before + lower;
+            before += mine[j];
         }
         if (cta == 0 && tid == 0) p.dest_offsets[D] = total;
     }
