@@ -58,7 +58,11 @@ extern "C" {
 #define COBALT_ERR_HOST_ALLOC (-6)           /* a host-side allocation failed (layout handle, planner scratch) */
 
 /* Supported envelope: N <= 8 nodes, Q <= 255 ranks per node, K <= 16, E <= 1024, D <= 4096,
- * P = T*K < 2^31, H a multiple of 8 (rows are whole 16-byte vectors). */
+ * P = T*K < 2^31, H a multiple of 8 (rows are whole 16-byte vectors).
+ * Every K from 1 to 16 gives the same results; the kernels of the separate stage calls are compiled with
+ * the K ids of a token in registers for K = 1, 2, 4, 6, 8, 10, 12, 16 and run a generic variant (loops
+ * to 16, a few microseconds slower per index stage) for the other K, while cobalt_route_index is compiled
+ * for every K. */
 #define COBALT_MAX_NODES 8
 #define COBALT_MAX_RANKS_PER_NODE 255
 #define COBALT_MAX_TOPK 16

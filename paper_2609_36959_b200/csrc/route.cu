@@ -98,22 +98,34 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 // bounded all the same, and a wait that runs out reports COBALT_DEVERR_WAIT_TIMEOUT and makes the
 // CTA return.  After the wait every CTA signs off on the same word and the last one clears it, so
 // that a replay of a captured launch (same epoch) starts from a word that differs from its epoch.
-// All three are called by all threads of the CTA.
+// Arrival and wait are separate calls (work that needs no other CTA goes in between); all are called by
+// all threads of the CTA.
 __device__ __forceinline__ void grid_barrier_init(unsigned long long* word, uint32_t epoch)
 {
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicExch(word, static_cast<unsigned long long>(epoch) << 32);
 }
 
-// Returns false on a timeout.
-__device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t epoch, uint32_t n_ctas,
-                                             uint32_t* err_word)
+// Arrival: the value the atomic returns is only looked at in grid_wait, so the arriving thread goes on
+// with whatever lies between the two calls while the atomic travels.
+__device__ __forceinline__ unsigned long long grid_arrive(unsigned long long* word)
 {
-    __shared__ int barrier_ok;
+    unsigned long long before = 0;
     __syncthreads();                       // this CTA's writes are done ...
     if (threadIdx.x == 0) {
         __threadfence();                   // ... and visible to the grid before the arrival is
+        before = atomicAdd(word, 1ull);
+    }
+    return before;
+}
+
+// Returns false on a timeout.  `before` is what grid_arrive returned.
+__device__ __forceinline__ bool grid_wait(unsigned long long* word, unsigned long long before, uint32_t epoch,
+                                          uint32_t n_ctas, uint32_t* err_word)
+{
+    __shared__ int barrier_ok;
+    if (threadIdx.x == 0) {
         const unsigned long long target = (static_cast<unsigned long long>(epoch) << 32) | n_ctas;
-        bool counted = (atomicAdd(word, 1ull) >> 32) == epoch;
+        bool counted = (before >> 32) == epoch;
         bool ok = false;
         for (uint32_t spin = 0; spin < kBarrierSpinLimit; ++spin) {
             const unsigned long long v = ld_acquire_u64(word);
@@ -131,8 +143,8 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* word, uint32_t 
         }
         if (ok) {
             // sign off; the last CTA to do so leaves the word cleared
-            const unsigned long long before = atomicAdd(word, 1ull);
-            if (static_cast<uint32_t>(before) + 1u == 2u * n_ctas) atomicExch(word, 0ull);
+            const unsigned long long old = atomicAdd(word, 1ull);
+            if (static_cast<uint32_t>(old) + 1u == 2u * n_ctas) atomicExch(word, 0ull);
         } else {
             flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
         }
@@ -298,7 +310,8 @@ route_fused_kernel(const RouteParams p)
     }
     for (int i = tid; i < p.tri_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(tri)[i] = make_uint4(0, 0, 0, 0);
     for (int i = tid; i < dest_words / 4; i += kRouteThreads) reinterpret_cast<uint4*>(cnt)[i] = make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < kRouteWarps * p.lane_stride; i += kRouteThreads) mask[i] = 0;
+    for (int i = tid; i < kRouteWarps * p.lane_stride / 4; i += kRouteThreads)      // 32 x stride words: whole vectors
+        reinterpret_cast<uint4*>(mask)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 2) cta_totals[tid] = 0;
     const TableView tv = table_view(p.lv, tab);
     asm volatile("cp.async.wait_all;" ::: "memory");      // the tables have arrived behind the clearing
@@ -451,7 +464,8 @@ route_fused_kernel(const RouteParams p)
         for (int i = tid; i < dest_words / 2; i += kRouteThreads) dst_cnt[i] = cnt[2 * i] | (cnt[2 * i + 1] << 16);
         if (p.totals && tid < 2) p.ws_tot[2 * cta + tid] = cta_totals[tid];
     }
-    // while those stores drain: what the ranks need from this CTA alone
+    const unsigned long long arrived = grid_arrive(p.barrier);
+    // between arrival and wait: what the ranks need from this CTA alone
     uint32_t round_pairs = 0;
     if (single) {
         const uint32_t lower_dests = block_exclusive_scan((tid < D) ? cnt[tid] : 0u, warp_sums, &round_pairs);
@@ -459,7 +473,7 @@ route_fused_kernel(const RouteParams p)
         __syncthreads();
         rank_round(t_lo + tid < t_hi);
     }
-    if (!grid_barrier(p.barrier, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word)) return;
+    if (!grid_wait(p.barrier, arrived, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word)) return;
 
     // ---- phase 2a and 2b side by side: both wait on loads of what the other CTAs published, so the
     // upper half of the CTA's warps sums this CTA's slice of the triangle over all partials (2a) while

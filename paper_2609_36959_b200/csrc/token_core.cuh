@@ -82,7 +82,8 @@ __device__ __forceinline__ void store_token_slots(int32_t* __restrict__ dst, con
 }
 
 // The K ids of a token in ascending order (a compare-exchange network, fully unrolled; entries past K
-// are padded with a value above every id so that they stay at the end).
+// are padded with a value above every id so that they stay at the end).  K = 8 takes the 19-exchange
+// network, the other sizes an odd-even transposition sort.
 template <int KT>
 __device__ __forceinline__ void sort_token_ids(const int32_t (&id)[TokenShape<KT>::KMAX], int K,
                                                int32_t (&s)[TokenShape<KT>::KMAX])
@@ -90,13 +91,21 @@ __device__ __forceinline__ void sort_token_ids(const int32_t (&id)[TokenShape<KT
     constexpr int KMAX = TokenShape<KT>::KMAX;
 #pragma unroll
     for (int a = 0; a < KMAX; ++a) s[a] = (a < K) ? id[a] : 0x7FFFFFFF;
+    auto exchange = [&](int a, int b) {
+        const int32_t lo = min(s[a], s[b]), hi = max(s[a], s[b]);
+        s[a] = lo;
+        s[b] = hi;
+    };
+    if (KT == 8) {
+        constexpr int net[19][2] = {{0, 1}, {2, 3}, {4, 5}, {6, 7}, {0, 2}, {1, 3}, {4, 6}, {5, 7}, {1, 2}, {5, 6},
+                                    {0, 4}, {3, 7}, {1, 5}, {2, 6}, {1, 4}, {3, 6}, {2, 4}, {3, 5}, {3, 4}};
 #pragma unroll
-    for (int pass = 0; pass < KMAX; ++pass) {
+        for (int i = 0; i < 19; ++i) exchange(net[i][0], net[i][1]);
+    } else {
 #pragma unroll
-        for (int a = pass & 1; a + 1 < KMAX; a += 2) {
-            const int32_t lo = min(s[a], s[a + 1]), hi = max(s[a], s[a + 1]);
-            s[a] = lo;
-            s[a + 1] = hi;
+        for (int pass = 0; pass < KMAX; ++pass) {
+#pragma unroll
+            for (int a = pass & 1; a + 1 < KMAX; a += 2) exchange(a, a + 1);
         }
     }
 }
