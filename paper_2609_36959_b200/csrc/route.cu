@@ -64,9 +64,13 @@ static RouteSmem route_smem(const LayoutView& lv, int K, bool packed)
     return r;
 }
 
+// Grid-wide sums kept in the workspace behind the destination totals, cleared with them: the two 64-bit
+// sums of Eq. 1 (V_cobalt, V_naive), as 32-bit words.
+constexpr int kGridSumWords = 4;
+
 // Workspace of the fused kernel (byte offsets, 256-byte aligned).
 struct RouteWorkspace {
-    size_t barrier_off, cnt_off, tot_off, tri_off, total;
+    size_t barrier_off, cnt_off, dtot_off, tri_off, total;
 };
 
 static RouteWorkspace route_workspace(const LayoutView& lv, bool packed)
@@ -76,7 +80,7 @@ static RouteWorkspace route_workspace(const LayoutView& lv, bool packed)
     size_t off = 0;
     w.barrier_off = off; off += 256;
     w.cnt_off = off;     off += round_up(sizeof(uint16_t) * kRouteMaxCtas * sm.dest_words, 256);
-    w.tot_off = off;     off += round_up(sizeof(unsigned long long) * 2 * kRouteMaxCtas, 256);
+    w.dtot_off = off;    off += round_up(sizeof(uint32_t) * (sm.dest_words + kGridSumWords), 256);
     w.tri_off = off;     off += round_up(sizeof(uint32_t) * kRouteMaxCtas * sm.tri_words, 256);
     w.total = off;
     return w;
@@ -90,19 +94,42 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 }
 
 // Grid-wide barrier on one 64-bit word of the workspace: epoch (high half) and arrival count.
-// The word may hold anything when the kernel starts.  CTA 0 sets it to (epoch, 0) first thing; a CTA
-// arrives by adding one and learns from the value it gets back whether the word already carried
-// this launch's epoch.  If not (it arrived before CTA 0's store landed: its increment is lost with
-// the old contents), it waits for the epoch to appear and adds again.  Every CTA of the grid is
+// The word may hold anything when the kernel starts.  CTA 0 sets it to (epoch, 0) once it has cleared
+// the grid-wide destination totals; a CTA adds to those totals only after it has seen the epoch
+// (grid_epoch_seen), so its additions cannot be lost to the clearing.  A CTA arrives by adding one and
+// learns from the value it gets back whether the word already carried this launch's epoch.  If not, it
+// waits for the epoch to appear and adds again.  Every CTA of the grid is
 // resident (cooperative launch), so the wait ends as soon as the slowest CTA has arrived; it is
 // bounded all the same, and a wait that runs out reports COBALT_DEVERR_WAIT_TIMEOUT and makes the
 // CTA return.  After the wait every CTA signs off on the same word and the last one clears it, so
 // that a replay of a captured launch (same epoch) starts from a word that differs from its epoch.
 // Arrival and wait are separate calls (work that needs no other CTA goes in between); all are called by
 // all threads of the CTA.
-__device__ __forceinline__ void grid_barrier_init(unsigned long long* word, uint32_t epoch)
+// Called by all threads; the last warp of CTA 0 does the work (the one most likely to have no token), the
+// rest of the CTA does not wait for it.
+__device__ __forceinline__ void grid_barrier_init(unsigned long long* word, uint32_t epoch, uint32_t* grid_sums,
+                                                  int n_words)
 {
-    if (blockIdx.x == 0 && threadIdx.x == 0) atomicExch(word, static_cast<unsigned long long>(epoch) << 32);
+    if (blockIdx.x != 0 || threadIdx.x < blockDim.x - 32) return;
+    const int lane = threadIdx.x & 31;
+    for (int i = lane; i < n_words; i += 32) grid_sums[i] = 0;
+    __syncwarp();
+    if (lane == 0) {
+        __threadfence();                   // the cleared words are visible before the epoch is
+        atomicExch(word, static_cast<unsigned long long>(epoch) << 32);
+    }
+}
+
+// Thread 0 of a CTA: has CTA 0 published this launch's epoch (and with it the cleared totals)?  `first`
+// is an earlier acquire load of the word, issued where its latency hides.  Bounded like the barrier's wait.
+__device__ __forceinline__ bool grid_epoch_seen(const unsigned long long* word, unsigned long long first, uint32_t epoch)
+{
+    if ((first >> 32) == epoch) return true;
+    for (uint32_t spin = 0; spin < kBarrierSpinLimit; ++spin) {
+        if ((ld_acquire_u64(word) >> 32) == epoch) return true;
+        __nanosleep(40);
+    }
+    return false;
 }
 
 // Arrival: the value the atomic returns is only looked at in grid_wait, so the arriving thread goes on
@@ -176,7 +203,8 @@ struct RouteParams {
     // workspace
     unsigned long long* barrier;
     uint16_t* ws_cnt;                  // [CTAs][dest_words], 16-bit: a CTA sends at most one pair per token to a destination
-    unsigned long long* ws_tot;        // [CTAs][2]
+    uint32_t* ws_dtot;                 // [dest_words] pairs per destination over the whole grid (atomic adds),
+                                       // then the two sums of Eq. 1 (64-bit each)
     uint32_t* ws_tri;                  // [CTAs][tri_words]
     uint32_t epoch;
     int tri_words, stage_words, tab_words, dest_words, lane_stride;
@@ -262,6 +290,7 @@ route_fused_kernel(const RouteParams p)
     uint32_t* pre = mask + kRouteWarps * p.lane_stride;        // [warps][lane_stride] the round's pairs to d in lower warps
     __shared__ unsigned long long cta_totals[2];
     __shared__ uint32_t warp_sums[kRouteWarps];
+    __shared__ int epoch_ok;
 
     constexpr int KMAX = TokenShape<KT>::KMAX;
     const int K = (KT > 0) ? KT : p.K_rt;
@@ -280,7 +309,6 @@ route_fused_kernel(const RouteParams p)
         seed_hi = static_cast<uint32_t>(sd >> 32);
     }
 
-    grid_barrier_init(p.barrier, p.epoch);
     const int64_t t_lo = min(p.T, static_cast<int64_t>(cta) * p.tokens_per_cta);
     const int64_t t_hi = min(p.T, t_lo + p.tokens_per_cta);
     const int n_rounds = static_cast<int>((t_hi - t_lo + kRouteThreads - 1) / kRouteThreads);
@@ -297,6 +325,7 @@ route_fused_kernel(const RouteParams p)
         load_token_ids<KT>(p.topk_ids, t_lo + tid, K, id);
         if (p.src_rank) s_t = __ldg(p.src_rank + t_lo + tid);
     }
+    grid_barrier_init(p.barrier, p.epoch, p.ws_dtot, dest_words + kGridSumWords);
     // the layout tables travel to shared memory asynchronously, behind the clearing of the other arrays
     {
         const uint4* src = reinterpret_cast<const uint4*>(p.lv.blob);
@@ -453,16 +482,26 @@ route_fused_kernel(const RouteParams p)
 
     // ---- publish this CTA's partial results ------------------------------------------------------
     // The triangle goes first (9.7 MB over the grid: the stores drain while the counts are worked out).
+    unsigned long long word_now = 0;
+    if (tid == 0) word_now = ld_acquire_u64(p.barrier);     // looked at below: has CTA 0 cleared the grid's totals?
     {
         uint4* dst = reinterpret_cast<uint4*>(p.ws_tri + static_cast<size_t>(cta) * p.tri_words);
         for (int v = tid; v < p.tri_words / 4; v += kRouteThreads) dst[v] = reinterpret_cast<const uint4*>(tri)[v];
     }
     if (single) count_round();               // cnt[d] from the lane masks
+    if (tid == 0) {
+        epoch_ok = grid_epoch_seen(p.barrier, word_now, p.epoch) ? 1 : 0;
+        if (!epoch_ok) flag_error(p.err_word, COBALT_DEVERR_WAIT_TIMEOUT);
+    }
     __syncthreads();
+    if (!epoch_ok) return;
     {
         uint32_t* dst_cnt = reinterpret_cast<uint32_t*>(p.ws_cnt + static_cast<size_t>(cta) * dest_words);
         for (int i = tid; i < dest_words / 2; i += kRouteThreads) dst_cnt[i] = cnt[2 * i] | (cnt[2 * i + 1] << 16);
-        if (p.totals && tid < 2) p.ws_tot[2 * cta + tid] = cta_totals[tid];
+        for (int d = tid; d < D; d += kRouteThreads)
+            if (cnt[d]) atomicAdd(p.ws_dtot + d, cnt[d]);
+        if (p.totals && tid < 2 && cta_totals[tid])
+            atomicAdd(reinterpret_cast<unsigned long long*>(p.ws_dtot + dest_words) + tid, cta_totals[tid]);
     }
     const unsigned long long arrived = grid_arrive(p.barrier);
     // between arrival and wait: what the ranks need from this CTA alone
@@ -486,27 +525,30 @@ route_fused_kernel(const RouteParams p)
     const int v0 = min(n_vec, cta * slice), v1 = min(n_vec, v0 + slice);
     const int n_mine = v1 - v0;
     const int n_acc = 4 * n_mine * kPerWord;                          // sums of the slice, 32 bits each
-    // 2b: the CTAs' counts are split over `parts` groups of threads; a thread sums eight consecutive
-    // destinations of its share of the CTAs and leaves its sums (all CTAs, lower CTAs) where the
-    // triangle was, behind the sums of the slice; one thread per destination adds them up.
+    // 2b: the pairs of the lower CTAs per destination.  The grid's totals are there already (atomic
+    // adds before the barrier), so a CTA of the lower half of the grid sums the counts of the CTAs below
+    // it and one of the upper half those from itself upwards, which it takes off the total: at most half
+    // of the CTAs' counts either way.  They are split over `parts` groups of threads; a thread sums eight
+    // consecutive destinations of its share of the CTAs and leaves its sums where the triangle was,
+    // behind the sums of the slice; one thread per destination adds them up.
+    const bool from_below = 2 * cta <= n_ctas;
+    const int c_begin = from_below ? 0 : cta, c_end = from_below ? cta : n_ctas;
     const int octs = dest_words / 8;
     int parts = max(1, kHalf / octs);
-    parts = min(parts, n_ctas);
-    if (parts > 1) parts = max(1, min(parts, (p.tri_words - n_acc) / (2 * dest_words)));
+    parts = min(parts, max(1, (n_ctas + 1) / 2));
+    if (parts > 1) parts = max(1, min(parts, (p.tri_words - n_acc) / dest_words));
     uint32_t* acc = tri;
-    uint32_t* part_all = tri + (n_acc + 3) / 4 * 4;                   // [parts][dest_words]
-    uint32_t* part_lower = part_all + parts * dest_words;             // [parts][dest_words]
-    if ((n_acc + 3) / 4 * 4 + 2 * parts * dest_words > p.tri_words) {   // a tiny triangle: one group, sums straight into cnt / base
+    uint32_t* part_sum = tri + (n_acc + 3) / 4 * 4;                   // [parts][dest_words]
+    if ((n_acc + 3) / 4 * 4 + parts * dest_words > p.tri_words) {     // a tiny triangle: one group, sums straight into base
         parts = 1;
-        part_all = cnt;
-        part_lower = base;
+        part_sum = base;
     }
     for (int i = tid; i < n_acc; i += kRouteThreads) acc[i] = 0;
     __syncthreads();
     if (tid >= kHalf) {
         // 2a: `groups` threads share a vector of the slice, each summing every groups-th partial in
         // registers (loads in flight together, lanes along consecutive vectors), then shared-memory adds
-        constexpr int kBatch = 5;
+        constexpr int kBatch = 9;
         const int ht = tid - kHalf;
         if (n_mine > 0) {
             const int groups = max(1, kHalf / n_mine);
@@ -542,48 +584,36 @@ route_fused_kernel(const RouteParams p)
                     if (sum[i]) atomicAdd(&acc[4 * kPerWord * v + i], sum[i]);
             }
         }
-        if (p.totals && cta == 0 && ht < 2) {
-            unsigned long long sum = 0;
-            for (int c = 0; c < n_ctas; ++c) sum += __ldcg(p.ws_tot + 2 * c + ht);
-            p.totals[ht] = sum;
-        }
+        if (p.totals && cta == 0 && ht < 2)
+            p.totals[ht] = __ldcg(reinterpret_cast<const unsigned long long*>(p.ws_dtot + dest_words) + ht);
     } else {
         constexpr int kBatch = 6;
         const int part = tid / octs, oct = tid - part * octs;
         if (part < parts) {
             const uint4* src = reinterpret_cast<const uint4*>(p.ws_cnt) + oct;
-            uint32_t all[8], lower[8];
+            uint32_t sum[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) all[i] = lower[i] = 0;
-            for (int c = part; c < n_ctas; c += parts * kBatch) {
+            for (int i = 0; i < 8; ++i) sum[i] = 0;
+            for (int c = c_begin + part; c < c_end; c += parts * kBatch) {
                 uint4 q[kBatch];
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int cc = c + u * parts;
-                    q[u] = (cc < n_ctas) ? __ldcg(src + static_cast<size_t>(cc) * octs) : make_uint4(0, 0, 0, 0);
+                    q[u] = (cc < c_end) ? __ldcg(src + static_cast<size_t>(cc) * octs) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
-                    const bool below = c + u * parts < cta;
                     const uint32_t word[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const uint32_t lo = word[i] & 0xFFFFu, hi = word[i] >> 16;
-                        all[2 * i] += lo;
-                        all[2 * i + 1] += hi;
-                        if (below) {
-                            lower[2 * i] += lo;
-                            lower[2 * i + 1] += hi;
-                        }
+                        sum[2 * i] += word[i] & 0xFFFFu;
+                        sum[2 * i + 1] += word[i] >> 16;
                     }
                 }
             }
-            uint4* dst_all = reinterpret_cast<uint4*>(part_all + part * dest_words + 8 * oct);
-            uint4* dst_lower = reinterpret_cast<uint4*>(part_lower + part * dest_words + 8 * oct);
-            dst_all[0] = make_uint4(all[0], all[1], all[2], all[3]);
-            dst_all[1] = make_uint4(all[4], all[5], all[6], all[7]);
-            dst_lower[0] = make_uint4(lower[0], lower[1], lower[2], lower[3]);
-            dst_lower[1] = make_uint4(lower[4], lower[5], lower[6], lower[7]);
+            uint4* dst = reinterpret_cast<uint4*>(part_sum + part * dest_words + 8 * oct);
+            dst[0] = make_uint4(sum[0], sum[1], sum[2], sum[3]);
+            dst[1] = make_uint4(sum[4], sum[5], sum[6], sum[7]);
         }
     }
     // (the two halves go on separately: each only waits for its own half until the rows are written)
@@ -608,18 +638,22 @@ route_fused_kernel(const RouteParams p)
             }
         }
     } else {
-        half_barrier(1);
         // 2b: totals over all CTAs, their exclusive scan over d (the offsets), first row of this CTA;
         // two consecutive destinations per thread
         uint32_t mine[2] = {0, 0}, lower[2] = {0, 0};
+        if (2 * tid < D) {                       // dest_words is even: the pair is inside the array
+            const uint2 both = __ldcg(reinterpret_cast<const uint2*>(p.ws_dtot) + tid);
+            mine[0] = both.x;
+            mine[1] = (2 * tid + 1 < D) ? both.y : 0u;
+        }
+        half_barrier(1);
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int d = 2 * tid + j;
             if (d < D) {
-                for (int g = 0; g < parts; ++g) {
-                    mine[j] += part_all[g * dest_words + d];
-                    lower[j] += part_lower[g * dest_words + d];
-                }
+                uint32_t s = 0;
+                for (int g = 0; g < parts; ++g) s += part_sum[g * dest_words + d];
+                lower[j] = from_below ? s : mine[j] - s;
             }
         }
         uint32_t total = 0;
@@ -780,7 +814,7 @@ static int launch_route(RouteArgs a, bool* launched)
     uint8_t* ws = static_cast<uint8_t*>(a.workspace);
     p.barrier = reinterpret_cast<unsigned long long*>(ws + w.barrier_off);
     p.ws_cnt = reinterpret_cast<uint16_t*>(ws + w.cnt_off);
-    p.ws_tot = reinterpret_cast<unsigned long long*>(ws + w.tot_off);
+    p.ws_dtot = reinterpret_cast<uint32_t*>(ws + w.dtot_off);
     p.ws_tri = reinterpret_cast<uint32_t*>(ws + w.tri_off);
     p.epoch = next_epoch();
 
