@@ -86,6 +86,13 @@ static RouteWorkspace route_workspace(const LayoutView& lv, bool packed)
     return w;
 }
 
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p)
 {
     unsigned long long v;
@@ -145,9 +152,10 @@ __device__ __forceinline__ unsigned long long grid_arrive(unsigned long long* wo
     return before;
 }
 
-// Returns false on a timeout.  `before` is what grid_arrive returned.
+// Returns false on a timeout.  `before` is what grid_arrive returned.  `*signed_off` (thread 0) receives
+// what the sign-off atomic returned; grid_leave looks at it when the CTA is done, so nobody waits for it.
 __device__ __forceinline__ bool grid_wait(unsigned long long* word, unsigned long long before, uint32_t epoch,
-                                          uint32_t n_ctas, uint32_t* err_word)
+                                          uint32_t n_ctas, uint32_t* err_word, unsigned long long* signed_off)
 {
     __shared__ int barrier_ok;
     if (threadIdx.x == 0) {
@@ -155,7 +163,7 @@ __device__ __forceinline__ bool grid_wait(unsigned long long* word, unsigned lon
         bool counted = (before >> 32) == epoch;
         bool ok = false;
         for (uint32_t spin = 0; spin < kBarrierSpinLimit; ++spin) {
-            const unsigned long long v = ld_acquire_u64(word);
+            const unsigned long long v = ld_relaxed_u64(word);
             if ((v >> 32) == epoch) {
                 if (!counted) {
                     counted = (atomicAdd(word, 1ull) >> 32) == epoch;
@@ -166,20 +174,21 @@ __device__ __forceinline__ bool grid_wait(unsigned long long* word, unsigned lon
                     break;
                 }
             }
-            __nanosleep(40);
+            if (spin >= 4096) __nanosleep(40);      // a barrier that is about to open is polled back to back
         }
-        if (ok) {
-            // sign off; the last CTA to do so leaves the word cleared
-            const unsigned long long old = atomicAdd(word, 1ull);
-            if (static_cast<uint32_t>(old) + 1u == 2u * n_ctas) atomicExch(word, 0ull);
-        } else {
-            flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
-        }
-        __threadfence();
+        __threadfence();                            // what the other CTAs published is read after this
+        if (ok) *signed_off = atomicAdd(word, 1ull);
+        else flag_error(err_word, COBALT_DEVERR_WAIT_TIMEOUT);
         barrier_ok = ok ? 1 : 0;
     }
     __syncthreads();
     return barrier_ok != 0;
+}
+
+// Thread 0, when the CTA is done: the last CTA to have signed off leaves the word cleared.
+__device__ __forceinline__ void grid_leave(unsigned long long* word, unsigned long long signed_off, uint32_t n_ctas)
+{
+    if (threadIdx.x == 0 && static_cast<uint32_t>(signed_off) + 1u == 2u * n_ctas) atomicExch(word, 0ull);
 }
 
 struct RouteParams {
@@ -325,7 +334,6 @@ route_fused_kernel(const RouteParams p)
         load_token_ids<KT>(p.topk_ids, t_lo + tid, K, id);
         if (p.src_rank) s_t = __ldg(p.src_rank + t_lo + tid);
     }
-    grid_barrier_init(p.barrier, p.epoch, p.ws_dtot, dest_words + kGridSumWords);
     // the layout tables travel to shared memory asynchronously, behind the clearing of the other arrays
     {
         const uint4* src = reinterpret_cast<const uint4*>(p.lv.blob);
@@ -345,6 +353,7 @@ route_fused_kernel(const RouteParams p)
     const TableView tv = table_view(p.lv, tab);
     asm volatile("cp.async.wait_all;" ::: "memory");      // the tables have arrived behind the clearing
     __syncthreads();
+    grid_barrier_init(p.barrier, p.epoch, p.ws_dtot, dest_words + kGridSumWords);   // no CTA looks before it publishes
 
     // ---- phase 1: statistics, Algorithm 1, destination counts ---------------------------------
     uint32_t cost_sum = 0, naive_sum = 0;
@@ -403,48 +412,32 @@ route_fused_kernel(const RouteParams p)
     }
     __syncthreads();
 
-    // Per destination, the pairs of the lower warps of a round (and the round's pairs in all): one warp
-    // per destination, lane w holding the pairs of warp w, an exclusive scan across the lanes.  The odd
-    // stride of the table keeps the lanes on different banks.  Needs the lane masks of the round.
-    auto count_round = [&]() {
-        // two destinations share a scan (16-bit halves: a warp sends at most 32 pairs to a destination, a
-        // round at most 1024), and two such scans are in flight per iteration
-        for (int d0 = warp; d0 < D; d0 += 4 * kRouteWarps) {
-            uint32_t c[2], incl[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
-                const uint32_t ca = (da < D) ? __popc(mask[lane * p.lane_stride + da]) : 0u;
-                const uint32_t cb = (db < D) ? __popc(mask[lane * p.lane_stride + db]) : 0u;
-                c[h] = ca | (cb << 16);
-                incl[h] = c[h];
-            }
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl[h], off);
-                    if (lane >= off) incl[h] += up;
-                }
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int da = d0 + 2 * h * kRouteWarps, db = da + kRouteWarps;
-                const uint32_t before = incl[h] - c[h];
-                if (da < D) {
-                    pre[lane * p.lane_stride + da] = before & 0xFFFFu;
-                    if (lane == 31) cnt[da] = incl[h] & 0xFFFFu;
-                }
-                if (db < D) {
-                    pre[lane * p.lane_stride + db] = before >> 16;
-                    if (lane == 31) cnt[db] = incl[h] >> 16;
-                }
+    // The ranks of a round's pairs come from the lane masks in three steps.  (1) count_dests: thread d
+    // adds up the pairs the 32 warps send to destination d (consecutive threads, consecutive words: no
+    // bank conflicts).  (2) A scan of those counts over d gives the place of d's first pair in the round's
+    // destination-major order, and prefix_dests walks down the warps once more and leaves in pre[w][d] the
+    // place of warp w's first pair to d.  (3) rank_round: a pair's place is pre[w][d] plus the lower lanes
+    // of its warp that send to d; the pair goes into the staged inverse map at that place, and the place
+    // (packed with d into out[], -1 for a pair without a destination) is kept for write_round.
+    auto count_dests = [&]() -> uint32_t {
+        uint32_t sum = 0;
+        if (tid < D) {
+#pragma unroll 8
+            for (int w = 0; w < kRouteWarps; ++w) sum += __popc(mask[w * p.lane_stride + tid]);
+        }
+        return sum;
+    };
+    auto prefix_dests = [&](uint32_t first) {
+        if (tid < D) {
+            uint32_t run = first;
+#pragma unroll 8
+            for (int w = 0; w < kRouteWarps; ++w) {
+                const uint32_t c = __popc(mask[w * p.lane_stride + tid]);
+                pre[w * p.lane_stride + tid] = run;
+                run += c;
             }
         }
     };
-    // The rank of each of the thread's pairs inside its destination among the pairs of the round (packed
-    // with the destination into out[], -1 for a pair without one), and the pair's entry in the staged
-    // inverse map.  Needs count_round and the scan of its counts over d (excl).
     auto rank_round = [&](bool has_token) {
         if (!has_token) return;
 #pragma unroll
@@ -452,30 +445,29 @@ route_fused_kernel(const RouteParams p)
             if (a < K && out[a] >= 0) {
                 const uint32_t d = static_cast<uint32_t>(out[a]);
                 const uint32_t r = my_pre[d] + __popc(my_mask[d] & lower_lanes);
-                if (p.pair_of_row) stage[excl[d] + r] = d | (static_cast<uint32_t>(tid * K + a) << kDestBits);
+                if (p.pair_of_row) stage[r] = d | (static_cast<uint32_t>(tid * K + a) << kDestBits);
                 out[a] = static_cast<int32_t>(d | (r << kDestBits));
             }
         }
     };
-    // Rows of the thread's pairs (the rank of rank_round on top of the first row of the round's pairs
-    // inside the destination), and the round's part of the inverse map in row order: consecutive
-    // threads write consecutive rows of a destination.
-    auto write_round = [&](bool has_token, int64_t t_round, uint32_t round_pairs) {
+    // Rows of the thread's pairs and the round's part of the inverse map in row order (consecutive
+    // threads write consecutive rows of a destination): a pair's row is its place in the round plus
+    // shift[d], the first row of the round's pairs inside d minus the place of the first of them.
+    auto write_round = [&](bool has_token, int64_t t_round, uint32_t round_pairs, const uint32_t* shift) {
         if (has_token) {
             int32_t row[KMAX];
 #pragma unroll
             for (int a = 0; a < KMAX; ++a) {
                 row[a] = -1;
                 if (a < K && out[a] >= 0)
-                    row[a] = static_cast<int32_t>(base[out[a] & ((1 << kDestBits) - 1)] + (static_cast<uint32_t>(out[a]) >> kDestBits));
+                    row[a] = static_cast<int32_t>(shift[out[a] & ((1 << kDestBits) - 1)] + (static_cast<uint32_t>(out[a]) >> kDestBits));
             }
             store_token_slots<KT>(p.row_of_pair + (t_round + tid) * K, row, K);
         }
         if (p.pair_of_row) {
             for (uint32_t j = tid; j < round_pairs; j += kRouteThreads) {
                 const uint32_t v = stage[j];
-                const uint32_t d = v & ((1u << kDestBits) - 1u);
-                p.pair_of_row[base[d] + (j - excl[d])] = static_cast<int32_t>(t_round * K + (v >> kDestBits));
+                p.pair_of_row[shift[v & ((1u << kDestBits) - 1u)] + j] = static_cast<int32_t>(t_round * K + (v >> kDestBits));
             }
         }
     };
@@ -488,31 +480,36 @@ route_fused_kernel(const RouteParams p)
         uint4* dst = reinterpret_cast<uint4*>(p.ws_tri + static_cast<size_t>(cta) * p.tri_words);
         for (int v = tid; v < p.tri_words / 4; v += kRouteThreads) dst[v] = reinterpret_cast<const uint4*>(tri)[v];
     }
-    if (single) count_round();               // cnt[d] from the lane masks
+    // this CTA's pairs to destination tid: from the lane masks (one round) or as counted in phase 1
+    uint32_t my_cnt = 0, first_place = 0, round_pairs = 0;
+    if (single) my_cnt = count_dests();
+    else if (tid < D) my_cnt = cnt[tid];
     if (tid == 0) {
         epoch_ok = grid_epoch_seen(p.barrier, word_now, p.epoch) ? 1 : 0;
         if (!epoch_ok) flag_error(p.err_word, COBALT_DEVERR_WAIT_TIMEOUT);
     }
-    __syncthreads();
+    if (single) first_place = block_exclusive_scan(my_cnt, warp_sums, &round_pairs);
+    else __syncthreads();
     if (!epoch_ok) return;
     {
-        uint32_t* dst_cnt = reinterpret_cast<uint32_t*>(p.ws_cnt + static_cast<size_t>(cta) * dest_words);
-        for (int i = tid; i < dest_words / 2; i += kRouteThreads) dst_cnt[i] = cnt[2 * i] | (cnt[2 * i + 1] << 16);
-        for (int d = tid; d < D; d += kRouteThreads)
-            if (cnt[d]) atomicAdd(p.ws_dtot + d, cnt[d]);
+        // 16-bit counts, two to a word: the even thread takes its neighbour's along
+        const uint32_t next_cnt = __shfl_down_sync(0xFFFFFFFFu, my_cnt, 1);
+        if (!(tid & 1) && tid < dest_words)
+            reinterpret_cast<uint32_t*>(p.ws_cnt + static_cast<size_t>(cta) * dest_words)[tid >> 1] = my_cnt | (next_cnt << 16);
+        if (my_cnt) atomicAdd(p.ws_dtot + tid, my_cnt);
         if (p.totals && tid < 2 && cta_totals[tid])
             atomicAdd(reinterpret_cast<unsigned long long*>(p.ws_dtot + dest_words) + tid, cta_totals[tid]);
     }
-    const unsigned long long arrived = grid_arrive(p.barrier);
-    // between arrival and wait: what the ranks need from this CTA alone
-    uint32_t round_pairs = 0;
+    // what the ranks need from this CTA alone: the prefixes before the arrival (the additions above travel
+    // meanwhile), the ranks between arrival and wait
     if (single) {
-        const uint32_t lower_dests = block_exclusive_scan((tid < D) ? cnt[tid] : 0u, warp_sums, &round_pairs);
-        if (tid < D) excl[tid] = lower_dests;
-        __syncthreads();
-        rank_round(t_lo + tid < t_hi);
+        prefix_dests(first_place);
+        if (tid < D) excl[tid] = first_place;
     }
-    if (!grid_wait(p.barrier, arrived, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word)) return;
+    const unsigned long long arrived = grid_arrive(p.barrier);
+    if (single) rank_round(t_lo + tid < t_hi);
+    unsigned long long signed_off = 0;
+    if (!grid_wait(p.barrier, arrived, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word, &signed_off)) return;
 
     // ---- phase 2a and 2b side by side: both wait on loads of what the other CTAs published, so the
     // upper half of the CTA's warps sums this CTA's slice of the triangle over all partials (2a) while
@@ -667,7 +664,8 @@ route_fused_kernel(const RouteParams p)
                     p.dest_counts[d] = mine[j];
                     p.dest_offsets[d] = before;
                 }
-                base[d] = before + lower[j];
+                // one round: its pairs' places are known already, so what is kept is the shift from place to row
+                base[d] = before + lower[j] - (single ? excl[d] : 0u);
             }
             before += mine[j];
         }
@@ -677,7 +675,8 @@ route_fused_kernel(const RouteParams p)
 
     // ---- phase 2c: rows of this CTA's pairs ------------------------------------------------------
     if (single) {
-        write_round(t_lo + tid < t_hi, t_lo, round_pairs);
+        write_round(t_lo + tid < t_hi, t_lo, round_pairs, base);
+        grid_leave(p.barrier, signed_off, static_cast<uint32_t>(n_ctas));
         return;
     }
     for (int round = 0; round < n_rounds; ++round) {
@@ -703,11 +702,10 @@ route_fused_kernel(const RouteParams p)
                 if (a < K && out[a] >= 0) atomicOr(&my_mask[out[a]], 1u << lane);
         }
         __syncthreads();
-        count_round();
-        __syncthreads();
-        const uint32_t round_total = (tid < D) ? cnt[tid] : 0u;
-        const uint32_t lower_dests = block_exclusive_scan(round_total, warp_sums, &round_pairs);
-        if (tid < D) excl[tid] = lower_dests;
+        const uint32_t round_total = count_dests();
+        const uint32_t round_first = block_exclusive_scan(round_total, warp_sums, &round_pairs);
+        prefix_dests(round_first);
+        if (tid < D) excl[tid] = base[tid] - round_first;        // the round's shift from place to row
         // the masks are cleared through the still unpacked slots before rank_round packs them
         __syncthreads();
         uint32_t touched[KMAX];
@@ -715,7 +713,7 @@ route_fused_kernel(const RouteParams p)
         for (int a = 0; a < KMAX; ++a) touched[a] = (has_token && a < K && out[a] >= 0) ? static_cast<uint32_t>(out[a]) : 0xFFFFFFFFu;
         rank_round(has_token);
         __syncthreads();
-        write_round(has_token, t_round, round_pairs);
+        write_round(has_token, t_round, round_pairs, excl);
         __syncthreads();
 #pragma unroll
         for (int a = 0; a < KMAX; ++a)
@@ -723,6 +721,7 @@ route_fused_kernel(const RouteParams p)
         if (tid < D) base[tid] += round_total;
         __syncthreads();
     }
+    grid_leave(p.barrier, signed_off, static_cast<uint32_t>(n_ctas));
 }
 
 // The grid the device can hold for this kernel and shared-memory size (one CTA per SM in practice),
