@@ -9,12 +9,13 @@
 //   phase 1  every CTA owns a contiguous range of tokens, one token per thread and round: the
 //            token's K(K+1)/2 pairs go into the CTA's private co-activation triangle in shared
 //            memory, Algorithm 1 picks its K slots (stored, and counted per destination).
-//   publish  the CTA writes its triangle, its destination counts and its Eq. 1 sums to the
-//            workspace (plain coalesced stores).  Then ONE grid-wide barrier (bounded wait).
+//   publish  the CTA writes its triangle and its destination counts to the workspace (plain
+//            coalesced stores) and adds the counts and its Eq. 1 sums to grid-wide totals there
+//            (atomic adds).  Then ONE grid-wide barrier (bounded wait).
 //   phase 2  every CTA sums a slice of the triangle over all CTAs' partials and STORES coact / load
-//            (no atomics on the outputs, nothing to clear beforehand); it derives, from all CTAs'
-//            destination counts, the offsets and the first row of its own tokens inside every
-//            destination; and ranks its pairs.  A token sends at most one pair to a destination
+//            (no atomics on the outputs, nothing to clear beforehand); it derives, from the totals
+//            and from the counts of at most half of the other CTAs, the offsets and the first row
+//            of its own tokens inside every destination; and ranks its pairs.  A token sends at most one pair to a destination
 //            (its experts, hence its slots, are distinct), so the rows of one destination inside a
 //            warp's 32 tokens are ordered by lane: each lane ORs its bit into a per-destination lane
 //            mask, and a pair's rank is the popcount of the lower lanes -- no sorting, no position
