@@ -103,17 +103,17 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 
 // Grid-wide barrier on one 64-bit word of the workspace: epoch (high half) and arrival count.
 // The word may hold anything when the kernel starts.  CTA 0 sets it to (epoch, 0) once it has cleared
-// the grid-wide destination totals; a CTA adds to those totals only after it has seen the epoch
-// (grid_epoch_seen), so its additions cannot be lost to the clearing.  A CTA arrives by adding one and
-// learns from the value it gets back whether the word already carried this launch's epoch.  If not, it
-// waits for the epoch to appear and adds again.  Every CTA of the grid is
+// the grid-wide totals; a CTA adds to those totals, and arrives, only after it has seen the epoch
+// (grid_epoch_seen), so neither can be lost to the clearing.  Arrival is one atomic add; the wait polls
+// until the count reaches the number of CTAs.  Every CTA of the grid is
 // resident (cooperative launch), so the wait ends as soon as the slowest CTA has arrived; it is
 // bounded all the same, and a wait that runs out reports COBALT_DEVERR_WAIT_TIMEOUT and makes the
 // CTA return.  After the wait every CTA signs off on the same word and the last one clears it, so
 // that a replay of a captured launch (same epoch) starts from a word that differs from its epoch.
 // Arrival and wait are separate calls (work that needs no other CTA goes in between); all are called by
 // all threads of the CTA.
-// Called by all threads; the last warp of CTA 0 does the work (the one most likely to have no token), the
+//
+// grid_barrier_init: the last warp of CTA 0 does the work (the one most likely to have no token), the
 // rest of the CTA does not wait for it.
 __device__ __forceinline__ void grid_barrier_init(unsigned long long* word, uint32_t epoch, uint32_t* grid_sums,
                                                   int n_words)
@@ -140,40 +140,31 @@ __device__ __forceinline__ bool grid_epoch_seen(const unsigned long long* word, 
     return false;
 }
 
-// Arrival: the value the atomic returns is only looked at in grid_wait, so the arriving thread goes on
-// with whatever lies between the two calls while the atomic travels.
-__device__ __forceinline__ unsigned long long grid_arrive(unsigned long long* word)
+// Arrival (after grid_epoch_seen): nothing comes back, so the arriving thread goes on with whatever lies
+// between this call and the wait while the atomic travels.
+__device__ __forceinline__ void grid_arrive(unsigned long long* word)
 {
-    unsigned long long before = 0;
     __syncthreads();                       // this CTA's writes are done ...
     if (threadIdx.x == 0) {
         __threadfence();                   // ... and visible to the grid before the arrival is
-        before = atomicAdd(word, 1ull);
+        atomicAdd(word, 1ull);
     }
-    return before;
 }
 
-// Returns false on a timeout.  `before` is what grid_arrive returned.  `*signed_off` (thread 0) receives
-// what the sign-off atomic returned; grid_leave looks at it when the CTA is done, so nobody waits for it.
-__device__ __forceinline__ bool grid_wait(unsigned long long* word, unsigned long long before, uint32_t epoch,
-                                          uint32_t n_ctas, uint32_t* err_word, unsigned long long* signed_off)
+// Returns false on a timeout.  `*signed_off` (thread 0) receives what the sign-off atomic returned;
+// grid_leave looks at it when the CTA is done, so nobody waits for it.
+__device__ __forceinline__ bool grid_wait(unsigned long long* word, uint32_t epoch, uint32_t n_ctas, uint32_t* err_word,
+                                          unsigned long long* signed_off)
 {
     __shared__ int barrier_ok;
     if (threadIdx.x == 0) {
         const unsigned long long target = (static_cast<unsigned long long>(epoch) << 32) | n_ctas;
-        bool counted = (before >> 32) == epoch;
         bool ok = false;
         for (uint32_t spin = 0; spin < kBarrierSpinLimit; ++spin) {
             const unsigned long long v = ld_relaxed_u64(word);
-            if ((v >> 32) == epoch) {
-                if (!counted) {
-                    counted = (atomicAdd(word, 1ull) >> 32) == epoch;
-                    continue;
-                }
-                if (v >= target) {
-                    ok = true;
-                    break;
-                }
+            if ((v >> 32) == epoch && v >= target) {
+                ok = true;
+                break;
             }
             if (spin >= 4096) __nanosleep(40);      // a barrier that is about to open is polled back to back
         }
@@ -507,10 +498,10 @@ route_fused_kernel(const RouteParams p)
         prefix_dests(first_place);
         if (tid < D) excl[tid] = first_place;
     }
-    const unsigned long long arrived = grid_arrive(p.barrier);
+    grid_arrive(p.barrier);
     if (single) rank_round(t_lo + tid < t_hi);
     unsigned long long signed_off = 0;
-    if (!grid_wait(p.barrier, arrived, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word, &signed_off)) return;
+    if (!grid_wait(p.barrier, p.epoch, static_cast<uint32_t>(n_ctas), p.err_word, &signed_off)) return;
 
     // ---- phase 2a and 2b side by side: both wait on loads of what the other CTAs published, so the
     // upper half of the CTA's warps sums this CTA's slice of the triangle over all partials (2a) while
