@@ -282,13 +282,15 @@ route_fused_kernel(const RouteParams p)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t* tri = smem;                                      // later: acc (phase 2a), part (phase 2b)
-    uint32_t* stage = tri + p.tri_words;                       // [1024 K] the inverse map of one round, in row order
+    uint32_t* stage = tri + p.tri_words;                       // [1024 K] the pairs of one round by place (destination-major)
     uint32_t* tab = stage + p.stage_words;
-    uint32_t* cnt = tab + p.tab_words;                         // [D] pairs of this CTA (round) per destination
-    uint32_t* base = cnt + p.dest_words;                       // [D] first row of this CTA's (round's) pairs inside d
-    uint32_t* excl = base + p.dest_words;                      // [D] pairs of this round in lower destinations
+    uint32_t* cnt = tab + p.tab_words;                         // [D] pairs of this CTA per destination (several rounds only)
+    uint32_t* base = cnt + p.dest_words;                       // [D] first row of the CTA's (round's) pairs inside d; with
+                                                               // one round: that minus the place of the first of them
+    uint32_t* excl = base + p.dest_words;                      // [D] place of d's first pair (one round); several rounds:
+                                                               // the round's shift from place to row
     uint32_t* mask = excl + p.dest_words;                      // [warps][lane_stride] lanes (tokens) of the warp that send to d
-    uint32_t* pre = mask + kRouteWarps * p.lane_stride;        // [warps][lane_stride] the round's pairs to d in lower warps
+    uint32_t* pre = mask + kRouteWarps * p.lane_stride;        // [warps][lane_stride] place of the warp's first pair to d
     __shared__ unsigned long long cta_totals[2];
     __shared__ uint32_t warp_sums[kRouteWarps];
     __shared__ int epoch_ok;
