@@ -379,6 +379,22 @@ def test_fused_pass_starts_from_any_workspace_contents_and_runs_beside_itself(cb
     for st in (step, other):
         for k, v in ref.items():
             assert torch.equal(getattr(st, k), v), k
+    # many calls in a row, the workspace (barrier word and grid totals included) and the outputs filled with
+    # random bytes every few calls: every output is stored anew by every call
+    ref["load"], ref["dest_counts"], ref["totals"] = step.load.clone(), step.dest_counts.clone(), step.totals.clone()
+    for it in range(300):
+        if it % 7 == 0:
+            step.workspace.view(torch.uint8).random_(0, 256)
+        if it % 11 == 0:
+            for k in ref:
+                getattr(step, k).view(torch.uint8).random_(0, 256)
+        cb.route_index(step.layout, step.topk_ids, step.src_rank, 99, step.coact, step.load, step.assigned_slot,
+                       step.dest_counts, step.dest_offsets, step.row_of_pair, step.workspace,
+                       remote_nodes=step.remote_nodes, totals=step.totals, pair_of_row=step.pair_of_row)
+        if it % 10 == 0 or it == 299:
+            for k, v in ref.items():
+                assert torch.equal(getattr(step, k), v), (it, k)
+    assert cb.read_and_clear_device_error() == 0
 
 
 def test_step_with_statistics_on_a_side_stream(cb):
